@@ -1,0 +1,423 @@
+"""Plain CPU checker for KV-block swap, copy-budget consumption and paged decode attention.
+
+TEST INFRASTRUCTURE ONLY.  Nothing in the product path may import this module: it exists so that
+the tests, the smoke check and the benchmark's CPU-baseline leg have an independent, slow,
+obviously-correct statement of what the hot path computes.  It shares no code with the CUDA
+library and imports nothing from it.
+
+What it follows (ProServe, Section 4.3 "Efficient Block Management", and Appendix B):
+
+* Eviction spills a request's KV blocks to host memory instead of dropping them; the device
+  blocks can be reclaimed only after the transfer has completed ("Asynchronous Offloading").
+  -> `swap_out` copies the blocks byte for byte into a host image; `reap` gives the blocks back.
+* A readmitted request gets its KV restored layer by layer ("Pipelined Reloading"; Appendix B:
+  one completion event per layer chunk).  -> `swap_in_begin`, `swap_in_layer`.
+* A per-step host-to-device copy budget B_copy (in blocks) is consumed in queue order at request
+  granularity: all missing blocks b_miss of a request if they fit, otherwise a partial copy with
+  the residual budget ("Put it Together", Alg. 1 lines 17 and 22-25).  -> `step_plan`, `step`.
+  The beta admission test of that paragraph depends on the scheduler's computable-token count and
+  is not modelled: a partial copy is always allowed and a request decodes only once complete.
+* The computation the reload overlaps with is the decode forward; its KV-consuming part is
+  attention over the paged cache.  The paper gives no formula; the textbook definition
+  softmax(q K^T / sqrt(d)) V is used, in float64, over KV gathered through the block table.
+
+Parity pins (tests/test_oracle_*.py): brute-force loops on tiny inputs, torch's own fp64
+scaled-dot-product attention on contiguous KV, scipy's logsumexp, closed forms (one token, equal
+keys, two-token sigmoid mix), masking and permutation invariants, hand-worked budget schedules,
+round-trip and ownership invariants.  No function here is "parity unpinned".
+
+Layouts (this build's reading; the paper is silent): per layer a K pool and a V pool,
+uint16[num_blocks][S][Hkv][D] holding bf16 bit patterns; host image of a request
+uint16[L][n_blk][2][S][Hkv][D] (layer-major, K slab then V slab per block).
+"""
+from __future__ import annotations
+
+import math
+from collections import deque
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+# status codes (same numeric contract as the C header; restated here, not imported)
+OK = 0
+ERR_INVALID = -1
+ERR_NOMEM = -2
+ERR_HOST_NOMEM = -3
+ERR_STATE = -4
+ERR_BUSY = -5
+
+# request states
+ST_RESIDENT = 1
+ST_SWAPPING_OUT = 2
+ST_HOST = 3
+ST_SWAPPING_IN = 4
+
+
+def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
+    """Exact value of bfloat16 bit patterns as float64 (bf16 is the top half of a float32)."""
+    u = np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    return u.view(np.float32).astype(np.float64)
+
+
+class _Req:
+    __slots__ = ("n_tokens", "table", "state", "image", "image_bytes", "layer_done", "old_table")
+
+    def __init__(self):
+        self.n_tokens = 0
+        self.table: List[int] = []
+        self.state = ST_RESIDENT
+        self.image: Optional[np.ndarray] = None
+        self.image_bytes = 0
+        self.layer_done: List[int] = []
+        self.old_table: List[int] = []
+
+
+class PsOracle:
+    def __init__(self, num_layers: int, num_kv_heads: int, num_q_heads: int, head_dim: int, block_size: int,
+                 num_gpu_blocks: int, initial_free_order: Optional[Sequence[int]] = None,
+                 kpool: Optional[np.ndarray] = None, vpool: Optional[np.ndarray] = None,
+                 host_pool_bytes: Optional[int] = None):
+        self.L, self.Hkv, self.Hq, self.D, self.S = num_layers, num_kv_heads, num_q_heads, head_dim, block_size
+        self.num_blocks = num_gpu_blocks
+        assert num_q_heads % num_kv_heads == 0
+        self.G = num_q_heads // num_kv_heads
+        order = list(range(num_gpu_blocks)) if initial_free_order is None else [int(v) for v in initial_free_order]
+        assert sorted(order) == list(range(num_gpu_blocks)), "initial_free_order must be a permutation"
+        # the stack's top is its last element; order[0] is handed out first
+        self.free: List[int] = order[::-1]
+        self.reqs: Dict[int, _Req] = {}
+        self.K = kpool
+        self.V = vpool
+        if kpool is not None:
+            want = (self.L, self.num_blocks, self.S, self.Hkv, self.D)
+            assert kpool.shape == want and vpool.shape == want and kpool.dtype == np.uint16
+        self.out_fifo: deque = deque()       # swap-outs whose blocks are not yet reclaimed, issue order
+        self.in_fifo: deque = deque()        # reload queue, issue order
+        self.host_pool_bytes = host_pool_bytes
+        self.host_used = 0
+
+    # ------------------------------------------------------------------ sizes
+    @property
+    def block_bytes(self) -> int:
+        """Bytes of one block across all layers (K and V): the copy budget's unit."""
+        return self.L * 2 * self.S * self.Hkv * self.D * 2
+
+    def blocks_for(self, n_tokens: int) -> int:
+        return -(-n_tokens // self.S)
+
+    # ------------------------------------------------------------------ allocation
+    def kv_alloc(self, req: int, n_tokens_total: int) -> int:
+        """Grow request `req` to hold n_tokens_total tokens; all-or-nothing; pops ids one at a time."""
+        if n_tokens_total < 0:
+            return ERR_INVALID
+        r = self.reqs.get(req)
+        if r is not None and r.state != ST_RESIDENT:
+            return ERR_STATE
+        have = 0 if r is None else len(r.table)
+        if r is not None and n_tokens_total < r.n_tokens:
+            return ERR_INVALID
+        need = self.blocks_for(n_tokens_total) - have
+        if need > len(self.free):
+            return ERR_NOMEM
+        if r is None:
+            r = self.reqs[req] = _Req()
+        for _ in range(need):
+            r.table.append(self.free.pop())
+        r.n_tokens = n_tokens_total
+        return OK
+
+    def kv_free(self, req: int) -> int:
+        r = self.reqs.get(req)
+        if r is None:
+            return ERR_INVALID
+        if r.state in (ST_SWAPPING_OUT, ST_SWAPPING_IN):
+            return ERR_BUSY
+        if r.state == ST_RESIDENT:
+            self.free.extend(r.table)            # pushed in table order: last entry ends on top
+        else:
+            self._release_image(r)
+        del self.reqs[req]
+        return OK
+
+    def block_table(self, req: int) -> Tuple[List[int], int]:
+        r = self.reqs[req]
+        return list(r.table), r.state
+
+    def num_free_blocks(self) -> int:
+        return len(self.free)
+
+    # ------------------------------------------------------------------ swap-out
+    def _image_bytes(self, n_blk: int) -> int:
+        return n_blk * self.block_bytes
+
+    def _release_image(self, r: _Req) -> None:
+        self.host_used -= r.image_bytes
+        r.image_bytes = 0
+        r.image = None
+
+    def swap_out(self, req: int) -> int:
+        """Spill the request's blocks to a host image; blocks stay owned until `reap`."""
+        r = self.reqs.get(req)
+        if r is None:
+            return ERR_INVALID
+        if r.state != ST_RESIDENT:
+            return ERR_STATE
+        n = len(r.table)
+        if self.host_pool_bytes is not None and self.host_used + self._image_bytes(n) > self.host_pool_bytes:
+            return ERR_HOST_NOMEM
+        r.image_bytes = self._image_bytes(n)
+        self.host_used += r.image_bytes
+        if self.K is not None:
+            img = np.empty((self.L, n, 2, self.S, self.Hkv, self.D), dtype=np.uint16)
+            for l in range(self.L):
+                for j, b in enumerate(r.table):
+                    img[l, j, 0] = self.K[l, b]
+                    img[l, j, 1] = self.V[l, b]
+            r.image = img
+        r.state = ST_SWAPPING_OUT
+        self.out_fifo.append(req)
+        return OK
+
+    def reap(self, count: Optional[int] = None) -> int:
+        """Transfers complete in issue order; give the blocks of the first `count` back (all if None)."""
+        done = 0
+        while self.out_fifo and (count is None or done < count):
+            r = self.reqs[self.out_fifo.popleft()]
+            self.free.extend(r.table)
+            r.old_table = r.table
+            r.table = []
+            r.state = ST_HOST
+            done += 1
+        return done
+
+    # ------------------------------------------------------------------ swap-in
+    def swap_in_begin(self, req: int) -> int:
+        """Queue a host-resident request for reload and give it fresh blocks (all-or-nothing)."""
+        r = self.reqs.get(req)
+        if r is None:
+            return ERR_INVALID
+        if r.state != ST_HOST:
+            return ERR_STATE
+        n = self.blocks_for(r.n_tokens)
+        if n > len(self.free):
+            return ERR_NOMEM
+        r.table = [self.free.pop() for _ in range(n)]
+        r.layer_done = [0] * self.L
+        r.state = ST_SWAPPING_IN
+        self.in_fifo.append(req)
+        return OK
+
+    def swap_in_cancel(self, req: int) -> int:
+        """Withdraw a queued reload that has not started; the fresh blocks go back in table order."""
+        r = self.reqs.get(req)
+        if r is None:
+            return ERR_INVALID
+        if r.state != ST_SWAPPING_IN:
+            return ERR_STATE
+        if any(r.layer_done):
+            return ERR_BUSY
+        self.free.extend(r.table)
+        r.table = []
+        r.state = ST_HOST
+        self.in_fifo.remove(req)
+        return OK
+
+    def swap_in_layer(self, req: int, layer: int, blk_lo: int, blk_hi: int) -> int:
+        """Restore logical blocks [blk_lo, blk_hi) of one layer from the host image into the fresh blocks."""
+        r = self.reqs.get(req)
+        if r is None:
+            return ERR_INVALID
+        if r.state != ST_SWAPPING_IN:
+            return ERR_STATE
+        n = len(r.table)
+        if not (0 <= layer < self.L) or not (0 <= blk_lo <= blk_hi <= n) or blk_lo != r.layer_done[layer]:
+            return ERR_INVALID
+        if self.K is not None:
+            for j in range(blk_lo, blk_hi):
+                b = r.table[j]
+                self.K[layer, b] = r.image[layer, j, 0]
+                self.V[layer, b] = r.image[layer, j, 1]
+        r.layer_done[layer] = blk_hi
+        if all(d == n for d in r.layer_done):
+            r.state = ST_RESIDENT
+            self._release_image(r)
+            r.old_table = []
+            self.in_fifo.remove(req)
+        return OK
+
+    # ------------------------------------------------------------------ copy budget
+    def missing_blocks(self, req: int) -> int:
+        """b_miss of Section 4.3: blocks on host that are not yet on the device."""
+        r = self.reqs[req]
+        if r.state != ST_SWAPPING_IN:
+            return 0
+        return len(r.table) - min(r.layer_done)
+
+    def step_plan(self, copy_budget_bytes: int) -> List[Tuple[int, int, int]]:
+        """Consume the budget over the reload queue in order; returns (req, blk_lo, blk_hi) per request.
+
+        Budget in blocks = floor(bytes / block_bytes) with a block spanning all layers; negative
+        means unlimited.  A request whose missing blocks fit is copied whole, otherwise it gets
+        what is left and the round ends.
+        """
+        left = None if copy_budget_bytes < 0 else copy_budget_bytes // self.block_bytes
+        plan = []
+        for req in self.in_fifo:
+            r = self.reqs[req]
+            lo = min(r.layer_done)
+            miss = len(r.table) - lo
+            if miss == 0:
+                continue
+            take = miss if left is None else min(miss, left)
+            if take == 0:
+                break
+            plan.append((req, lo, lo + take))
+            if left is not None:
+                left -= take
+                if left == 0:
+                    break
+        return plan
+
+    def step(self, copy_budget_bytes: int, reqs: Optional[Sequence[int]] = None,
+             q_bits: Optional[np.ndarray] = None):
+        """One engine step: reload under the budget (every layer), then decode the complete requests.
+
+        Returns (plan, decoded mask, out) with out float64 [L][B][Hq][D] (rows of requests that
+        did not decode are NaN) or None when no queries were given.
+        """
+        plan = self.step_plan(copy_budget_bytes)
+        for req, lo, hi in plan:
+            for l in range(self.L):
+                rc = self.swap_in_layer(req, l, lo, hi)
+                assert rc == OK, rc
+        if reqs is None:
+            return plan, None, None
+        mask = [1 if (q in self.reqs and self.reqs[q].state == ST_RESIDENT) else 0 for q in reqs]
+        out = None
+        if q_bits is not None:
+            out = np.full((self.L, len(reqs), self.Hq, self.D), np.nan)
+            live = [i for i, m in enumerate(mask) if m]
+            for l in range(self.L):
+                if live:
+                    o, _ = self.decode_attn(l, q_bits[l][live], [reqs[i] for i in live])
+                    out[l, live] = o
+        return plan, mask, out
+
+    # ------------------------------------------------------------------ attention
+    def gather_kv(self, layer: int, req: int) -> Tuple[np.ndarray, np.ndarray]:
+        """Contiguous K, V of a request for one layer: float64 [ctx][Hkv][D]."""
+        r = self.reqs[req]
+        ks = np.concatenate([self.K[layer, b] for b in r.table], axis=0)[: r.n_tokens]
+        vs = np.concatenate([self.V[layer, b] for b in r.table], axis=0)[: r.n_tokens]
+        return bf16_bits_to_f64(ks), bf16_bits_to_f64(vs)
+
+    def decode_attn(self, layer: int, q_bits: np.ndarray, reqs: Sequence[int]):
+        """o = softmax(q K^T / sqrt(D)) V per request and query head, float64.
+
+        q_bits: uint16 bf16 patterns [B][Hq][D].  Query head h reads KV head h // G.
+        Returns (o [B][Hq][D], lse [B][Hq]) with lse = log sum exp of the scaled logits.
+        A request with no tokens gives o = 0 and lse = -inf.
+        """
+        B = len(reqs)
+        q = bf16_bits_to_f64(q_bits).reshape(B, self.Hq, self.D)
+        o = np.zeros((B, self.Hq, self.D))
+        lse = np.full((B, self.Hq), -np.inf)
+        for i, req in enumerate(reqs):
+            r = self.reqs[req]
+            assert r.state == ST_RESIDENT, "only complete, resident requests decode"
+            if r.n_tokens == 0:
+                continue
+            k, v = self.gather_kv(layer, req)                       # [T][Hkv][D]
+            for h in range(self.Hq):
+                g = h // self.G
+                s = (k[:, g, :] @ q[i, h]) / math.sqrt(self.D)      # [T]
+                m = s.max()
+                e = np.exp(s - m)
+                z = e.sum()
+                o[i, h] = (e / z) @ v[:, g, :]
+                lse[i, h] = m + math.log(z)
+        return o, lse
+
+    def attn_probs(self, layer: int, q_bits: np.ndarray, req: int) -> np.ndarray:
+        """Attention weights p [Hq][ctx] of one request (for the rows-sum-to-one pin)."""
+        q = bf16_bits_to_f64(q_bits).reshape(self.Hq, self.D)
+        k, _ = self.gather_kv(layer, req)
+        out = []
+        for h in range(self.Hq):
+            s = (k[:, h // self.G, :] @ q[h]) / math.sqrt(self.D)
+            e = np.exp(s - s.max())
+            out.append(e / e.sum())
+        return np.stack(out)
+
+    # ------------------------------------------------------------------ invariants
+    def check_invariants(self) -> None:
+        """free list and all tables partition the block ids; sizes and states are legal."""
+        owned: List[int] = list(self.free)
+        for rid, r in self.reqs.items():
+            assert r.state in (ST_RESIDENT, ST_SWAPPING_OUT, ST_HOST, ST_SWAPPING_IN), (rid, r.state)
+            if r.state == ST_HOST:
+                assert r.table == [], rid
+            else:
+                assert len(r.table) == self.blocks_for(r.n_tokens), (rid, len(r.table), r.n_tokens)
+            owned.extend(r.table)
+        assert len(owned) == self.num_blocks, (len(owned), self.num_blocks)
+        assert sorted(owned) == list(range(self.num_blocks)), "a block id is owned twice or lost"
+
+
+# -------------------------------------------------------------------------------------------------
+# Brute-force restatements for tiny inputs (pure Python loops and floats)
+# -------------------------------------------------------------------------------------------------
+
+def _bf16_to_float(b: int) -> float:
+    """One bf16 pattern to a Python float via its sign / exponent / mantissa fields."""
+    sign = -1.0 if (b >> 15) & 1 else 1.0
+    exp = (b >> 7) & 0xFF
+    man = b & 0x7F
+    if exp == 0:
+        return sign * man * 2.0 ** (-126 - 7)
+    if exp == 0xFF:
+        return sign * math.inf if man == 0 else math.nan
+    return sign * (1.0 + man / 128.0) * 2.0 ** (exp - 127)
+
+
+def brute_force_attn(K, V, table, n_tokens, q_bits, S, G):
+    """Loop-by-loop decode attention for one request and one layer.
+
+    K, V: uint16 [num_blocks][S][Hkv][D]; q_bits uint16 [Hq][D].  Returns nested lists o[Hq][D].
+    """
+    Hq, D = len(q_bits), len(q_bits[0])
+    out = []
+    for h in range(Hq):
+        g = h // G
+        logits = []
+        for t in range(n_tokens):
+            blk, slot = table[t // S], t % S
+            acc = 0.0
+            for d in range(D):
+                acc += _bf16_to_float(int(q_bits[h][d])) * _bf16_to_float(int(K[blk][slot][g][d]))
+            logits.append(acc / math.sqrt(D))
+        m = max(logits)
+        w = [math.exp(x - m) for x in logits]
+        z = sum(w)
+        row = []
+        for d in range(D):
+            acc = 0.0
+            for t in range(n_tokens):
+                blk, slot = table[t // S], t % S
+                acc += (w[t] / z) * _bf16_to_float(int(V[blk][slot][g][d]))
+            row.append(acc)
+        out.append(row)
+    return out
+
+
+def brute_force_image(K, V, table, L, S, Hkv, D):
+    """Element-by-element host image of a request: flat list in [L][n_blk][K|V][S][Hkv][D] order."""
+    flat = []
+    for l in range(L):
+        for b in table:
+            for pool in (K, V):
+                for s in range(S):
+                    for h in range(Hkv):
+                        for d in range(D):
+                            flat.append(int(pool[l][b][s][h][d]))
+    return flat
