@@ -1,0 +1,275 @@
+/*
+ * ps_kvswap.h -- C ABI of the KV-block swap / paged decode library (single GPU, sm_100a).
+ *
+ * The calls implement the data path underneath ProServe's engine-layer block management
+ * (Section 4.3 "Efficient Block Management"; Appendix B "Implementation Details"):
+ *   - a device pool of M KV blocks of s_blk tokens with a free count b_f (Section 4.3, App. A),
+ *   - asynchronous offloading of a preempted request's blocks to host memory on a copy stream,
+ *     the device blocks being reclaimable only once the transfer has completed,
+ *   - pipelined reloading: host-to-device copies on a dedicated copy stream, one completion
+ *     event per layer chunk, the compute stream waiting on a chunk's event only before it
+ *     runs that chunk,
+ *   - a per-step host-to-device copy budget B_copy consumed in queue order at request
+ *     granularity, partially for the request that does not fit (Alg. 1 lines 17, 22-25),
+ *   - the decode forward the reload overlaps with, here its KV-consuming part: paged
+ *     grouped-query attention over the block table.
+ * Which request to evict and how large the budget should be are scheduler decisions and stay
+ * with the caller.
+ *
+ * Conventions
+ *   - Every function returns a ps_status (0 = PS_OK, negative = error).  On error nothing is
+ *     partially applied (allocation is all-or-nothing).  No function throws or aborts.
+ *   - "device pointer" = address in the memory of the CUDA device that was current when
+ *     ps_create was called; "host pointer" = ordinary process memory unless it says pinned.
+ *   - One caller thread per context.  All GPU work is asynchronous with respect to the host
+ *     unless a function says it waits.  Asynchronous CUDA failures surface as PS_ERR_CUDA (and
+ *     kernel-side id checks as PS_ERR_BOUNDS) from the next ps_poll / ps_sync / ps_step.
+ *   - Layouts.  bf16 everywhere.  Per layer there is one K pool and one V pool, each
+ *     [num_gpu_blocks][block_size][num_kv_heads][head_dim]; the "slab" of a block is its
+ *     block_size*num_kv_heads*head_dim contiguous elements in one pool.  The host image of a
+ *     swapped-out request with n blocks is [num_layers][n][2 (K,V)][block_size][num_kv_heads]
+ *     [head_dim]: for one layer, a run of logical blocks is one contiguous byte range.
+ *   - The KV pools and the compute stream belong to the caller and must outlive the context.
+ *     The context owns its copy streams, events, staging buffers, descriptor buffers, attention
+ *     scratch and (unless one is passed in) the pinned host pool.
+ */
+#ifndef PS_KVSWAP_H
+#define PS_KVSWAP_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ps_ctx ps_ctx;
+
+enum ps_status {
+    PS_OK = 0,
+    PS_ERR_INVALID = -1,     /* bad argument, unknown request, unsupported shape */
+    PS_ERR_NOMEM = -2,       /* not enough free device blocks */
+    PS_ERR_HOST_NOMEM = -3,  /* host pool cannot hold the image */
+    PS_ERR_STATE = -4,       /* request is in the wrong state for this call */
+    PS_ERR_BUSY = -5,        /* a transfer of this request is still in flight */
+    PS_ERR_TIMEOUT = -6,     /* bounded host wait ran out */
+    PS_ERR_CUDA = -7,        /* a CUDA call failed; see ps_last_error */
+    PS_ERR_BOUNDS = -8       /* a kernel met a block id outside the pool and skipped it */
+};
+
+enum ps_req_state {
+    PS_REQ_NONE = 0,
+    PS_REQ_RESIDENT = 1,      /* all blocks on the device (may still be gated on reload events) */
+    PS_REQ_SWAPPING_OUT = 2,  /* offload in flight; blocks still owned */
+    PS_REQ_HOST = 3,          /* image on host; owns no device block */
+    PS_REQ_SWAPPING_IN = 4    /* queued for / in the middle of a reload; owns fresh blocks */
+};
+
+enum ps_flags {
+    /* Block tables, states, budget plans and error codes only: no CUDA call is made, no byte is
+       moved, transfers "complete" at once.  For host-logic tests on machines without a GPU;
+       ps_decode_attn and the q/out arguments of ps_step are rejected in this mode. */
+    PS_FLAG_BOOKKEEPING_ONLY = 1,
+    /* Record CUDA events around every kernel and transfer so that ps_get_profile can report
+       per-kind device times.  Costs two event records per launch. */
+    PS_FLAG_PROFILE = 2,
+    /* Ablation (Section 5, block-management ablation "w/o async"): ps_step finishes the whole
+       reload before the first attention launch instead of pipelining it layer by layer. */
+    PS_FLAG_SYNC_RELOAD = 4
+};
+
+enum ps_attn_kernel {
+    PS_ATTN_AUTO = 0,
+    PS_ATTN_SIMT = 1,   /* CUDA-core kernel, warp-shuffle softmax; any supported shape */
+    PS_ATTN_MMA = 2     /* tensor-core kernel for head_dim 128 with whole-slab bulk-copy staging */
+};
+
+typedef struct ps_config {
+    int32_t num_layers;          /* L */
+    int32_t num_kv_heads;        /* Hkv */
+    int32_t num_q_heads;         /* Hq, a multiple of Hkv; group G = Hq/Hkv in {1,2,4,8} */
+    int32_t head_dim;            /* D in {64, 128} */
+    int32_t block_size;          /* s_blk, tokens per block */
+    int32_t num_gpu_blocks;      /* M, blocks in every per-layer pool */
+    int32_t max_blocks_per_req;  /* longest block table */
+    int32_t max_batch;           /* largest decode batch passed to ps_decode_attn / ps_step */
+    int32_t flags;               /* OR of ps_flags */
+    int32_t attn_kernel;         /* ps_attn_kernel */
+    int32_t kv_split_tokens;     /* tokens per split-KV work item; 0 = chosen per batch */
+    int32_t reserved0;
+    int64_t host_pool_bytes;     /* capacity for host images */
+    int64_t staging_bytes;       /* device staging per direction (split into 4 slots); 0 = 256 MiB */
+    const int32_t* initial_free_order; /* host pointer to a permutation of 0..M-1: the order in
+                                          which block ids are first handed out; NULL = 0,1,2,.. */
+} ps_config;
+
+typedef struct ps_step_stats {
+    int64_t h2d_bytes;          /* reload bytes issued by this step */
+    int64_t blocks_copied;      /* blocks (all layers) issued by this step */
+    int32_t reloads_completed;  /* requests whose last missing block was issued by this step */
+    int32_t swapouts_reaped;    /* offloads found complete; their blocks went back to the pool */
+    int32_t decoded;            /* requests that ran attention in this step */
+    int32_t gated;              /* of those, requests whose attention waited on reload events */
+    int32_t kernel_launches;    /* kernels of this library launched by this step */
+    int32_t reserved0;
+} ps_step_stats;
+
+typedef struct ps_profile {
+    double attn_ms;     int64_t attn_launches;     int64_t attn_kv_bytes;   /* K+V bytes addressed */
+    double merge_ms;    int64_t merge_launches;
+    double gather_ms;   int64_t gather_launches;   int64_t gather_bytes;    /* payload bytes (read once, written once) */
+    double scatter_ms;  int64_t scatter_launches;  int64_t scatter_bytes;
+    double d2h_ms;      int64_t d2h_copies;        int64_t d2h_bytes;
+    double h2d_ms;      int64_t h2d_copies;        int64_t h2d_bytes;
+} ps_profile;
+
+/* ---- context ---------------------------------------------------------------------------- */
+
+/* Creates a context on the current CUDA device.
+ *   k_pools, v_pools : host arrays of num_layers device pointers (the per-layer pools above).
+ *   host_pool        : pinned host memory of host_pool_bytes, or NULL to let the library pin its own.
+ *   compute_stream   : the caller's cudaStream_t (0 = legacy default stream) on which attention
+ *                      runs and against which block reuse is ordered.
+ * The first allocation order of block ids is initial_free_order; afterwards the pool is a LIFO
+ * stack: ps_kv_alloc pops one id at a time, a release pushes a table's ids in table order.
+ * Errors: PS_ERR_INVALID (shape outside the supported set, bad permutation), PS_ERR_CUDA,
+ * PS_ERR_HOST_NOMEM (pinning failed). */
+int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_pools, void* host_pool,
+                  void* compute_stream, ps_ctx** out);
+
+/* Waits for the context's outstanding work (bounded), then frees everything it owns. */
+int32_t ps_destroy(ps_ctx* ctx);
+
+/* Text of the most recent error of this context (static storage inside the context; never NULL).
+   With ctx == NULL: the most recent ps_create failure. */
+const char* ps_last_error(const ps_ctx* ctx);
+
+/* ---- block pool (Section 4.3: pool of M blocks, b_f free; per-request b_device) ---------- */
+
+/* Grows request `req` (created on first use) so that it can hold n_tokens_total tokens, i.e. to
+ * ceil(n_tokens_total / block_size) blocks.  All-or-nothing.  Only RESIDENT requests grow.
+ * Errors: PS_ERR_NOMEM, PS_ERR_STATE, PS_ERR_INVALID (shrinking, table would exceed
+ * max_blocks_per_req). */
+int32_t ps_kv_alloc(ps_ctx* ctx, int64_t req, int32_t n_tokens_total);
+
+/* Forgets the request.  RESIDENT: its blocks go back to the pool; HOST: its image is released.
+ * PS_ERR_BUSY while a transfer of it is in flight (SWAPPING_OUT, SWAPPING_IN, or a reload whose
+ * copies have not been seen complete yet). */
+int32_t ps_kv_free(ps_ctx* ctx, int64_t req);
+
+/* Copies the request's block table into out_ids (host, capacity cap; may be NULL with cap 0) and
+ * reports its length, state (ps_req_state) and token count.  Any out pointer may be NULL. */
+int32_t ps_block_table(ps_ctx* ctx, int64_t req, int32_t* out_ids, int32_t cap, int32_t* n_blocks,
+                       int32_t* state, int32_t* n_tokens);
+
+int32_t ps_num_free_blocks(ps_ctx* ctx, int32_t* out);
+
+/* ---- swap-out (Section 4.3 "Asynchronous Offloading"; App. B: D2H on a separate stream) --- */
+
+/* Starts the offload of a RESIDENT request: its blocks, every layer, are gathered through the
+ * block table into device staging and copied to a host image, ordered after all work already
+ * enqueued on the compute stream.  Returns at once; the request is SWAPPING_OUT and still owns
+ * its blocks.  When a later ps_poll / ps_step / ps_sync finds the transfer complete (offloads
+ * complete in issue order) the blocks are pushed back to the pool and the state becomes HOST.
+ * Errors: PS_ERR_STATE, PS_ERR_HOST_NOMEM, PS_ERR_INVALID, PS_ERR_CUDA. */
+int32_t ps_swap_out(ps_ctx* ctx, int64_t req);
+
+/* Host address and size of a HOST / SWAPPING_IN request's image (valid until the reload completes
+ * or the request is freed).  For checks; the bytes are final only once the state is HOST. */
+int32_t ps_host_image(ps_ctx* ctx, int64_t req, void** ptr, int64_t* bytes);
+
+/* ---- swap-in (Section 4.3 "Pipelined Reloading"; App. B: per-layer-chunk events) ---------- */
+
+/* Queues a HOST request for reload: gives it fresh blocks for its whole table (all-or-nothing)
+ * and appends it to the reload FIFO that ps_step consumes.  State becomes SWAPPING_IN.
+ * Errors: PS_ERR_STATE, PS_ERR_NOMEM. */
+int32_t ps_swap_in_begin(ps_ctx* ctx, int64_t req);
+
+/* Withdraws a queued reload of which no block has been issued yet: blocks go back to the pool in
+ * table order, state returns to HOST.  PS_ERR_BUSY once any block has been issued. */
+int32_t ps_swap_in_cancel(ps_ctx* ctx, int64_t req);
+
+/* Issues, on the copy streams, the reload of logical blocks [blk_lo, blk_hi) of one layer: one
+ * contiguous host range -> device staging -> scattered into the request's fresh blocks, then
+ * records that layer's completion event.  blk_lo must equal the number of blocks already issued
+ * for this layer (a prefix that grows).  When every layer has reached the table's length the
+ * request becomes RESIDENT; attention over it waits on the layers' events until the copies have
+ * been seen complete.  ps_step calls this path for every layer itself; the entry point is for
+ * callers that drive the layer loop on their own.
+ * Errors: PS_ERR_STATE, PS_ERR_INVALID, PS_ERR_CUDA. */
+int32_t ps_swap_in_layer(ps_ctx* ctx, int64_t req, int32_t layer, int32_t blk_lo, int32_t blk_hi);
+
+/* b_miss of Section 4.3 for one request: blocks on host not yet issued to the device. */
+int32_t ps_missing_blocks(ps_ctx* ctx, int64_t req, int32_t* out);
+
+/* ---- decode attention (the forward the reload hides under) -------------------------------- */
+
+/* One layer of paged grouped-query decode attention on the compute stream:
+ *   out[b][h][:] = softmax_t( q[b][h] . K[t][h/G] / sqrt(head_dim) ) . V[t][h/G],  t < n_tokens(reqs[b]),
+ * K/V addressed through the request's block table; bf16 inputs, fp32 accumulation, bf16 output
+ * (round to nearest even).  A request with 0 tokens gives zeros (lse = -inf).
+ *   q, out : device pointers, bf16 [batch][num_q_heads][head_dim]
+ *   lse    : device pointer, fp32 [batch][num_q_heads] (natural log of the softmax denominator
+ *            including the max), or NULL
+ *   reqs   : host array of `batch` request ids, all RESIDENT, batch <= max_batch
+ * If a request's reload copies are not known to be complete the launch is ordered after this
+ * layer's reload event.  Errors: PS_ERR_STATE, PS_ERR_INVALID, PS_ERR_CUDA. */
+int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, float* lse,
+                       const int64_t* reqs, int32_t batch);
+
+/* ---- one engine step under the copy budget (Section 4.3 "Put it Together"; Alg. 1) -------- */
+
+/* In order: reaps finished offloads; turns copy_budget_bytes into blocks (floor(bytes /
+ * (num_layers * 2 * slab bytes)); negative = unlimited) and consumes the reload FIFO in order --
+ * a request whose missing blocks fit is taken whole, the first that does not fit gets what is
+ * left; then for each layer issues that layer's reload (as ps_swap_in_layer) and launches that
+ * layer's attention for the requests of `reqs` that are RESIDENT once this step's reload is
+ * issued.  Requests complete before the step run without waiting; requests completed by this
+ * step run in a second launch that waits on the layer's reload event.  Everything is enqueued
+ * asynchronously.
+ *   q_all_layers, out_all_layers : device, bf16 [num_layers][batch][num_q_heads][head_dim]; rows of
+ *                                  requests that do not decode are left untouched.  Both may be
+ *                                  NULL with batch 0 for a copy-only step.
+ *   decoded_mask                 : host int32[batch] (or NULL): 1 where the request decoded
+ *   stats                        : host (or NULL)
+ * Errors: PS_ERR_INVALID, PS_ERR_CUDA, PS_ERR_BOUNDS. */
+int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs,
+                int32_t batch, int64_t copy_budget_bytes, int32_t* decoded_mask, ps_step_stats* stats);
+
+/* ---- completion ------------------------------------------------------------------------- */
+
+/* Non-blocking: reaps finished offloads (in issue order), releases host images of finished
+ * reloads.  *n_reaped (may be NULL) = offloads reaped by this call. */
+int32_t ps_poll(ps_ctx* ctx, int32_t* n_reaped);
+
+/* Waits until every transfer and kernel this context has enqueued (copy streams and the compute
+ * stream) is complete, then reaps as ps_poll.  timeout_ms < 0 waits without limit.
+ * PS_ERR_TIMEOUT leaves everything in flight. */
+int32_t ps_sync(ps_ctx* ctx, int32_t timeout_ms);
+
+/* ---- measurement ------------------------------------------------------------------------ */
+
+/* Kernels launched by this context since creation. */
+int32_t ps_launch_count(ps_ctx* ctx, int64_t* out);
+
+/* Accumulated device times per kind since the last reset (needs PS_FLAG_PROFILE; call after
+ * ps_sync).  reset != 0 clears the accumulators afterwards. */
+int32_t ps_get_profile(ps_ctx* ctx, ps_profile* out, int32_t reset);
+
+/* Pinned-memory host link probe: best-of-`iters` cudaMemcpyAsync of `bytes` between a pinned host
+ * buffer and a device buffer, timed with CUDA events.  direction 0 = host-to-device, 1 = device-
+ * to-host, 2 = both at once on two streams (reports the sum).  *gb_per_s in 1e9 bytes/s.
+ * Allocates and frees its own buffers; needs no context. */
+int32_t ps_link_probe(int64_t bytes, int32_t direction, int32_t iters, double* gb_per_s);
+
+/* On-device gather / scatter of `n_blocks` blocks of one layer between the pools and a contiguous
+ * device buffer, without any host transfer: the kernels of ps_swap_out / ps_swap_in_layer alone,
+ * for measuring them against HBM bandwidth.  `staging` is a device pointer with room for
+ * n_blocks * 2 slabs ([n][K,V][slab]); ids is a host array of n_blocks block ids.  Runs on the
+ * compute stream.  direction 0 = gather (pool -> staging), 1 = scatter (staging -> pool). */
+int32_t ps_copy_blocks(ps_ctx* ctx, int32_t layer, const int32_t* ids, int32_t n_blocks, void* staging,
+                       int32_t direction);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PS_KVSWAP_H */

@@ -1,0 +1,283 @@
+"""Thin ctypes binding of libps_kvswap.so: argument marshalling only, same names as the C ABI.
+
+Every step of the hot path (block bookkeeping, gather/scatter, transfers, attention, the step loop)
+runs inside the library; this module converts Python values to pointers and sizes.  PyTorch appears
+only as the owner of device memory and of the compute stream (`tensor.data_ptr()`,
+`torch.cuda.current_stream().cuda_stream`).
+
+The library must have been built (`python -m paper_2512_12928_b200.build`); loading fails loudly
+otherwise.  There is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence, Tuple
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "lib", "libps_kvswap.so")
+
+# status codes / states / flags (values fixed by include/ps_kvswap.h)
+PS_OK, PS_ERR_INVALID, PS_ERR_NOMEM, PS_ERR_HOST_NOMEM = 0, -1, -2, -3
+PS_ERR_STATE, PS_ERR_BUSY, PS_ERR_TIMEOUT, PS_ERR_CUDA, PS_ERR_BOUNDS = -4, -5, -6, -7, -8
+PS_REQ_NONE, PS_REQ_RESIDENT, PS_REQ_SWAPPING_OUT, PS_REQ_HOST, PS_REQ_SWAPPING_IN = 0, 1, 2, 3, 4
+PS_FLAG_BOOKKEEPING_ONLY, PS_FLAG_PROFILE, PS_FLAG_SYNC_RELOAD = 1, 2, 4
+PS_ATTN_AUTO, PS_ATTN_SIMT, PS_ATTN_MMA = 0, 1, 2
+
+EXPORTS = [
+    "ps_create", "ps_destroy", "ps_last_error", "ps_kv_alloc", "ps_kv_free", "ps_block_table",
+    "ps_num_free_blocks", "ps_swap_out", "ps_host_image", "ps_swap_in_begin", "ps_swap_in_cancel",
+    "ps_swap_in_layer", "ps_missing_blocks", "ps_decode_attn", "ps_step", "ps_poll", "ps_sync",
+    "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks",
+]
+
+
+class PsConfig(C.Structure):
+    _fields_ = [
+        ("num_layers", C.c_int32), ("num_kv_heads", C.c_int32), ("num_q_heads", C.c_int32),
+        ("head_dim", C.c_int32), ("block_size", C.c_int32), ("num_gpu_blocks", C.c_int32),
+        ("max_blocks_per_req", C.c_int32), ("max_batch", C.c_int32), ("flags", C.c_int32),
+        ("attn_kernel", C.c_int32), ("kv_split_tokens", C.c_int32), ("reserved0", C.c_int32),
+        ("host_pool_bytes", C.c_int64), ("staging_bytes", C.c_int64),
+        ("initial_free_order", C.POINTER(C.c_int32)),
+    ]
+
+
+class PsStepStats(C.Structure):
+    _fields_ = [
+        ("h2d_bytes", C.c_int64), ("blocks_copied", C.c_int64), ("reloads_completed", C.c_int32),
+        ("swapouts_reaped", C.c_int32), ("decoded", C.c_int32), ("gated", C.c_int32),
+        ("kernel_launches", C.c_int32), ("reserved0", C.c_int32),
+    ]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_ if k != "reserved0"}
+
+
+class PsProfile(C.Structure):
+    _fields_ = [
+        ("attn_ms", C.c_double), ("attn_launches", C.c_int64), ("attn_kv_bytes", C.c_int64),
+        ("merge_ms", C.c_double), ("merge_launches", C.c_int64),
+        ("gather_ms", C.c_double), ("gather_launches", C.c_int64), ("gather_bytes", C.c_int64),
+        ("scatter_ms", C.c_double), ("scatter_launches", C.c_int64), ("scatter_bytes", C.c_int64),
+        ("d2h_ms", C.c_double), ("d2h_copies", C.c_int64), ("d2h_bytes", C.c_int64),
+        ("h2d_ms", C.c_double), ("h2d_copies", C.c_int64), ("h2d_bytes", C.c_int64),
+    ]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class PsError(RuntimeError):
+    def __init__(self, code: int, where: str, text: str = ""):
+        super().__init__(f"{where} failed with status {code}" + (f": {text}" if text else ""))
+        self.code = code
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Loads the shared library and declares the prototypes.  Raises if it is not built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2512_12928_b200.build` "
+            "(there is no fallback implementation)")
+    lib = C.CDLL(LIB_PATH)
+    vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+    p32, p64 = C.POINTER(C.c_int32), C.POINTER(C.c_int64)
+    proto = {
+        "ps_create": (i32, [C.POINTER(PsConfig), C.POINTER(vp), C.POINTER(vp), vp, vp, C.POINTER(vp)]),
+        "ps_destroy": (i32, [vp]),
+        "ps_last_error": (C.c_char_p, [vp]),
+        "ps_kv_alloc": (i32, [vp, i64, i32]),
+        "ps_kv_free": (i32, [vp, i64]),
+        "ps_block_table": (i32, [vp, i64, p32, i32, p32, p32, p32]),
+        "ps_num_free_blocks": (i32, [vp, p32]),
+        "ps_swap_out": (i32, [vp, i64]),
+        "ps_host_image": (i32, [vp, i64, C.POINTER(vp), p64]),
+        "ps_swap_in_begin": (i32, [vp, i64]),
+        "ps_swap_in_cancel": (i32, [vp, i64]),
+        "ps_swap_in_layer": (i32, [vp, i64, i32, i32, i32]),
+        "ps_missing_blocks": (i32, [vp, i64, p32]),
+        "ps_decode_attn": (i32, [vp, i32, vp, vp, vp, p64, i32]),
+        "ps_step": (i32, [vp, vp, vp, p64, i32, i64, p32, C.POINTER(PsStepStats)]),
+        "ps_poll": (i32, [vp, p32]),
+        "ps_sync": (i32, [vp, i32]),
+        "ps_launch_count": (i32, [vp, p64]),
+        "ps_get_profile": (i32, [vp, C.POINTER(PsProfile), i32]),
+        "ps_link_probe": (i32, [i64, i32, i32, C.POINTER(C.c_double)]),
+        "ps_copy_blocks": (i32, [vp, i32, p32, i32, vp, i32]),
+    }
+    for name, (res, args) in proto.items():
+        fn = getattr(lib, name)
+        fn.restype = res
+        fn.argtypes = args
+    _lib = lib
+    return lib
+
+
+def ps_link_probe(nbytes: int, direction: int, iters: int = 10) -> float:
+    """Pinned-copy host link rate in GB/s (1e9): 0 = H2D, 1 = D2H, 2 = both at once (sum)."""
+    out = C.c_double(0.0)
+    rc = load().ps_link_probe(nbytes, direction, iters, C.byref(out))
+    if rc != PS_OK:
+        raise PsError(rc, "ps_link_probe", load().ps_last_error(None).decode())
+    return out.value
+
+
+def _i64_array(vals: Sequence[int]):
+    return (C.c_int64 * max(len(vals), 1))(*[int(v) for v in vals])
+
+
+class KVSwap:
+    """One library context.  Methods carry the C entry points' names without the `ps_` prefix and
+    return the raw status code where the call can legitimately fail (so a test script can drive the
+    library and a checker side by side); `check=True` variants raise instead."""
+
+    def __init__(self, *, num_layers: int, num_kv_heads: int, num_q_heads: int, head_dim: int, block_size: int,
+                 num_gpu_blocks: int, max_blocks_per_req: int, max_batch: int = 0, host_pool_bytes: int = 0,
+                 staging_bytes: int = 0, initial_free_order=None, k_pools=None, v_pools=None, flags: int = 0,
+                 attn_kernel: int = PS_ATTN_AUTO, kv_split_tokens: int = 0, host_pool_ptr: int = 0,
+                 compute_stream: Optional[int] = None):
+        self.lib = load()
+        self.L = num_layers
+        self.Hq, self.D = num_q_heads, head_dim
+        cfg = PsConfig()
+        cfg.num_layers, cfg.num_kv_heads, cfg.num_q_heads = num_layers, num_kv_heads, num_q_heads
+        cfg.head_dim, cfg.block_size, cfg.num_gpu_blocks = head_dim, block_size, num_gpu_blocks
+        cfg.max_blocks_per_req, cfg.max_batch, cfg.flags = max_blocks_per_req, max_batch, flags
+        cfg.attn_kernel, cfg.kv_split_tokens = attn_kernel, kv_split_tokens
+        cfg.host_pool_bytes, cfg.staging_bytes = host_pool_bytes, staging_bytes
+        self._order = None
+        if initial_free_order is not None:
+            self._order = (C.c_int32 * num_gpu_blocks)(*[int(v) for v in initial_free_order])
+            cfg.initial_free_order = C.cast(self._order, C.POINTER(C.c_int32))
+        self._pools = (k_pools, v_pools)      # keep the tensors alive
+        kp = vp = None
+        if not (flags & PS_FLAG_BOOKKEEPING_ONLY):
+            if k_pools is None or v_pools is None or len(k_pools) != num_layers or len(v_pools) != num_layers:
+                raise ValueError("k_pools and v_pools must be lists of num_layers device tensors")
+            kp = (C.c_void_p * num_layers)(*[t.data_ptr() for t in k_pools])
+            vp = (C.c_void_p * num_layers)(*[t.data_ptr() for t in v_pools])
+            if compute_stream is None:
+                import torch
+                compute_stream = torch.cuda.current_stream().cuda_stream
+        self.compute_stream = compute_stream or 0
+        handle = C.c_void_p()
+        rc = self.lib.ps_create(C.byref(cfg), kp, vp, C.c_void_p(host_pool_ptr or None),
+                                C.c_void_p(self.compute_stream or None), C.byref(handle))
+        if rc != PS_OK:
+            raise PsError(rc, "ps_create", self.lib.ps_last_error(None).decode())
+        self.h = handle
+
+    # ---- lifetime
+    def destroy(self) -> None:
+        if getattr(self, "h", None):
+            self.lib.ps_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def last_error(self) -> str:
+        return self.lib.ps_last_error(self.h).decode()
+
+    def _ck(self, rc: int, where: str) -> int:
+        if rc != PS_OK:
+            raise PsError(rc, where, self.last_error())
+        return rc
+
+    # ---- pool
+    def kv_alloc(self, req: int, n_tokens_total: int) -> int:
+        return self.lib.ps_kv_alloc(self.h, req, n_tokens_total)
+
+    def kv_free(self, req: int) -> int:
+        return self.lib.ps_kv_free(self.h, req)
+
+    def block_table(self, req: int) -> Tuple[List[int], int]:
+        n, st, nt = C.c_int32(), C.c_int32(), C.c_int32()
+        self._ck(self.lib.ps_block_table(self.h, req, None, 0, C.byref(n), C.byref(st), C.byref(nt)), "ps_block_table")
+        ids = (C.c_int32 * max(n.value, 1))()
+        self._ck(self.lib.ps_block_table(self.h, req, ids, n.value, None, None, None), "ps_block_table")
+        return list(ids[: n.value]), st.value
+
+    def n_tokens(self, req: int) -> int:
+        nt = C.c_int32()
+        self._ck(self.lib.ps_block_table(self.h, req, None, 0, None, None, C.byref(nt)), "ps_block_table")
+        return nt.value
+
+    def num_free_blocks(self) -> int:
+        out = C.c_int32()
+        self._ck(self.lib.ps_num_free_blocks(self.h, C.byref(out)), "ps_num_free_blocks")
+        return out.value
+
+    # ---- swap
+    def swap_out(self, req: int) -> int:
+        return self.lib.ps_swap_out(self.h, req)
+
+    def host_image(self, req: int) -> Tuple[int, int]:
+        ptr, nbytes = C.c_void_p(), C.c_int64()
+        self._ck(self.lib.ps_host_image(self.h, req, C.byref(ptr), C.byref(nbytes)), "ps_host_image")
+        return ptr.value or 0, nbytes.value
+
+    def swap_in_begin(self, req: int) -> int:
+        return self.lib.ps_swap_in_begin(self.h, req)
+
+    def swap_in_cancel(self, req: int) -> int:
+        return self.lib.ps_swap_in_cancel(self.h, req)
+
+    def swap_in_layer(self, req: int, layer: int, blk_lo: int, blk_hi: int) -> int:
+        return self.lib.ps_swap_in_layer(self.h, req, layer, blk_lo, blk_hi)
+
+    def missing_blocks(self, req: int) -> int:
+        out = C.c_int32()
+        self._ck(self.lib.ps_missing_blocks(self.h, req, C.byref(out)), "ps_missing_blocks")
+        return out.value
+
+    # ---- attention / step
+    def decode_attn(self, layer: int, q, out, reqs: Sequence[int], lse=None) -> int:
+        """q, out: device bf16 tensors [B][Hq][D]; lse: device fp32 [B][Hq] or None."""
+        arr = _i64_array(reqs)
+        return self.lib.ps_decode_attn(self.h, layer, C.c_void_p(q.data_ptr()), C.c_void_p(out.data_ptr()),
+                                       C.c_void_p(lse.data_ptr()) if lse is not None else None, arr, len(reqs))
+
+    def step(self, q_all, out_all, reqs: Sequence[int], copy_budget_bytes: int):
+        """Returns (status, decoded mask list, stats dict).  q_all/out_all: device bf16 [L][B][Hq][D] or None."""
+        arr = _i64_array(reqs)
+        mask = (C.c_int32 * max(len(reqs), 1))()
+        st = PsStepStats()
+        rc = self.lib.ps_step(self.h, C.c_void_p(q_all.data_ptr()) if q_all is not None else None,
+                              C.c_void_p(out_all.data_ptr()) if out_all is not None else None, arr, len(reqs),
+                              copy_budget_bytes, mask, C.byref(st))
+        return rc, list(mask[: len(reqs)]), st.as_dict()
+
+    # ---- completion
+    def poll(self) -> int:
+        n = C.c_int32()
+        self._ck(self.lib.ps_poll(self.h, C.byref(n)), "ps_poll")
+        return n.value
+
+    def sync(self, timeout_ms: int = 120000) -> int:
+        return self.lib.ps_sync(self.h, timeout_ms)
+
+    # ---- measurement
+    def launch_count(self) -> int:
+        out = C.c_int64()
+        self._ck(self.lib.ps_launch_count(self.h, C.byref(out)), "ps_launch_count")
+        return out.value
+
+    def get_profile(self, reset: bool = False) -> dict:
+        p = PsProfile()
+        self._ck(self.lib.ps_get_profile(self.h, C.byref(p), 1 if reset else 0), "ps_get_profile")
+        return p.as_dict()
+
+    def copy_blocks(self, layer: int, ids: Sequence[int], staging, direction: int) -> int:
+        arr = (C.c_int32 * max(len(ids), 1))(*[int(v) for v in ids])
+        return self.lib.ps_copy_blocks(self.h, layer, arr, len(ids), C.c_void_p(staging.data_ptr()), direction)

@@ -1,0 +1,75 @@
+// Internal declarations shared by the runtime and the kernel translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ps {
+
+// ---- block gather / scatter (swap-out and swap-in kernels) -----------------------------------
+
+// A "slab" is one block of one layer in one pool: slab_vec 16-byte vectors, contiguous.
+//
+// Gather: image slab s (s in [slab_begin, slab_begin + slab_count)) of a request with n_blk blocks
+// lives at layer l = s / (2 n_blk), logical block j = (s % (2 n_blk)) / 2, tensor t = s & 1
+// (0 = K, 1 = V); it is copied from pool[l][t] + table[j] * slab to dst + (s - slab_begin) * slab.
+cudaError_t launch_gather_image(const void* const* d_kpools, const void* const* d_vpools, const int32_t* d_table,
+                                int32_t n_blk, int64_t slab_begin, int64_t slab_count, void* dst, int32_t slab_vec,
+                                int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
+
+// Scatter for one layer: src holds n consecutive (K slab, V slab) pairs; pair i goes to block
+// d_ids[i] of kpool / vpool.
+cudaError_t launch_scatter_layer(void* kpool, void* vpool, const int32_t* d_ids, int32_t n, const void* src,
+                                 int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
+
+// Gather for one layer into the same pair layout (the inverse of launch_scatter_layer).
+cudaError_t launch_gather_layer(const void* kpool, const void* vpool, const int32_t* d_ids, int32_t n, void* dst,
+                                int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
+
+// ---- paged decode attention --------------------------------------------------------------------
+
+// One split-KV work item: tokens [t_begin, t_end) of batch row b.  `part` indexes the partial
+// result slot; `n_parts` is how many items row b has (1 = the kernel writes the final output).
+struct AttnItem {
+    int32_t b;
+    int32_t t_begin;
+    int32_t t_end;
+    int32_t part;
+    int32_t n_parts;
+    int32_t pad0, pad1, pad2;
+};
+
+struct AttnShape {
+    int32_t num_kv_heads, num_q_heads, head_dim, block_size, num_blocks;
+};
+
+struct AttnBatch {                 // device pointers to the per-batch metadata
+    const int32_t* block_tables;   // [B][table_stride]
+    const int32_t* ctx_len;        // [B]
+    const AttnItem* items;         // [n_items]
+    const int32_t* row_first_part; // [B] first partial slot of the row
+    const int32_t* row_parts;      // [B] number of partial slots of the row
+    int32_t table_stride;
+    int32_t batch;
+};
+
+// Partial results: per (part, q head): D floats of unnormalised output, then the running max
+// (log2 units) and the running sum.  Row stride D + 2 floats.
+size_t attn_partial_bytes(const AttnShape& sh, int32_t max_parts);
+
+// Launches the attention kernel for items [item_begin, item_end).  kernel: 1 = SIMT, 2 = MMA.
+cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool, const void* q,
+                               void* out, float* lse, const AttnBatch& batch, int32_t item_begin, int32_t item_end,
+                               float* partials, int32_t* d_status, cudaStream_t stream);
+
+// Merges the partial results of every row with more than one part into out / lse.
+cudaError_t launch_attn_merge(const AttnShape& sh, void* out, float* lse, const AttnBatch& batch,
+                              const float* partials, cudaStream_t stream);
+
+// Whether the tensor-core kernel supports the shape.
+bool attn_mma_supported(const AttnShape& sh);
+
+// One-time per-process kernel attribute set-up (dynamic shared memory opt-in).
+cudaError_t attn_init();
+
+}  // namespace ps
