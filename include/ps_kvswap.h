@@ -122,6 +122,17 @@ typedef struct ps_profile {
     double h2d_ms;      int64_t h2d_copies;        int64_t h2d_bytes;
 } ps_profile;
 
+/* One timed span of the trace: what ran, for which layer, and when (microseconds after ps_trace
+ * was switched on, device clock).  kind: 0 attention, 1 split-KV merge, 2 gather, 3 scatter,
+ * 4 device-to-host copy, 5 host-to-device copy.  tag: the layer (attention launches that waited on
+ * a reload event carry 1000 + layer), or -1. */
+typedef struct ps_trace_span {
+    int32_t kind;
+    int32_t tag;
+    float start_us;
+    float end_us;
+} ps_trace_span;
+
 /* ---- context ---------------------------------------------------------------------------- */
 
 /* Creates a context on the current CUDA device.
@@ -254,6 +265,13 @@ int32_t ps_launch_count(ps_ctx* ctx, int64_t* out);
 /* Accumulated device times per kind since the last reset (needs PS_FLAG_PROFILE; call after
  * ps_sync).  reset != 0 clears the accumulators afterwards. */
 int32_t ps_get_profile(ps_ctx* ctx, ps_profile* out, int32_t reset);
+
+/* Timeline of the copy streams against the compute stream (the per-layer-chunk overlap of
+ * Appendix B made visible).  ps_trace(ctx, 1) starts recording every kernel and transfer span of a
+ * PS_FLAG_PROFILE context relative to "now" on the compute stream; ps_trace(ctx, 0) stops.
+ * ps_trace_read copies up to cap spans (call after ps_sync) and reports how many exist. */
+int32_t ps_trace(ps_ctx* ctx, int32_t enable);
+int32_t ps_trace_read(ps_ctx* ctx, ps_trace_span* out, int32_t cap, int32_t* n);
 
 /* Pinned-memory host link probe: best-of-`iters` cudaMemcpyAsync of `bytes` between a pinned host
  * buffer and a device buffer, timed with CUDA events.  direction 0 = host-to-device, 1 = device-

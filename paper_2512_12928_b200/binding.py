@@ -28,7 +28,7 @@ EXPORTS = [
     "ps_create", "ps_destroy", "ps_last_error", "ps_kv_alloc", "ps_kv_free", "ps_block_table",
     "ps_num_free_blocks", "ps_swap_out", "ps_host_image", "ps_swap_in_begin", "ps_swap_in_cancel",
     "ps_swap_in_layer", "ps_missing_blocks", "ps_decode_attn", "ps_step", "ps_poll", "ps_sync",
-    "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks",
+    "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
 ]
 
 
@@ -66,6 +66,13 @@ class PsProfile(C.Structure):
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class PsTraceSpan(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("tag", C.c_int32), ("start_us", C.c_float), ("end_us", C.c_float)]
+
+
+TRACE_KINDS = ["attn", "merge", "gather", "scatter", "d2h", "h2d"]
 
 
 class PsError(RuntimeError):
@@ -111,6 +118,8 @@ def load() -> C.CDLL:
         "ps_get_profile": (i32, [vp, C.POINTER(PsProfile), i32]),
         "ps_link_probe": (i32, [i64, i32, i32, C.POINTER(C.c_double)]),
         "ps_copy_blocks": (i32, [vp, i32, p32, i32, vp, i32]),
+        "ps_trace": (i32, [vp, i32]),
+        "ps_trace_read": (i32, [vp, C.POINTER(PsTraceSpan), i32, p32]),
     }
     for name, (res, args) in proto.items():
         fn = getattr(lib, name)
@@ -277,6 +286,17 @@ class KVSwap:
         p = PsProfile()
         self._ck(self.lib.ps_get_profile(self.h, C.byref(p), 1 if reset else 0), "ps_get_profile")
         return p.as_dict()
+
+    def trace(self, enable: bool) -> int:
+        return self.lib.ps_trace(self.h, 1 if enable else 0)
+
+    def trace_read(self):
+        """List of (kind name, tag, start_us, end_us), call after sync()."""
+        n = C.c_int32()
+        self._ck(self.lib.ps_trace_read(self.h, None, 0, C.byref(n)), "ps_trace_read")
+        buf = (PsTraceSpan * max(n.value, 1))()
+        self._ck(self.lib.ps_trace_read(self.h, buf, n.value, C.byref(n)), "ps_trace_read")
+        return [(TRACE_KINDS[s.kind], s.tag, s.start_us, s.end_us) for s in buf[: n.value]]
 
     def copy_blocks(self, layer: int, ids: Sequence[int], staging, direction: int) -> int:
         arr = (C.c_int32 * max(len(ids), 1))(*[int(v) for v in ids])

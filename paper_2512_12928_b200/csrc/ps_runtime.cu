@@ -103,6 +103,7 @@ enum ProfKind { kProfAttn = 0, kProfMerge, kProfGather, kProfScatter, kProfD2H, 
 
 struct ProfSpan {
     int kind;
+    int tag;  // layer, or -1
     cudaEvent_t e0, e1;
 };
 
@@ -176,6 +177,9 @@ struct ps_ctx {
     double prof_ms[kProfKinds]{};
     int64_t prof_n[kProfKinds]{};
     int64_t prof_bytes[kProfKinds]{};
+    bool tracing = false;
+    cudaEvent_t trace_base = nullptr;
+    std::vector<ps_trace_span> trace;
 
     int32_t fail(int32_t code, const std::string& msg) {
         err = msg;
@@ -305,7 +309,8 @@ struct ProfScope {
     cudaStream_t s;
     cudaEvent_t e0 = nullptr;
     bool on = false;
-    ProfScope(ps_ctx* c, int k, cudaStream_t st, int64_t bytes) : ctx(c), kind(k), s(st) {
+    int tag;
+    ProfScope(ps_ctx* c, int k, cudaStream_t st, int64_t bytes, int tg = -1) : ctx(c), kind(k), s(st), tag(tg) {
         ctx->prof_bytes[kind] += bytes;
         ctx->prof_n[kind] += 1;
         if (ctx->profile && !ctx->bk && get_event(ctx, true, &e0) == cudaSuccess) {
@@ -317,7 +322,7 @@ struct ProfScope {
         cudaEvent_t e1;
         if (get_event(ctx, true, &e1) != cudaSuccess) return;
         cudaEventRecord(e1, s);
-        ctx->spans.push_back({kind, e0, e1});
+        ctx->spans.push_back({kind, tag, e0, e1});
     }
 };
 
@@ -328,6 +333,11 @@ void resolve_profile(ps_ctx* ctx) {
         float ms = 0.f;
         if (cudaEventQuery(sp.e1) == cudaSuccess && cudaEventElapsedTime(&ms, sp.e0, sp.e1) == cudaSuccess) {
             ctx->prof_ms[sp.kind] += ms;
+            if (ctx->tracing && ctx->trace_base) {
+                float t0 = 0.f;
+                if (cudaEventElapsedTime(&t0, ctx->trace_base, sp.e0) == cudaSuccess)
+                    ctx->trace.push_back({sp.kind, sp.tag, t0 * 1e3f, (t0 + ms) * 1e3f});
+            }
             ctx->ev_pool_timing.push_back(sp.e0);
             ctx->ev_pool_timing.push_back(sp.e1);
         } else {
@@ -425,7 +435,7 @@ int32_t issue_reload_layer(ps_ctx* ctx, int32_t layer, const std::vector<PlanEnt
             const int64_t take = std::min<int64_t>(plan[i].hi - lo, cap - used);
             if (take > 0) {
                 const char* src = ctx->host_pool + r.img_off + ((int64_t)layer * n_blk + lo) * Bl;
-                ProfScope prof(ctx, kProfH2D, ctx->s_h2d, take * Bl);
+                ProfScope prof(ctx, kProfH2D, ctx->s_h2d, take * Bl, layer);
                 CK(cudaMemcpyAsync(sp + used * Bl, src, (size_t)(take * Bl), cudaMemcpyHostToDevice, ctx->s_h2d));
             }
             for (int64_t j = lo; j < lo + take; ++j) ids.push_back(r.table[(size_t)j]);
@@ -445,7 +455,7 @@ int32_t issue_reload_layer(ps_ctx* ctx, int32_t layer, const std::vector<PlanEnt
             memcpy(ctx->a_scatter.h + off, ids.data(), ids.size() * sizeof(int32_t));
             CK(cudaMemcpyAsync(ctx->a_scatter.d + off, ctx->a_scatter.h + off, ids.size() * sizeof(int32_t),
                                cudaMemcpyHostToDevice, ctx->s_scatter));
-            ProfScope prof(ctx, kProfScatter, ctx->s_scatter, (int64_t)ids.size() * Bl);
+            ProfScope prof(ctx, kProfScatter, ctx->s_scatter, (int64_t)ids.size() * Bl, layer);
             CK(ps::launch_scatter_layer(ctx->kpools[layer], ctx->vpools[layer], (const int32_t*)(ctx->a_scatter.d + off),
                                         (int32_t)ids.size(), sp, ctx->slab_vec, ctx->cfg.num_gpu_blocks,
                                         ctx->d_status, ctx->s_scatter));
@@ -635,7 +645,7 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
     const int64_t bytes = m.kv_bytes_per_layer;
     const int64_t ungated_bytes = m.n_items ? bytes * m.n_ungated_items / m.n_items : 0;
     if (m.n_ungated_items > 0) {
-        ProfScope prof(ctx, kProfAttn, ctx->compute, ungated_bytes);
+        ProfScope prof(ctx, kProfAttn, ctx->compute, ungated_bytes, layer);
         CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev, 0,
                                   m.n_ungated_items, ctx->partials, ctx->d_status, ctx->compute));
         ctx->launches++;
@@ -643,14 +653,14 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
     }
     if (m.n_items > m.n_ungated_items) {
         if (wait_event) CK(cudaStreamWaitEvent(ctx->compute, wait_event, 0));
-        ProfScope prof(ctx, kProfAttn, ctx->compute, bytes - ungated_bytes);
+        ProfScope prof(ctx, kProfAttn, ctx->compute, bytes - ungated_bytes, 1000 + layer);
         CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev,
                                   m.n_ungated_items, m.n_items, ctx->partials, ctx->d_status, ctx->compute));
         ctx->launches++;
         ++*n_launched;
     }
     if (m.any_multi) {
-        ProfScope prof(ctx, kProfMerge, ctx->compute, 0);
+        ProfScope prof(ctx, kProfMerge, ctx->compute, 0, layer);
         CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials, ctx->compute));
         ctx->launches++;
         ++*n_launched;
@@ -666,7 +676,7 @@ void destroy_ctx(ps_ctx* ctx) {
             for (cudaEvent_t e : {ctx->e_gathered[i], ctx->e_drained[i], ctx->e_loaded[i], ctx->e_scattered[i]})
                 if (e) cudaEventDestroy(e);
         for (cudaEvent_t e : ctx->ev_in) cudaEventDestroy(e);
-        for (cudaEvent_t e : {ctx->e_mark, ctx->e_mark2, ctx->e_ids})
+        for (cudaEvent_t e : {ctx->e_mark, ctx->e_mark2, ctx->e_ids, ctx->trace_base})
             if (e) cudaEventDestroy(e);
         for (auto& t : {&ctx->t_d2h, &ctx->t_scatter, &ctx->t_compute})
             for (auto& p : t->pending) cudaEventDestroy(p.second);
@@ -1298,6 +1308,28 @@ int32_t ps_get_profile(ps_ctx* ctx, ps_profile* out, int32_t reset) {
             ctx->prof_bytes[k] = 0;
         }
     }
+    return PS_OK;
+}
+
+int32_t ps_trace(ps_ctx* ctx, int32_t enable) {
+    if (!ctx) return PS_ERR_INVALID;
+    if (ctx->bk || !ctx->profile) return ctx->fail(PS_ERR_INVALID, "ps_trace: needs a device context created with PS_FLAG_PROFILE");
+    ctx->trace.clear();
+    ctx->tracing = enable != 0;
+    if (ctx->tracing) {
+        if (!ctx->trace_base) CK(cudaEventCreate(&ctx->trace_base));
+        CK(cudaEventRecord(ctx->trace_base, ctx->compute));
+    }
+    return PS_OK;
+}
+
+int32_t ps_trace_read(ps_ctx* ctx, ps_trace_span* out, int32_t cap, int32_t* n) {
+    if (!ctx || !n || cap < 0 || (cap > 0 && !out)) return PS_ERR_INVALID;
+    if (!ctx->bk) resolve_profile(ctx);
+    const int32_t have = (int32_t)ctx->trace.size();
+    const int32_t m = std::min(cap, have);
+    if (m > 0) memcpy(out, ctx->trace.data(), (size_t)m * sizeof(ps_trace_span));
+    *n = have;
     return PS_OK;
 }
 

@@ -291,7 +291,7 @@ def test_errors_on_device_context():
     assert p.both("swap_in_begin", r) == B.PS_ERR_STATE
     assert p.both("swap_in_cancel", r) == B.PS_OK
     assert p.both("kv_free", r) == B.PS_OK
-    assert p.both("kv_alloc", 1000, 10 ** 6) == B.PS_ERR_NOMEM
+    assert p.both("kv_alloc", 1000, 250 * 16) == B.PS_ERR_NOMEM
     p.assert_tables_equal([x for x in range(len(w.ctx_lens)) if x != r])
     q = torch.zeros((1, 8, 64), dtype=torch.bfloat16, device="cuda")
     assert p.lib.decode_attn(5, q, q, [0]) == B.PS_ERR_INVALID
