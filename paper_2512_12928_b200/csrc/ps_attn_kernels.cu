@@ -209,10 +209,11 @@ decode_attn_simt_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bflo
 template <int D>
 __global__ void __launch_bounds__(D)
 attn_merge_kernel(__nv_bfloat16* __restrict__ out, float* __restrict__ lse, AttnBatch batch, int32_t Hq,
-                  const float* __restrict__ partials) {
+                  const float* __restrict__ partials, int32_t lane) {
     const int b = blockIdx.x;
     const int n = batch.row_parts[b];
     if (n <= 1) return;
+    if (lane >= 0 && batch.row_lane[b] != lane) return;
     const int h = blockIdx.y;
     const int d = threadIdx.x;
     const float* base = partials + ((int64_t)batch.row_first_part[b] * Hq + h) * (D + 2);
@@ -277,13 +278,13 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
 }
 
 cudaError_t launch_attn_merge(const AttnShape& sh, void* out, float* lse, const AttnBatch& batch,
-                              const float* partials, cudaStream_t stream) {
+                              const float* partials, int32_t lane, cudaStream_t stream) {
     if (batch.batch <= 0) return cudaSuccess;
     dim3 grid((unsigned)batch.batch, (unsigned)sh.num_q_heads);
     if (sh.head_dim == 128)
-        attn_merge_kernel<128><<<grid, 128, 0, stream>>>((__nv_bfloat16*)out, lse, batch, sh.num_q_heads, partials);
+        attn_merge_kernel<128><<<grid, 128, 0, stream>>>((__nv_bfloat16*)out, lse, batch, sh.num_q_heads, partials, lane);
     else if (sh.head_dim == 64)
-        attn_merge_kernel<64><<<grid, 64, 0, stream>>>((__nv_bfloat16*)out, lse, batch, sh.num_q_heads, partials);
+        attn_merge_kernel<64><<<grid, 64, 0, stream>>>((__nv_bfloat16*)out, lse, batch, sh.num_q_heads, partials, lane);
     else
         return cudaErrorNotSupported;
     return cudaGetLastError();

@@ -79,6 +79,31 @@ layer_copy_kernel(uint4* __restrict__ kpool, uint4* __restrict__ vpool, const in
         copy_piece(pool_slab, pair_slab, piece * kPieceVec, slab_vec);
 }
 
+struct ParamIds {
+    int32_t ids[kMaxParamIds];
+};
+
+__global__ void __launch_bounds__(kCopyThreads)
+scatter_param_ids_kernel(uint4* __restrict__ kpool, uint4* __restrict__ vpool, const __grid_constant__ ParamIds ids,
+                         const uint4* __restrict__ pairs, int32_t slab_vec, int32_t pieces, int32_t num_blocks,
+                         int32_t* status) {
+    const int local = blockIdx.x / pieces;
+    const int piece = blockIdx.x - local * pieces;
+    const int id = ids.ids[local >> 1];
+    if ((unsigned)id >= (unsigned)num_blocks) {
+        if (threadIdx.x == 0) *(volatile int32_t*)status = 1;
+        return;
+    }
+    uint4* pool_slab = ((local & 1) ? vpool : kpool) + (int64_t)id * slab_vec;
+    copy_piece(pairs + (int64_t)local * slab_vec, pool_slab, piece * kPieceVec, slab_vec);
+}
+
+__global__ void __launch_bounds__(256)
+upload_kernel(uint4* __restrict__ dst, const uint4* __restrict__ src, int64_t n_vec) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (int64_t)gridDim.x * blockDim.x)
+        dst[i] = src[i];
+}
+
 inline int pieces_for(int32_t slab_vec) { return (slab_vec + kPieceVec - 1) / kPieceVec; }
 
 }  // namespace
@@ -104,6 +129,30 @@ cudaError_t launch_scatter_layer(void* kpool, void* vpool, const int32_t* d_ids,
     if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
     layer_copy_kernel<true><<<(unsigned)grid, kCopyThreads, 0, stream>>>(
         (uint4*)kpool, (uint4*)vpool, d_ids, (uint4*)const_cast<void*>(src), slab_vec, pieces, num_blocks, d_status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_scatter_layer_ids(void* kpool, void* vpool, const int32_t* h_ids, int32_t n, const void* src,
+                                     int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream) {
+    if (n <= 0) return cudaSuccess;
+    if (n > kMaxParamIds) return cudaErrorInvalidValue;
+    ParamIds ids;
+    for (int32_t i = 0; i < n; ++i) ids.ids[i] = h_ids[i];
+    for (int32_t i = n; i < kMaxParamIds; ++i) ids.ids[i] = 0;
+    const int pieces = pieces_for(slab_vec);
+    const int64_t grid = 2LL * n * pieces;
+    scatter_param_ids_kernel<<<(unsigned)grid, kCopyThreads, 0, stream>>>(
+        (uint4*)kpool, (uint4*)vpool, ids, (const uint4*)src, slab_vec, pieces, num_blocks, d_status);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_upload(void* dst, const void* src_mapped, size_t bytes, cudaStream_t stream) {
+    if (bytes == 0) return cudaSuccess;
+    if (bytes % 16) return cudaErrorInvalidValue;
+    const int64_t n_vec = (int64_t)(bytes / 16);
+    const int64_t want = (n_vec + 255) / 256;
+    const unsigned grid = (unsigned)(want < 64 ? want : 64);
+    upload_kernel<<<grid, 256, 0, stream>>>((uint4*)dst, (const uint4*)src_mapped, n_vec);
     return cudaGetLastError();
 }
 

@@ -22,6 +22,17 @@ cudaError_t launch_gather_image(const void* const* d_kpools, const void* const* 
 cudaError_t launch_scatter_layer(void* kpool, void* vpool, const int32_t* d_ids, int32_t n, const void* src,
                                  int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
 
+// Same, with the block ids passed by value in the kernel parameters (no descriptor upload at all);
+// h_ids is a host array, n <= kMaxParamIds per call.
+constexpr int kMaxParamIds = 960;
+cudaError_t launch_scatter_layer_ids(void* kpool, void* vpool, const int32_t* h_ids, int32_t n, const void* src,
+                                     int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
+
+// Copies `bytes` (a multiple of 16) from mapped pinned host memory (device view src) to device
+// memory with a small kernel, so that descriptor uploads never queue behind bulk transfers in a
+// copy engine.
+cudaError_t launch_upload(void* dst, const void* src_mapped, size_t bytes, cudaStream_t stream);
+
 // Gather for one layer into the same pair layout (the inverse of launch_scatter_layer).
 cudaError_t launch_gather_layer(const void* kpool, const void* vpool, const int32_t* d_ids, int32_t n, void* dst,
                                 int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
@@ -49,6 +60,7 @@ struct AttnBatch {                 // device pointers to the per-batch metadata
     const AttnItem* items;         // [n_items]
     const int32_t* row_first_part; // [B] first partial slot of the row
     const int32_t* row_parts;      // [B] number of partial slots of the row
+    const int32_t* row_lane;       // [B] 0 = main lane, 1 = reload lane (attention waits on reload events)
     int32_t table_stride;
     int32_t batch;
 };
@@ -62,9 +74,10 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
                                void* out, float* lse, const AttnBatch& batch, int32_t item_begin, int32_t item_end,
                                float* partials, int32_t* d_status, cudaStream_t stream);
 
-// Merges the partial results of every row with more than one part into out / lse.
+// Merges the partial results of every row with more than one part into out / lse.  lane: 0 or 1
+// restricts the merge to the rows of that lane, -1 takes all rows.
 cudaError_t launch_attn_merge(const AttnShape& sh, void* out, float* lse, const AttnBatch& batch,
-                              const float* partials, cudaStream_t stream);
+                              const float* partials, int32_t lane, cudaStream_t stream);
 
 // Whether the tensor-core kernel supports the shape.
 bool attn_mma_supported(const AttnShape& sh);

@@ -50,8 +50,9 @@ struct Tracker {  // completion tickets on one stream
     uint64_t next = 1, done = 0;
 };
 
-struct Arena {  // pinned + device ring of chunks for descriptor uploads on ONE stream
-    char* h = nullptr;
+struct Arena {  // pinned (mapped) + device ring of chunks for descriptor uploads on ONE stream
+    char* h = nullptr;   // host view of the pinned buffer
+    char* hd = nullptr;  // device view of the same pinned buffer (source of the upload kernel)
     char* d = nullptr;
     size_t chunk = 0;
     int nchunks = 0, cur = 0;
@@ -120,7 +121,7 @@ struct BatchMeta {  // cached device metadata of the last prepared decode batch
     ps::AttnBatch dev{};
     int32_t n_items = 0, n_ungated_items = 0, n_parts = 0;
     int32_t n_gated_rows = 0;
-    bool any_multi = false;
+    bool any_multi = false, lane_multi[2] = {false, false};
     int64_t kv_bytes_per_layer = 0;
 };
 
@@ -147,7 +148,8 @@ struct ps_ctx {
     char* host_pool = nullptr;
     bool own_host_pool = false;
     HostPool hpool;
-    cudaStream_t compute = nullptr, s_gather = nullptr, s_d2h = nullptr, s_h2d = nullptr, s_scatter = nullptr;
+    cudaStream_t compute = nullptr, s_gather = nullptr, s_d2h = nullptr, s_h2d = nullptr, s_scatter = nullptr,
+                 s_lane = nullptr;
     char* stage_out = nullptr;
     char* stage_in = nullptr;
     int64_t slot_bytes = 0;
@@ -155,14 +157,14 @@ struct ps_ctx {
     bool out_used[kSlots]{}, in_used[kSlots]{};
     uint64_t out_next = 0, in_next = 0;
     std::vector<cudaEvent_t> ev_in;  // per layer
-    cudaEvent_t e_mark = nullptr, e_mark2 = nullptr, e_ids = nullptr;
+    cudaEvent_t e_mark = nullptr, e_mark2 = nullptr, e_ids = nullptr, e_fork = nullptr, e_join = nullptr;
     bool ids_fenced = false;
     int32_t* h_ids = nullptr;
     int32_t* d_ids = nullptr;
     int32_t* status = nullptr;  // mapped pinned word written by kernels on a bad block id
     int32_t* d_status = nullptr;
     Tracker t_d2h, t_scatter, t_compute;
-    Arena a_gather, a_scatter, a_meta;
+    Arena a_gather, a_meta;
     std::vector<cudaEvent_t> ev_pool, ev_pool_timing;
     std::deque<std::pair<uint64_t, std::pair<int64_t, int64_t>>> img_release;  // in_ticket -> (off, bytes)
     std::vector<int64_t> gated_reqs;
@@ -259,7 +261,8 @@ int32_t arena_init(ps_ctx* ctx, Arena& a, size_t chunk, int nchunks, cudaStream_
     a.s = s;
     a.cur = 0;
     a.used = 0;
-    CK(cudaHostAlloc((void**)&a.h, a.chunk * nchunks, cudaHostAllocDefault));
+    CK(cudaHostAlloc((void**)&a.h, a.chunk * nchunks, cudaHostAllocMapped));
+    CK(cudaHostGetDevicePointer((void**)&a.hd, a.h, 0));
     CK(cudaMalloc((void**)&a.d, a.chunk * nchunks));
     a.fence.resize(nchunks);
     a.fenced.assign(nchunks, 0);
@@ -448,17 +451,12 @@ int32_t issue_reload_layer(ps_ctx* ctx, int32_t layer, const std::vector<PlanEnt
         }
         CK(cudaEventRecord(ctx->e_loaded[slot], ctx->s_h2d));
         CK(cudaStreamWaitEvent(ctx->s_scatter, ctx->e_loaded[slot], 0));
-        if (!ids.empty()) {
-            size_t off = 0;
-            int32_t rc = arena_alloc(ctx, ctx->a_scatter, ids.size() * sizeof(int32_t), &off);
-            if (rc != PS_OK) return rc;
-            memcpy(ctx->a_scatter.h + off, ids.data(), ids.size() * sizeof(int32_t));
-            CK(cudaMemcpyAsync(ctx->a_scatter.d + off, ctx->a_scatter.h + off, ids.size() * sizeof(int32_t),
-                               cudaMemcpyHostToDevice, ctx->s_scatter));
-            ProfScope prof(ctx, kProfScatter, ctx->s_scatter, (int64_t)ids.size() * Bl, layer);
-            CK(ps::launch_scatter_layer(ctx->kpools[layer], ctx->vpools[layer], (const int32_t*)(ctx->a_scatter.d + off),
-                                        (int32_t)ids.size(), sp, ctx->slab_vec, ctx->cfg.num_gpu_blocks,
-                                        ctx->d_status, ctx->s_scatter));
+        for (size_t c0 = 0; c0 < ids.size(); c0 += ps::kMaxParamIds) {
+            const int32_t n = (int32_t)std::min<size_t>(ps::kMaxParamIds, ids.size() - c0);
+            ProfScope prof(ctx, kProfScatter, ctx->s_scatter, (int64_t)n * Bl, layer);
+            CK(ps::launch_scatter_layer_ids(ctx->kpools[layer], ctx->vpools[layer], ids.data() + c0, n,
+                                            sp + (int64_t)c0 * Bl, ctx->slab_vec, ctx->cfg.num_gpu_blocks,
+                                            ctx->d_status, ctx->s_scatter));
             ctx->launches++;
         }
         CK(cudaEventRecord(ctx->e_scattered[slot], ctx->s_scatter));
@@ -559,7 +557,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     std::vector<int32_t> row_first(B, 0), row_parts(B, 0), ctx_len(B, 0);
     std::vector<ps::AttnItem> items;
     int32_t parts = 0, n_ungated = 0, n_gated_rows = 0;
-    bool any_multi = false;
+    bool any_multi = false, lane_multi[2] = {false, false};
     for (int pass = 0; pass < 2; ++pass) {  // rows that need no wait first, gated rows after them
         for (int32_t b = 0; b < B; ++b) {
             if (!active[b] || (gated[b] ? 1 : 0) != pass) continue;
@@ -569,6 +567,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
             row_parts[b] = n;
             ctx_len[b] = r.n_tokens;
             any_multi |= n > 1;
+            lane_multi[pass] |= n > 1;
             for (int32_t k = 0; k < n; ++k) {
                 ps::AttnItem it{};
                 it.b = b;
@@ -588,7 +587,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     const size_t sz_tables = (size_t)round_up((int64_t)B * stride * 4, 256);
     const size_t sz_vec = (size_t)round_up((int64_t)B * 4, 256);
     const size_t sz_items = (size_t)round_up((int64_t)std::max<size_t>(items.size(), 1) * sizeof(ps::AttnItem), 256);
-    const size_t total = sz_tables + 3 * sz_vec + sz_items;
+    const size_t total = sz_tables + 4 * sz_vec + sz_items;
     if (total > ctx->a_meta.chunk) return ctx->fail(PS_ERR_INVALID, "decode batch metadata exceeds its buffer");
     // a fresh chunk: the chunk of the cached batch stays intact until this point
     int32_t rc = arena_next_chunk(ctx, ctx->a_meta, /*record_fence=*/false);
@@ -608,8 +607,13 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     memcpy(h + sz_tables, ctx_len.data(), (size_t)B * 4);
     memcpy(h + sz_tables + sz_vec, row_first.data(), (size_t)B * 4);
     memcpy(h + sz_tables + 2 * sz_vec, row_parts.data(), (size_t)B * 4);
-    if (!items.empty()) memcpy(h + sz_tables + 3 * sz_vec, items.data(), items.size() * sizeof(ps::AttnItem));
-    CK(cudaMemcpyAsync(d, h, total, cudaMemcpyHostToDevice, ctx->compute));
+    {
+        int32_t* lane = (int32_t*)(h + sz_tables + 3 * sz_vec);
+        for (int32_t b = 0; b < B; ++b) lane[b] = gated[b] ? 1 : 0;
+    }
+    if (!items.empty()) memcpy(h + sz_tables + 4 * sz_vec, items.data(), items.size() * sizeof(ps::AttnItem));
+    CK(ps::launch_upload(d, ctx->a_meta.hd + off, total, ctx->compute));
+    ctx->launches++;
     // the pinned side of this chunk may be rewritten once this upload has run
     CK(cudaEventRecord(ctx->a_meta.fence[ctx->a_meta.cur], ctx->compute));
     ctx->a_meta.fenced[ctx->a_meta.cur] = 1;
@@ -623,7 +627,8 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     m.dev.ctx_len = (const int32_t*)(d + sz_tables);
     m.dev.row_first_part = (const int32_t*)(d + sz_tables + sz_vec);
     m.dev.row_parts = (const int32_t*)(d + sz_tables + 2 * sz_vec);
-    m.dev.items = (const ps::AttnItem*)(d + sz_tables + 3 * sz_vec);
+    m.dev.row_lane = (const int32_t*)(d + sz_tables + 3 * sz_vec);
+    m.dev.items = (const ps::AttnItem*)(d + sz_tables + 4 * sz_vec);
     m.dev.table_stride = stride;
     m.dev.batch = B;
     m.n_items = (int32_t)items.size();
@@ -631,19 +636,24 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     m.n_parts = parts;
     m.n_gated_rows = n_gated_rows;
     m.any_multi = any_multi;
+    m.lane_multi[0] = lane_multi[0];
+    m.lane_multi[1] = lane_multi[1];
     m.kv_bytes_per_layer = total_tokens * 2 * ctx->cfg.num_kv_heads * ctx->cfg.head_dim * 2;
     return PS_OK;
 }
 
 // Launches one layer of attention for the prepared batch.  wait_event: the layer's reload event for
-// the gated rows (nullptr = nothing is gated).
+// the gated rows (nullptr = no wait).  lanes == false: everything on the compute stream (main rows,
+// wait, gated rows, one merge).  lanes == true: the gated rows run on the reload-lane stream behind
+// the wait, with their own merge, so the main rows of the next layer never queue behind them.
 int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, float* lse, cudaEvent_t wait_event,
-                          int32_t* n_launched) {
+                          bool lanes, int32_t* n_launched) {
     BatchMeta& m = ctx->meta;
     ps::AttnShape sh{ctx->cfg.num_kv_heads, ctx->cfg.num_q_heads, ctx->cfg.head_dim, ctx->cfg.block_size,
                      ctx->cfg.num_gpu_blocks};
     const int64_t bytes = m.kv_bytes_per_layer;
     const int64_t ungated_bytes = m.n_items ? bytes * m.n_ungated_items / m.n_items : 0;
+    const bool have_gated = m.n_items > m.n_ungated_items;
     if (m.n_ungated_items > 0) {
         ProfScope prof(ctx, kProfAttn, ctx->compute, ungated_bytes, layer);
         CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev, 0,
@@ -651,17 +661,32 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
         ctx->launches++;
         ++*n_launched;
     }
-    if (m.n_items > m.n_ungated_items) {
-        if (wait_event) CK(cudaStreamWaitEvent(ctx->compute, wait_event, 0));
-        ProfScope prof(ctx, kProfAttn, ctx->compute, bytes - ungated_bytes, 1000 + layer);
-        CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev,
-                                  m.n_ungated_items, m.n_items, ctx->partials, ctx->d_status, ctx->compute));
+    if (lanes && have_gated && m.lane_multi[0]) {
+        ProfScope prof(ctx, kProfMerge, ctx->compute, 0, layer);
+        CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials, 0, ctx->compute));
         ctx->launches++;
         ++*n_launched;
     }
-    if (m.any_multi) {
+    if (have_gated) {
+        cudaStream_t gs = lanes ? ctx->s_lane : ctx->compute;
+        if (wait_event) CK(cudaStreamWaitEvent(gs, wait_event, 0));
+        {
+            ProfScope prof(ctx, kProfAttn, gs, bytes - ungated_bytes, 1000 + layer);
+            CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev,
+                                      m.n_ungated_items, m.n_items, ctx->partials, ctx->d_status, gs));
+            ctx->launches++;
+            ++*n_launched;
+        }
+        if (lanes && m.lane_multi[1]) {
+            ProfScope prof(ctx, kProfMerge, gs, 0, 1000 + layer);
+            CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials, 1, gs));
+            ctx->launches++;
+            ++*n_launched;
+        }
+    }
+    if (!(lanes && have_gated) && m.any_multi) {
         ProfScope prof(ctx, kProfMerge, ctx->compute, 0, layer);
-        CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials, ctx->compute));
+        CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials, -1, ctx->compute));
         ctx->launches++;
         ++*n_launched;
     }
@@ -670,13 +695,13 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
 
 void destroy_ctx(ps_ctx* ctx) {
     if (!ctx->bk) {
-        for (cudaStream_t s : {ctx->s_gather, ctx->s_d2h, ctx->s_h2d, ctx->s_scatter})
+        for (cudaStream_t s : {ctx->s_gather, ctx->s_d2h, ctx->s_h2d, ctx->s_scatter, ctx->s_lane})
             if (s) cudaStreamDestroy(s);
         for (int i = 0; i < kSlots; ++i)
             for (cudaEvent_t e : {ctx->e_gathered[i], ctx->e_drained[i], ctx->e_loaded[i], ctx->e_scattered[i]})
                 if (e) cudaEventDestroy(e);
         for (cudaEvent_t e : ctx->ev_in) cudaEventDestroy(e);
-        for (cudaEvent_t e : {ctx->e_mark, ctx->e_mark2, ctx->e_ids, ctx->trace_base})
+        for (cudaEvent_t e : {ctx->e_mark, ctx->e_mark2, ctx->e_ids, ctx->e_fork, ctx->e_join, ctx->trace_base})
             if (e) cudaEventDestroy(e);
         for (auto& t : {&ctx->t_d2h, &ctx->t_scatter, &ctx->t_compute})
             for (auto& p : t->pending) cudaEventDestroy(p.second);
@@ -687,7 +712,6 @@ void destroy_ctx(ps_ctx* ctx) {
             cudaEventDestroy(sp.e1);
         }
         arena_free(ctx->a_gather);
-        arena_free(ctx->a_scatter);
         arena_free(ctx->a_meta);
         if (ctx->stage_out) cudaFree(ctx->stage_out);
         if (ctx->stage_in) cudaFree(ctx->stage_in);
@@ -820,6 +844,8 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     CKC(cudaStreamCreateWithPriority(&ctx->s_d2h, cudaStreamNonBlocking, prio_hi));
     CKC(cudaStreamCreateWithPriority(&ctx->s_h2d, cudaStreamNonBlocking, prio_hi));
     CKC(cudaStreamCreateWithPriority(&ctx->s_scatter, cudaStreamNonBlocking, prio_hi));
+    // the reload lane: attention of requests whose reload is landing in this step (same priority as compute)
+    CKC(cudaStreamCreateWithPriority(&ctx->s_lane, cudaStreamNonBlocking, prio_lo));
     ctx->t_d2h.s = ctx->s_d2h;
     ctx->t_scatter.s = ctx->s_scatter;
     ctx->t_compute.s = ctx->compute;
@@ -839,17 +865,19 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     CKC(cudaEventCreateWithFlags(&ctx->e_mark, cudaEventDisableTiming));
     CKC(cudaEventCreateWithFlags(&ctx->e_mark2, cudaEventDisableTiming));
     CKC(cudaEventCreateWithFlags(&ctx->e_ids, cudaEventDisableTiming));
+    CKC(cudaEventCreateWithFlags(&ctx->e_fork, cudaEventDisableTiming));
+    CKC(cudaEventCreateWithFlags(&ctx->e_join, cudaEventDisableTiming));
     CKC(cudaHostAlloc((void**)&ctx->status, 64, cudaHostAllocMapped));
     memset(ctx->status, 0, 64);
     CKC(cudaHostGetDevicePointer((void**)&ctx->d_status, ctx->status, 0));
     CKC(cudaHostAlloc((void**)&ctx->h_ids, sizeof(int32_t) * (size_t)cfg->num_gpu_blocks, cudaHostAllocDefault));
     CKC(cudaMalloc((void**)&ctx->d_ids, sizeof(int32_t) * (size_t)cfg->num_gpu_blocks));
 
-    // descriptor arenas: a table per swap-out; id lists per scatter launch; one decode batch per chunk
+    // descriptor arenas: a table per swap-out; one decode batch per chunk (scatter ids travel as
+    // kernel parameters).  Uploads are done by a kernel reading the mapped pinned side, so the copy
+    // engines carry bulk KV traffic only.
     const size_t desc_chunk = std::max<size_t>((size_t)cfg->max_blocks_per_req * 4 * 8, 1 << 20);
     CKR(arena_init(ctx, ctx->a_gather, desc_chunk, 4, ctx->s_gather));
-    CKR(arena_init(ctx, ctx->a_scatter, std::max<size_t>(desc_chunk, (size_t)(ctx->slot_bytes / ctx->layer_block_bytes) * 4 * 4),
-                   4, ctx->s_scatter));
 
     // split-KV scratch
     ctx->attn_kernel = PS_ATTN_SIMT;
@@ -990,8 +1018,9 @@ int32_t ps_swap_out(ps_ctx* ctx, int64_t req) {
             ctx->hpool.release(off, bytes);
             return ctx->fail_cuda(ce, what);
         };
-        e = cudaMemcpyAsync(ctx->a_gather.d + toff, ctx->a_gather.h + toff, (size_t)n_blk * 4, cudaMemcpyHostToDevice,
-                            ctx->s_gather);
+        e = ps::launch_upload(ctx->a_gather.d + toff, ctx->a_gather.hd + toff, (size_t)round_up(n_blk * 4, 16),
+                              ctx->s_gather);
+        ctx->launches++;
         if (e != cudaSuccess) return bail(e, "table upload");
         const int64_t total_slabs = 2 * n_blk * ctx->cfg.num_layers;
         const int64_t slot_slabs = ctx->slot_bytes / ctx->slab_bytes;
@@ -1142,7 +1171,7 @@ int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, flo
     if (rc != PS_OK) return rc;
     int32_t launched = 0;
     return launch_layer_attn(ctx, layer, q, out, lse, ctx->meta.n_gated_rows ? ctx->ev_in[(size_t)layer] : nullptr,
-                             &launched);
+                             /*lanes=*/false, &launched);
 }
 
 int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs, int32_t batch,
@@ -1208,6 +1237,11 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
     if (attn) {
         const int64_t layer_bytes = (int64_t)batch * ctx->cfg.num_q_heads * ctx->cfg.head_dim * 2;
         const bool any_gated = ctx->meta.n_gated_rows > 0;
+        const bool lanes = any_gated && !sync_reload;
+        if (lanes) {  // the reload lane starts where the compute stream stands now (metadata uploaded)
+            CK(cudaEventRecord(ctx->e_fork, ctx->compute));
+            CK(cudaStreamWaitEvent(ctx->s_lane, ctx->e_fork, 0));
+        }
         for (int l = 0; l < L; ++l) {
             if (!sync_reload) {
                 rc = issue_reload_layer(ctx, l, plan);
@@ -1222,8 +1256,12 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
             }
             int32_t launched = 0;
             rc = launch_layer_attn(ctx, l, (const char*)q_all_layers + l * layer_bytes,
-                                   (char*)out_all_layers + l * layer_bytes, nullptr, wait, &launched);
+                                   (char*)out_all_layers + l * layer_bytes, nullptr, wait, lanes, &launched);
             if (rc != PS_OK) return rc;
+        }
+        if (lanes) {  // the step is complete on the compute stream only when the reload lane is
+            CK(cudaEventRecord(ctx->e_join, ctx->s_lane));
+            CK(cudaStreamWaitEvent(ctx->compute, ctx->e_join, 0));
         }
     }
 
