@@ -569,7 +569,7 @@ def main():
     ap.add_argument("--steps", type=int, default=3)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--budget-mib", type=int, default=256, help="copy budget per step in MiB for phase B (-1 = unlimited)")
+    ap.add_argument("--budget-mib", type=int, default=-1, help="copy budget per step in MiB for phase B (-1 = unlimited)")
     ap.add_argument("--no-overlap", action="store_true", help="skip the overlap budget sweep")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     args = ap.parse_args()

@@ -250,23 +250,335 @@ cudaError_t launch_simt(const AttnShape& sh, const void* kpool, const void* vpoo
     return cudaGetLastError();
 }
 
+
+// ------------------------------------------------------------------------------------------------
+// Tensor-core kernel (head_dim 128, 8 KV heads, block size a multiple of 16).
+//
+// Work: the lane's contexts are cut into 16-token tiles; the tiles of all rows form one sequence
+// that is divided evenly over the CTAs (one per SM), so every CTA streams the same number of bytes
+// whatever the context-length mix.  A CTA walks its items (row, token range); consecutive items
+// keep the copy pipeline full across row boundaries.
+//
+// Data path: a tile is 16 token rows of K and 16 of V; a token row holds all 8 KV heads (2 KiB,
+// contiguous in the pool).  One producer thread issues a bulk async copy (TMA) per row into a
+// 3-stage shared-memory ring, signalled through mbarriers; rows sit at a 2064-byte pitch so that
+// ldmatrix over 8 tokens of one head touches 8 different bank groups.  Rows past the end of a
+// context are never copied (the ring is zeroed once, so a stale row is always finite).
+//
+// Math: warp w owns KV head w.  Scores: mma.m16n8k16 with the G query heads of the group as the
+// M rows (padded to 16) and 8 tokens as N; softmax statistics per query head are reduced over the
+// 4 lanes of a quad with shuffles; P is re-packed in registers as the A operand of P.V with V read
+// through ldmatrix.trans.  Tensor cores are used to keep the FMA work off the ALUs: the kernel is
+// bound by HBM (G flop per KV byte), not by the tensor pipe.
+// ------------------------------------------------------------------------------------------------
+constexpr int kMmaD = 128;
+constexpr int kMmaHkv = 8;
+constexpr int kMmaStages = 3;
+constexpr int kMmaRowBytes = kMmaHkv * kMmaD * 2;         // 2048: one token, all KV heads
+constexpr int kMmaPitch = kMmaRowBytes + 16;              // 2064: breaks the 2 KiB bank alignment
+constexpr int kMmaSlabBytes = kMmaTileTokens * kMmaPitch; // one K (or V) tile in shared memory
+constexpr int kMmaStageBytes = 2 * kMmaSlabBytes;
+constexpr int kMmaRingBytes = kMmaStages * kMmaStageBytes;
+constexpr int kMmaSmemBytes = kMmaRingBytes + 64;         // + barriers and the abort word
+constexpr int kMmaConsumerWarps = kMmaHkv;
+constexpr int kMmaThreads = (kMmaConsumerWarps + 1) * 32;
+constexpr int kSpinLimit = 1 << 22;
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls (a fraction of a second), raises the CTA's abort
+// word and reports through the status word instead of spinning for ever.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int32_t* abort_word,
+                                          int32_t* status) {
+    for (int i = 0; i < kSpinLimit; ++i) {
+        if (mbar_test(bar, parity)) return true;
+        if (*abort_word) return false;
+        if (i > 32) __nanosleep(40);
+    }
+    *abort_word = 1;
+    *(volatile int32_t*)status = 3;
+    return false;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+template <int G>
+__global__ void __launch_bounds__(kMmaThreads, 1)
+decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloat16* __restrict__ vpool,
+                       const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
+                       AttnBatch batch, const int32_t* __restrict__ cta_begin, int32_t block_size, int32_t block_shift,
+                       int32_t num_blocks, float* __restrict__ partials, float scale_log2e, int32_t* status) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int Hq = kMmaHkv * G;
+    const uint32_t ring = smem_u32(smem);
+    const uint32_t bar_full = ring + kMmaRingBytes;        // kMmaStages x 8 bytes
+    const uint32_t bar_empty = bar_full + 8 * kMmaStages;  // kMmaStages x 8 bytes
+    volatile int32_t* abort_word = reinterpret_cast<volatile int32_t*>(smem + kMmaRingBytes + 16 * kMmaStages);
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    // one-time set-up: barriers, a finite ring
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kMmaStages; ++s) {
+            mbar_init(bar_full + 8 * s, 1);
+            mbar_init(bar_empty + 8 * s, kMmaConsumerWarps);
+        }
+        *abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    for (int i = threadIdx.x; i < kMmaRingBytes / 16; i += kMmaThreads)
+        reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy zeroes before async-proxy writes
+    __syncthreads();
+
+    const int item0 = cta_begin[blockIdx.x];
+    const int item1 = cta_begin[blockIdx.x + 1];
+
+    if (warp == kMmaConsumerWarps) {
+        // ------------------------------------------------ producer: one thread feeds the ring
+        if (lane == 0) {
+            int n = 0;
+            bool ok = true;
+            for (int it = item0; it < item1 && ok; ++it) {
+                const AttnItem item = batch.items[it];
+                const int32_t* table = batch.block_tables + (int64_t)item.b * batch.table_stride;
+                for (int t0 = item.t_begin; t0 < item.t_end && ok; t0 += kMmaTileTokens, ++n) {
+                    const int s = n % kMmaStages;
+                    if (n >= kMmaStages)
+                        ok = mbar_wait(bar_empty + 8 * s, ((n / kMmaStages) - 1) & 1, abort_word, status);
+                    if (!ok) break;
+                    const int rows = min(kMmaTileTokens, item.t_end - t0);
+                    const int blk = block_shift >= 0 ? (t0 >> block_shift) : (t0 / block_size);
+                    const int slot = t0 - blk * block_size;
+                    const int id = table[blk];
+                    const uint32_t full = bar_full + 8 * s;
+                    if ((unsigned)id >= (unsigned)num_blocks) {
+                        // skip the copy: consumers see the previous (finite) contents; the host sees the error
+                        *(volatile int32_t*)status = 2;
+                        mbar_arrive(full);
+                        continue;
+                    }
+                    mbar_expect_tx(full, (uint32_t)rows * 2u * kMmaRowBytes);
+                    const int64_t off = ((int64_t)id * block_size + slot) * (kMmaRowBytes / 2);  // elements
+                    const uint32_t ks = ring + s * kMmaStageBytes;
+                    const uint32_t vs = ks + kMmaSlabBytes;
+                    for (int r = 0; r < rows; ++r) {
+                        bulk_g2s(ks + r * kMmaPitch, kpool + off + (int64_t)r * (kMmaRowBytes / 2), kMmaRowBytes, full);
+                        bulk_g2s(vs + r * kMmaPitch, vpool + off + (int64_t)r * (kMmaRowBytes / 2), kMmaRowBytes, full);
+                    }
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------ consumers: warp = KV head
+        const int g = lane >> 2;  // row of the mma tile = query head inside the group (valid if g < G)
+        const int t = lane & 3;
+        const int h = warp;
+        // ldmatrix row addresses (byte offsets inside a slab), see the layout comments above
+        const int ld_row = lane & 7;
+        const int ld_mat = lane >> 3;
+        // K (no transpose): matrices {tok 0-7, d lo}, {tok 0-7, d hi}, {tok 8-15, d lo}, {tok 8-15, d hi}
+        const uint32_t k_lane_off = (uint32_t)((ld_row + ((ld_mat & 2) ? 8 : 0)) * kMmaPitch + h * 256 + ((ld_mat & 1) ? 16 : 0));
+        // V (transpose): matrices {tok 0-7, d lo}, {tok 8-15, d lo}, {tok 0-7, d hi}, {tok 8-15, d hi}
+        const uint32_t v_lane_off = (uint32_t)((ld_row + ((ld_mat & 1) ? 8 : 0)) * kMmaPitch + h * 256 + ((ld_mat & 2) ? 16 : 0));
+        int n = 0;
+        bool ok = true;
+        for (int it = item0; it < item1 && ok; ++it) {
+            const AttnItem item = batch.items[it];
+            // Q fragments of this head group: rows g < G are real, everything else is zero
+            uint32_t qa[8][2];
+            {
+                const __nv_bfloat16* qrow = q + ((int64_t)item.b * Hq + h * G + g) * kMmaD;
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    qa[j][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 2 * t) : 0u;
+                    qa[j][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 8 + 2 * t) : 0u;
+                }
+            }
+            float o[16][4];
+#pragma unroll
+            for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
+            float m_run = kNegBig, l_run = 0.f;
+
+            for (int t0 = item.t_begin; t0 < item.t_end; t0 += kMmaTileTokens, ++n) {
+                const int s = n % kMmaStages;
+                ok = mbar_wait(bar_full + 8 * s, (n / kMmaStages) & 1, abort_word, status);
+                ok = __all_sync(0xffffffffu, ok);  // the warp leaves together (full-mask shuffles below)
+                if (!ok) break;
+                const int rows = min(kMmaTileTokens, item.t_end - t0);
+                const uint32_t ks = ring + s * kMmaStageBytes;
+                const uint32_t vs = ks + kMmaSlabBytes;
+
+                // scores for 16 tokens: two n-tiles of 8 tokens
+                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4(ks + k_lane_off + 32 * j, b0, b1, b2, b3);
+                    mma_bf16(s0, qa[j][0], 0u, qa[j][1], 0u, b0, b1);
+                    mma_bf16(s1, qa[j][0], 0u, qa[j][1], 0u, b2, b3);
+                }
+                // this lane's four tokens of row g: 2t, 2t+1, 8+2t, 9+2t
+                float x0 = s0[0] * scale_log2e, x1 = s0[1] * scale_log2e;
+                float x2 = s1[0] * scale_log2e, x3 = s1[1] * scale_log2e;
+                const bool v0 = 2 * t < rows, v1 = 2 * t + 1 < rows, v2 = 8 + 2 * t < rows, v3 = 9 + 2 * t < rows;
+                float mx = kNegBig;
+                if (v0) mx = fmaxf(mx, x0);
+                if (v1) mx = fmaxf(mx, x1);
+                if (v2) mx = fmaxf(mx, x2);
+                if (v3) mx = fmaxf(mx, x3);
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                const float m_new = fmaxf(m_run, mx);
+                const float alpha = exp2f(m_run - m_new);
+                m_run = m_new;
+                const float p0 = v0 ? exp2f(x0 - m_new) : 0.f;
+                const float p1 = v1 ? exp2f(x1 - m_new) : 0.f;
+                const float p2 = v2 ? exp2f(x2 - m_new) : 0.f;
+                const float p3 = v3 ? exp2f(x3 - m_new) : 0.f;
+                l_run = l_run * alpha + (p0 + p1 + p2 + p3);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    o[i][0] *= alpha;
+                    o[i][1] *= alpha;
+                }
+                const uint32_t pa0 = pack_bf16(p0, p1);  // row g, tokens 2t, 2t+1
+                const uint32_t pa2 = pack_bf16(p2, p3);  // row g, tokens 8+2t, 9+2t
+#pragma unroll
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4_t(vs + v_lane_off + 32 * c, b0, b1, b2, b3);
+                    mma_bf16(o[2 * c], pa0, 0u, pa2, 0u, b0, b1);
+                    mma_bf16(o[2 * c + 1], pa0, 0u, pa2, 0u, b2, b3);
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar_empty + 8 * s);
+            }
+            if (!ok) break;
+
+            // finalise the item for row g
+            float L = l_run;
+            L += __shfl_xor_sync(0xffffffffu, L, 1);
+            L += __shfl_xor_sync(0xffffffffu, L, 2);
+            if (g < G) {
+                const int hq = h * G + g;
+                if (item.n_parts == 1) {
+                    const float inv = L > 0.f ? 1.f / L : 0.f;
+                    __nv_bfloat16* orow = out + ((int64_t)item.b * Hq + hq) * kMmaD;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        *reinterpret_cast<uint32_t*>(orow + 8 * i + 2 * t) = pack_bf16(o[i][0] * inv, o[i][1] * inv);
+                    if (lse != nullptr && t == 0)
+                        lse[(int64_t)item.b * Hq + hq] = L > 0.f ? (m_run + log2f(L)) * kLn2 : -CUDART_INF_F;
+                } else {
+                    float* pr = partials + ((int64_t)item.part * Hq + hq) * (kMmaD + 2);
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        *reinterpret_cast<float2*>(pr + 8 * i + 2 * t) = make_float2(o[i][0], o[i][1]);
+                    if (t == 0) {
+                        pr[kMmaD] = m_run;
+                        pr[kMmaD + 1] = L;
+                    }
+                }
+            }
+        }
+    }
+}
+
+template <int G>
+cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool, const void* q, void* out, float* lse,
+                       const AttnBatch& batch, int32_t lane, float* partials, int32_t* d_status, cudaStream_t stream) {
+    const float scale_log2e = 1.4426950408889634f / sqrtf((float)kMmaD);
+    decode_attn_mma_kernel<G><<<(unsigned)batch.n_cta[lane], kMmaThreads, kMmaSmemBytes, stream>>>(
+        (const __nv_bfloat16*)kpool, (const __nv_bfloat16*)vpool, (const __nv_bfloat16*)q, (__nv_bfloat16*)out, lse, batch,
+        batch.cta_begin[lane], sh.block_size, shift_of(sh.block_size), sh.num_blocks, partials, scale_log2e, d_status);
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 size_t attn_partial_bytes(const AttnShape& sh, int32_t max_parts) {
     return (size_t)max_parts * sh.num_q_heads * (sh.head_dim + 2) * sizeof(float);
 }
 
-bool attn_mma_supported(const AttnShape&) { return false; }
+bool attn_mma_supported(const AttnShape& sh) {
+    const int G = sh.num_q_heads / sh.num_kv_heads;
+    return sh.head_dim == kMmaD && sh.num_kv_heads == kMmaHkv && (G == 1 || G == 2 || G == 4 || G == 8) &&
+           sh.block_size % kMmaTileTokens == 0;
+}
 
-cudaError_t attn_init() { return cudaSuccess; }
+cudaError_t attn_init() {
+    cudaError_t e;
+#define PS_MMA_ATTR(GG)                                                                                    \
+    e = cudaFuncSetAttribute(decode_attn_mma_kernel<GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
+                             kMmaSmemBytes);                                                               \
+    if (e != cudaSuccess) return e;
+    PS_MMA_ATTR(1) PS_MMA_ATTR(2) PS_MMA_ATTR(4) PS_MMA_ATTR(8)
+#undef PS_MMA_ATTR
+    return cudaSuccess;
+}
 
 cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool, const void* q,
-                               void* out, float* lse, const AttnBatch& batch, int32_t item_begin, int32_t item_end,
-                               float* partials, int32_t* d_status, cudaStream_t stream) {
-    const int n_items = item_end - item_begin;
+                               void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials,
+                               int32_t* d_status, cudaStream_t stream) {
+    if (lane < 0 || lane > 1) return cudaErrorInvalidValue;
+    const int item_begin = batch.lane_items[lane];
+    const int n_items = batch.lane_items[lane + 1] - item_begin;
     if (n_items <= 0) return cudaSuccess;
-    if (kernel != 1) return cudaErrorNotSupported;
     const int G = sh.num_q_heads / sh.num_kv_heads;
+    if (kernel == 2) {
+        if (!attn_mma_supported(sh) || batch.n_cta[lane] <= 0) return cudaErrorNotSupported;
+        switch (G) {
+            case 1: return launch_mma<1>(sh, kpool, vpool, q, out, lse, batch, lane, partials, d_status, stream);
+            case 2: return launch_mma<2>(sh, kpool, vpool, q, out, lse, batch, lane, partials, d_status, stream);
+            case 4: return launch_mma<4>(sh, kpool, vpool, q, out, lse, batch, lane, partials, d_status, stream);
+            case 8: return launch_mma<8>(sh, kpool, vpool, q, out, lse, batch, lane, partials, d_status, stream);
+        }
+        return cudaErrorNotSupported;
+    }
+    if (kernel != 1) return cudaErrorNotSupported;
 #define PS_SIMT_CASE(DD, GG)                                                                                       \
     if (sh.head_dim == DD && G == GG)                                                                              \
         return launch_simt<DD, GG>(sh, kpool, vpool, q, out, lse, batch, item_begin, n_items, partials, d_status, \

@@ -171,6 +171,7 @@ struct ps_ctx {
     float* partials = nullptr;
     int32_t max_parts = 0;
     int attn_kernel = 1;
+    int32_t num_sms = 1;
     BatchMeta meta;
 
     // measurement
@@ -553,32 +554,93 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
         stride = std::max<int32_t>(stride, (int32_t)r.table.size());
         total_tokens += r.n_tokens;
     }
-    const int32_t split = choose_split(ctx, total_tokens);
     std::vector<int32_t> row_first(B, 0), row_parts(B, 0), ctx_len(B, 0);
     std::vector<ps::AttnItem> items;
+    std::vector<int32_t> cta_begin[2];
     int32_t parts = 0, n_ungated = 0, n_gated_rows = 0;
     bool any_multi = false, lane_multi[2] = {false, false};
-    for (int pass = 0; pass < 2; ++pass) {  // rows that need no wait first, gated rows after them
-        for (int32_t b = 0; b < B; ++b) {
-            if (!active[b] || (gated[b] ? 1 : 0) != pass) continue;
-            const Req& r = ctx->reqs[reqs[b]];
-            const int32_t n = std::max(1, (r.n_tokens + split - 1) / split);
-            row_first[b] = parts;
-            row_parts[b] = n;
-            ctx_len[b] = r.n_tokens;
-            any_multi |= n > 1;
-            lane_multi[pass] |= n > 1;
-            for (int32_t k = 0; k < n; ++k) {
-                ps::AttnItem it{};
-                it.b = b;
-                it.t_begin = k * split;
-                it.t_end = std::min(r.n_tokens, (k + 1) * split);
-                it.part = parts + k;
-                it.n_parts = n;
-                items.push_back(it);
+    const bool mma = ctx->attn_kernel == PS_ATTN_MMA;
+    const int32_t split = mma ? 0 : choose_split(ctx, total_tokens);
+    for (int pass = 0; pass < 2; ++pass) {  // lane 0: rows that need no wait; lane 1: gated rows
+        if (!mma) {
+            // SIMT kernel: one CTA per (item, KV head); items are fixed-size token ranges of a row
+            for (int32_t b = 0; b < B; ++b) {
+                if (!active[b] || (gated[b] ? 1 : 0) != pass) continue;
+                const Req& r = ctx->reqs[reqs[b]];
+                const int32_t n = std::max(1, (r.n_tokens + split - 1) / split);
+                row_first[b] = parts;
+                row_parts[b] = n;
+                ctx_len[b] = r.n_tokens;
+                any_multi |= n > 1;
+                lane_multi[pass] |= n > 1;
+                for (int32_t k = 0; k < n; ++k) {
+                    ps::AttnItem it{};
+                    it.b = b;
+                    it.t_begin = k * split;
+                    it.t_end = std::min(r.n_tokens, (k + 1) * split);
+                    it.part = parts + k;
+                    it.n_parts = n;
+                    items.push_back(it);
+                }
+                parts += n;
+                if (pass == 1) ++n_gated_rows;
             }
-            parts += n;
-            if (pass == 1) ++n_gated_rows;
+        } else {
+            // Tensor-core kernel: the lane's 16-token tiles form one sequence, cut into equal shares,
+            // one per CTA; an item is the part of a row that falls into one CTA's share.
+            constexpr int kTile = ps::kMmaTileTokens;
+            constexpr int64_t kMinTilesPerCta = 8;
+            int64_t total_tiles = 0;
+            int32_t lane_rows = 0;
+            for (int32_t b = 0; b < B; ++b)
+                if (active[b] && (gated[b] ? 1 : 0) == pass) {
+                    total_tiles += (ctx->reqs[reqs[b]].n_tokens + kTile - 1) / kTile;
+                    ++lane_rows;
+                }
+            int64_t n_cta = 0;
+            if (lane_rows > 0)
+                n_cta = std::min<int64_t>(std::max<int64_t>((total_tiles + kMinTilesPerCta - 1) / kMinTilesPerCta, 1),
+                                          ctx->num_sms);
+            const int64_t per = n_cta > 0 ? std::max<int64_t>((total_tiles + n_cta - 1) / n_cta, 1) : 1;
+            int64_t filled = 0;
+            if (n_cta > 0) cta_begin[pass].push_back((int32_t)items.size());
+            for (int32_t b = 0; b < B; ++b) {
+                if (!active[b] || (gated[b] ? 1 : 0) != pass) continue;
+                const Req& r = ctx->reqs[reqs[b]];
+                const int64_t tiles_b = (r.n_tokens + kTile - 1) / kTile;
+                const size_t first_item = items.size();
+                ctx_len[b] = r.n_tokens;
+                row_first[b] = parts;
+                if (tiles_b == 0) {  // empty context: one item without tiles writes the zero row
+                    ps::AttnItem it{};
+                    it.b = b;
+                    it.part = parts;
+                    items.push_back(it);
+                }
+                for (int64_t lo = 0; lo < tiles_b;) {
+                    if (filled == per && (int64_t)cta_begin[pass].size() < n_cta) {
+                        cta_begin[pass].push_back((int32_t)items.size());
+                        filled = 0;
+                    }
+                    const int64_t take = std::min(tiles_b - lo, per - filled);
+                    ps::AttnItem it{};
+                    it.b = b;
+                    it.t_begin = (int32_t)(lo * kTile);
+                    it.t_end = (int32_t)std::min<int64_t>(r.n_tokens, (lo + take) * kTile);
+                    it.part = parts + (int32_t)(items.size() - first_item);
+                    items.push_back(it);
+                    lo += take;
+                    filled += take;
+                }
+                const int32_t n = (int32_t)(items.size() - first_item);
+                for (size_t k = first_item; k < items.size(); ++k) items[k].n_parts = n;
+                row_parts[b] = n;
+                parts += n;
+                any_multi |= n > 1;
+                lane_multi[pass] |= n > 1;
+                if (pass == 1) ++n_gated_rows;
+            }
+            while (n_cta > 0 && (int64_t)cta_begin[pass].size() < n_cta + 1) cta_begin[pass].push_back((int32_t)items.size());
         }
         if (pass == 0) n_ungated = (int32_t)items.size();
     }
@@ -587,7 +649,8 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     const size_t sz_tables = (size_t)round_up((int64_t)B * stride * 4, 256);
     const size_t sz_vec = (size_t)round_up((int64_t)B * 4, 256);
     const size_t sz_items = (size_t)round_up((int64_t)std::max<size_t>(items.size(), 1) * sizeof(ps::AttnItem), 256);
-    const size_t total = sz_tables + 4 * sz_vec + sz_items;
+    const size_t sz_cta = (size_t)round_up((int64_t)(cta_begin[0].size() + cta_begin[1].size() + 2) * 4, 256);
+    const size_t total = sz_tables + 4 * sz_vec + sz_items + sz_cta;
     if (total > ctx->a_meta.chunk) return ctx->fail(PS_ERR_INVALID, "decode batch metadata exceeds its buffer");
     // a fresh chunk: the chunk of the cached batch stays intact until this point
     int32_t rc = arena_next_chunk(ctx, ctx->a_meta, /*record_fence=*/false);
@@ -612,6 +675,11 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
         for (int32_t b = 0; b < B; ++b) lane[b] = gated[b] ? 1 : 0;
     }
     if (!items.empty()) memcpy(h + sz_tables + 4 * sz_vec, items.data(), items.size() * sizeof(ps::AttnItem));
+    {
+        int32_t* cb = (int32_t*)(h + sz_tables + 4 * sz_vec + sz_items);
+        if (!cta_begin[0].empty()) memcpy(cb, cta_begin[0].data(), cta_begin[0].size() * 4);
+        if (!cta_begin[1].empty()) memcpy(cb + cta_begin[0].size(), cta_begin[1].data(), cta_begin[1].size() * 4);
+    }
     CK(ps::launch_upload(d, ctx->a_meta.hd + off, total, ctx->compute));
     ctx->launches++;
     // the pinned side of this chunk may be rewritten once this upload has run
@@ -629,6 +697,16 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     m.dev.row_parts = (const int32_t*)(d + sz_tables + 2 * sz_vec);
     m.dev.row_lane = (const int32_t*)(d + sz_tables + 3 * sz_vec);
     m.dev.items = (const ps::AttnItem*)(d + sz_tables + 4 * sz_vec);
+    {
+        const int32_t* cb = (const int32_t*)(d + sz_tables + 4 * sz_vec + sz_items);
+        m.dev.cta_begin[0] = cb;
+        m.dev.cta_begin[1] = cb + cta_begin[0].size();
+        m.dev.n_cta[0] = cta_begin[0].empty() ? 0 : (int32_t)cta_begin[0].size() - 1;
+        m.dev.n_cta[1] = cta_begin[1].empty() ? 0 : (int32_t)cta_begin[1].size() - 1;
+        m.dev.lane_items[0] = 0;
+        m.dev.lane_items[1] = n_ungated;
+        m.dev.lane_items[2] = (int32_t)items.size();
+    }
     m.dev.table_stride = stride;
     m.dev.batch = B;
     m.n_items = (int32_t)items.size();
@@ -657,7 +735,7 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
     if (m.n_ungated_items > 0) {
         ProfScope prof(ctx, kProfAttn, ctx->compute, ungated_bytes, layer);
         CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev, 0,
-                                  m.n_ungated_items, ctx->partials, ctx->d_status, ctx->compute));
+                                  ctx->partials, ctx->d_status, ctx->compute));
         ctx->launches++;
         ++*n_launched;
     }
@@ -673,7 +751,7 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
         {
             ProfScope prof(ctx, kProfAttn, gs, bytes - ungated_bytes, 1000 + layer);
             CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev,
-                                      m.n_ungated_items, m.n_items, ctx->partials, ctx->d_status, gs));
+                                      1, ctx->partials, ctx->d_status, gs));
             ctx->launches++;
             ++*n_launched;
         }
@@ -897,10 +975,18 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
         } else {
             max_parts = std::max<int64_t>(1, 4096 / cfg->num_kv_heads) + max_batch;
         }
+        {
+            int dev = 0, sms = 0;
+            CKC(cudaGetDevice(&dev));
+            CKC(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+            ctx->num_sms = std::max(sms, 1);
+        }
+        // the tensor-core kernel cuts a lane into at most num_sms shares: rows + shares parts per lane
+        max_parts = std::max<int64_t>(max_parts, max_batch + 2 * (int64_t)ctx->num_sms + 8);
         ctx->max_parts = (int32_t)std::min<int64_t>(max_parts, 1 << 22);
         CKC(cudaMalloc((void**)&ctx->partials, ps::attn_partial_bytes(sh, ctx->max_parts)));
-        const size_t meta_chunk = (size_t)max_batch * cfg->max_blocks_per_req * 4 + (size_t)max_batch * 12 +
-                                  (size_t)ctx->max_parts * sizeof(ps::AttnItem) + 4096;
+        const size_t meta_chunk = (size_t)max_batch * cfg->max_blocks_per_req * 4 + (size_t)max_batch * 16 +
+                                  (size_t)ctx->max_parts * sizeof(ps::AttnItem) + (size_t)ctx->num_sms * 8 + 8192;
         CKR(arena_init(ctx, ctx->a_meta, meta_chunk, 3, ctx->compute));
     }
 #undef CKC

@@ -115,6 +115,13 @@ SHAPES = [
     (8, 32, 128, 16, B.PS_ATTN_SIMT, 0),
     (2, 16, 128, 16, B.PS_ATTN_SIMT, 48),
     (2, 4, 128, 24, B.PS_ATTN_SIMT, 100),      # block size that is not a power of two, ragged split
+    # tensor-core kernel (head_dim 128, 8 KV heads): every group size, block sizes 16 / 32 / 48
+    (8, 8, 128, 16, B.PS_ATTN_MMA, 0),
+    (8, 16, 128, 16, B.PS_ATTN_MMA, 0),
+    (8, 32, 128, 16, B.PS_ATTN_MMA, 0),
+    (8, 64, 128, 16, B.PS_ATTN_MMA, 0),
+    (8, 64, 128, 32, B.PS_ATTN_MMA, 0),
+    (8, 32, 128, 48, B.PS_ATTN_MMA, 0),
 ]
 
 
@@ -122,7 +129,7 @@ SHAPES = [
 def test_decode_attn_shapes_ragged_contexts(Hkv, Hq, D, S, kernel, split):
     L, nb = 2, 160
     sh = wl.KVShape(L, Hkv, Hq, D, S, nb)
-    rng = np.random.default_rng([Hkv, Hq, D, S, split])
+    rng = np.random.default_rng([Hkv, Hq, D, S, split, kernel])
     K = wl.randn_bf16_bits(rng, (L, nb, S, Hkv, D))
     V = wl.randn_bf16_bits(rng, (L, nb, S, Hkv, D))
     p = Pair(sh, rng.permutation(nb), K, V, max_batch=16, attn_kernel=kernel, kv_split_tokens=split)
