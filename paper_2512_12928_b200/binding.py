@@ -15,7 +15,8 @@ import os
 from typing import List, Optional, Sequence, Tuple
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "lib", "libps_kvswap.so")
+# PS_KVSWAP_LIB selects another build of the same library (e.g. one with -G or extra checks)
+LIB_PATH = os.environ.get("PS_KVSWAP_LIB") or os.path.join(_PKG, "lib", "libps_kvswap.so")
 
 # status codes / states / flags (values fixed by include/ps_kvswap.h)
 PS_OK, PS_ERR_INVALID, PS_ERR_NOMEM, PS_ERR_HOST_NOMEM = 0, -1, -2, -3
