@@ -254,22 +254,31 @@ cudaError_t launch_simt(const AttnShape& sh, const void* kpool, const void* vpoo
 // ------------------------------------------------------------------------------------------------
 // Tensor-core kernel (head_dim 128, 8 KV heads, block size a multiple of 16).
 //
-// Work: the lane's contexts are cut into 16-token tiles; the tiles of all rows form one sequence
-// that is divided evenly over the CTAs (one per SM), so every CTA streams the same number of bytes
-// whatever the context-length mix.  A CTA walks its items (row, token range); consecutive items
-// keep the copy pipeline full across row boundaries.
+// Work: the lane's contexts are cut into 16-token tiles forming one sequence.  Its first ~85 % is
+// divided evenly over the CTAs (one per SM): every CTA streams the same number of bytes whatever
+// the context-length mix.  The rest is cut into small chunks handed out through an atomic counter
+// to whichever CTA finishes first, so that an SM slowed down by a neighbour (scatter kernels, the
+// reload lane) does not stretch the launch.  An item is a (row, token range); each item produces
+// one result (final if it covers the whole row, else a partial for the merge kernel).
 //
 // Data path: a tile is 16 token rows of K and 16 of V; a token row holds all 8 KV heads (2 KiB,
-// contiguous in the pool).  A producer warp issues one bulk async copy (TMA) per row into a
-// 3-stage shared-memory ring, signalled through mbarriers; rows sit at a 2064-byte pitch so that
-// ldmatrix over 8 tokens of one head touches 8 different bank groups.  Rows past the end of a
-// context are never copied (the ring is zeroed once, so a stale row is always finite).
+// contiguous in the pool).  The producer warp issues one bulk async copy (TMA) per row -- lane r
+// the K row r, lane 16 + r the V row r -- into a 3-stage shared-memory ring signalled through
+// mbarriers; next to each stage it publishes which item and tile the stage holds, and the
+// consumers follow that stream.  Rows sit at a 2064-byte pitch so that ldmatrix over 8 tokens of one
+// head touches 8 different bank groups.  Rows past the end of a context are never copied (the ring
+// is zeroed once, so a stale row is always finite).
 //
-// Math: warp w owns KV head w.  Scores: mma.m16n8k16 with the G query heads of the group as the
-// M rows (padded to 16) and 8 tokens as N; softmax statistics per query head are reduced over the
-// 4 lanes of a quad with shuffles; P is re-packed in registers as the A operand of P.V with V read
-// through ldmatrix.trans.  Tensor cores are used to keep the FMA work off the ALUs: the kernel is
-// bound by HBM (G flop per KV byte), not by the tensor pipe.
+// Math: KV head h is served by two warps, one per 8-token half of the tile (16 consumer warps keep
+// enough independent instruction streams in flight to cover the mma / ldmatrix latencies).
+// Scores: mma.m16n8k16 with the G query heads of the group as the M rows (padded to 16) and the 8
+// tokens as N; softmax statistics per query head are reduced over the 4 lanes of a quad with
+// shuffles; P is re-packed in registers as the A operand of P.V (mma.m16n8k8) with V read through
+// ldmatrix.trans.  At the end of an item the two halves are combined through shared memory.
+// Tensor cores keep the FMA work off the ALUs: the kernel is bound by HBM (G flop per KV byte).
+//
+// Every wait is bounded: after kSpinLimit polls a thread raises the CTA's abort word, reports
+// through the status word and everybody leaves.
 // ------------------------------------------------------------------------------------------------
 constexpr int kMmaD = 128;
 constexpr int kMmaHkv = 8;
@@ -279,10 +288,21 @@ constexpr int kMmaPitch = kMmaRowBytes + 16;              // 2064: breaks the 2 
 constexpr int kMmaSlabBytes = kMmaTileTokens * kMmaPitch; // one K (or V) tile in shared memory
 constexpr int kMmaStageBytes = 2 * kMmaSlabBytes;
 constexpr int kMmaRingBytes = kMmaStages * kMmaStageBytes;
-constexpr int kMmaSmemBytes = kMmaRingBytes + 64;         // + barriers and the abort word
-constexpr int kMmaConsumerWarps = kMmaHkv;
+constexpr int kMmaCtrlBytes = 256;                        // barriers, stage descriptors, abort word
+constexpr int kMmaConsumerWarps = 2 * kMmaHkv;
 constexpr int kMmaThreads = (kMmaConsumerWarps + 1) * 32;
+constexpr int kMmaXRow = kMmaD + 2;                       // exchange row: D outputs, max, sum
 constexpr int kSpinLimit = 1 << 22;
+constexpr int kFlagFirst = 1, kFlagLast = 2, kFlagEnd = 4;
+
+constexpr int mma_smem_bytes(int G) { return kMmaRingBytes + kMmaCtrlBytes + kMmaHkv * G * kMmaXRow * 4; }
+
+struct StageDesc {  // published by the producer next to every ring stage
+    int32_t item;   // index into batch.items
+    int32_t t0;     // first token of the tile
+    int32_t rows;   // valid token rows (0 for the pseudo-tile of an empty context)
+    int32_t flags;  // kFlagFirst | kFlagLast | kFlagEnd
+};
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -304,18 +324,23 @@ __device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-// Bounded wait: gives up after kSpinLimit polls (a fraction of a second), raises the CTA's abort
-// word and reports through the status word instead of spinning for ever.
+// Bounded, warp-uniform wait.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int32_t* abort_word,
                                           int32_t* status) {
+    bool ok = false;
     for (int i = 0; i < kSpinLimit; ++i) {
-        if (mbar_test(bar, parity)) return true;
-        if (*abort_word) return false;
+        if (mbar_test(bar, parity)) {
+            ok = true;
+            break;
+        }
+        if (*abort_word) break;
         if (i > 32) __nanosleep(40);
     }
-    *abort_word = 1;
-    *(volatile int32_t*)status = 3;
-    return false;
+    if (!ok && !*abort_word) {
+        *abort_word = 1;
+        *(volatile int32_t*)status = 3;
+    }
+    return __all_sync(0xffffffffu, ok);
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -332,12 +357,22 @@ __device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t& r0, uint32_t&
                  : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
                  : "r"(addr));
 }
-__device__ __forceinline__ void mma_bf16(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                         uint32_t b1) {
+// D = A(16x16) B(16x8) + C; only rows 0-7 of A are populated (a1 = a3 = 0), rows 8-15 of D are dropped.
+__device__ __forceinline__ void mma_k16(float& d0, float& d1, uint32_t a0, uint32_t a2, uint32_t b0, uint32_t b1,
+                                        float c0, float c1) {
+    float x2, x3;
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%10,%11,%12,%13};"
+        : "=f"(d0), "=f"(d1), "=f"(x2), "=f"(x3)
+        : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(c0), "f"(c1), "f"(0.f), "f"(0.f));
+}
+// D = A(16x8) B(8x8) + C, same row convention.
+__device__ __forceinline__ void mma_k8(float& d0, float& d1, uint32_t a0, uint32_t b0, float c0, float c1) {
+    float x2, x3;
+    asm volatile(
+        "mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%8,%9,%10};"
+        : "=f"(d0), "=f"(d1), "=f"(x2), "=f"(x3)
+        : "r"(a0), "r"(0u), "r"(b0), "f"(c0), "f"(c1), "f"(0.f), "f"(0.f));
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
@@ -348,22 +383,32 @@ template <int G>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloat16* __restrict__ vpool,
                        const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
-                       AttnBatch batch, const int32_t* __restrict__ cta_begin, int32_t block_size, int32_t block_shift,
-                       int32_t num_blocks, float* __restrict__ partials, float scale_log2e, int32_t* status) {
+                       AttnBatch batch, int32_t sched_lane, int32_t block_size, int32_t block_shift,
+                       int32_t num_blocks, float* __restrict__ partials, int32_t* __restrict__ sched,
+                       float scale_log2e, int32_t* status) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int Hq = kMmaHkv * G;
     const uint32_t ring = smem_u32(smem);
-    const uint32_t bar_full = ring + kMmaRingBytes;        // kMmaStages x 8 bytes
-    const uint32_t bar_empty = bar_full + 8 * kMmaStages;  // kMmaStages x 8 bytes
-    volatile int32_t* abort_word = reinterpret_cast<volatile int32_t*>(smem + kMmaRingBytes + 16 * kMmaStages);
+    unsigned char* ctrl = smem + kMmaRingBytes;
+    const uint32_t bar_full = ring + kMmaRingBytes;         // [kMmaStages]
+    const uint32_t bar_empty = bar_full + 8 * kMmaStages;   // [kMmaStages]
+    const uint32_t bar_xfull = bar_empty + 8 * kMmaStages;  // [kMmaHkv] second half has published its state
+    const uint32_t bar_xfree = bar_xfull + 8 * kMmaHkv;     // [kMmaHkv] first half has read it
+    // 8 * (3 + 3 + 8 + 8) = 176 bytes of barriers, then the stage descriptors and the abort word
+    volatile StageDesc* sdesc = reinterpret_cast<volatile StageDesc*>(ctrl + 176);
+    volatile int32_t* abort_word = reinterpret_cast<volatile int32_t*>(ctrl + 176 + 16 * kMmaStages);
+    float* xbuf = reinterpret_cast<float*>(smem + kMmaRingBytes + kMmaCtrlBytes);  // [Hkv][G][kMmaXRow]
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
-    // one-time set-up: barriers, a finite ring
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMmaStages; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, kMmaConsumerWarps);
+        }
+        for (int h = 0; h < kMmaHkv; ++h) {
+            mbar_init(bar_xfull + 8 * h, 1);
+            mbar_init(bar_xfree + 8 * h, 1);
         }
         *abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -373,107 +418,148 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy zeroes before async-proxy writes
     __syncthreads();
 
+    const int32_t* cta_begin = batch.cta_begin[sched_lane];
     const int item0 = cta_begin[blockIdx.x];
     const int item1 = cta_begin[blockIdx.x + 1];
+    const int dyn_begin = cta_begin[gridDim.x];         // the lane's dynamic chunks follow the static shares
+    const int dyn_end = batch.lane_items[sched_lane + 1];
 
     if (warp == kMmaConsumerWarps) {
-        // ------------------------------------------------ producer warp: lane r issues the copy of K row r,
-        // lane 16 + r that of V row r (one thread issuing all 32 requests of a tile caps the kernel at ~80 %
-        // of what the same pipeline reaches with the requests spread over the warp)
-        {
-            int n = 0;
-            bool ok = true;
-            for (int it = item0; it < item1 && ok; ++it) {
-                const AttnItem item = batch.items[it];
-                const int32_t* table = batch.block_tables + (int64_t)item.b * batch.table_stride;
-                for (int t0 = item.t_begin; t0 < item.t_end && ok; t0 += kMmaTileTokens, ++n) {
-                    const int s = n % kMmaStages;
-                    if (n >= kMmaStages)
-                        ok = mbar_wait(bar_empty + 8 * s, ((n / kMmaStages) - 1) & 1, abort_word, status);
-                    ok = __all_sync(0xffffffffu, ok);
-                    if (!ok) break;
-                    const int rows = min(kMmaTileTokens, item.t_end - t0);
+        // ------------------------------------------------ producer warp
+        int n = 0;
+        bool ok = true;
+        int32_t* counter = sched + 2 * sched_lane;
+        int it = item0;
+        bool dynamic = false;
+        while (ok) {
+            if (!dynamic && it >= item1) dynamic = true;
+            if (dynamic) {
+                int c = 0;
+                if (lane == 0) c = atomicAdd(counter, 1);
+                c = __shfl_sync(0xffffffffu, c, 0);
+                it = dyn_begin + c;
+                if (it >= dyn_end) break;
+            }
+            const AttnItem item = batch.items[it];
+            const int32_t* table = batch.block_tables + (int64_t)item.b * batch.table_stride;
+            const int ntiles = max(1, (item.t_end - item.t_begin + kMmaTileTokens - 1) / kMmaTileTokens);
+            for (int ti = 0; ti < ntiles; ++ti, ++n) {
+                const int s = n % kMmaStages;
+                if (n >= kMmaStages) ok = mbar_wait(bar_empty + 8 * s, ((n / kMmaStages) - 1) & 1, abort_word, status);
+                if (!ok) break;
+                const int t0 = item.t_begin + ti * kMmaTileTokens;
+                const int rows = max(0, min(kMmaTileTokens, item.t_end - t0));
+                const uint32_t full = bar_full + 8 * s;
+                int id = 0, slot = 0;
+                bool copy = rows > 0;
+                if (copy) {
                     const int blk = block_shift >= 0 ? (t0 >> block_shift) : (t0 / block_size);
-                    const int slot = t0 - blk * block_size;
-                    const int id = table[blk];
-                    const uint32_t full = bar_full + 8 * s;
-                    if ((unsigned)id >= (unsigned)num_blocks) {
-                        // skip the copy: consumers see the previous (finite) contents; the host sees the error
+                    slot = t0 - blk * block_size;
+                    id = table[blk];
+                    if ((unsigned)id >= (unsigned)num_blocks) {  // the stage keeps its old, finite contents
                         *(volatile int32_t*)status = 2;
-                        if (lane == 0) mbar_arrive(full);
-                        continue;
+                        copy = false;
                     }
-                    if (lane == 0) mbar_expect_tx(full, (uint32_t)rows * 2u * kMmaRowBytes);
-                    __syncwarp();  // the expected byte count is posted before any copy can complete
-                    const int64_t off = ((int64_t)id * block_size + slot) * (kMmaRowBytes / 2);  // elements
-                    const uint32_t ks = ring + s * kMmaStageBytes;
-                    const uint32_t vs = ks + kMmaSlabBytes;
+                }
+                if (lane == 0) {
+                    sdesc[s].item = it;
+                    sdesc[s].t0 = t0;
+                    sdesc[s].rows = rows;
+                    sdesc[s].flags = (ti == 0 ? kFlagFirst : 0) | (ti == ntiles - 1 ? kFlagLast : 0);
+                    if (copy)
+                        mbar_expect_tx(full, (uint32_t)rows * 2u * kMmaRowBytes);
+                    else
+                        mbar_arrive(full);
+                }
+                __syncwarp();  // descriptor and expected byte count are posted before any copy can complete
+                if (copy) {
                     const int r = lane & 15;
                     if (r < rows) {
-                        const __nv_bfloat16* src = (lane < 16 ? kpool : vpool) + off + (int64_t)r * (kMmaRowBytes / 2);
-                        bulk_g2s((lane < 16 ? ks : vs) + r * kMmaPitch, src, kMmaRowBytes, full);
+                        const int64_t off = ((int64_t)id * block_size + slot + r) * (kMmaRowBytes / 2);  // elements
+                        const uint32_t dst = ring + s * kMmaStageBytes + (lane < 16 ? 0 : kMmaSlabBytes) + r * kMmaPitch;
+                        bulk_g2s(dst, (lane < 16 ? kpool : vpool) + off, kMmaRowBytes, full);
                     }
                 }
             }
+            if (!dynamic) ++it;
+        }
+        if (ok) {  // end-of-stream marker
+            const int s = n % kMmaStages;
+            if (n >= kMmaStages) ok = mbar_wait(bar_empty + 8 * s, ((n / kMmaStages) - 1) & 1, abort_word, status);
+            if (ok && lane == 0) {
+                sdesc[s].flags = kFlagEnd;
+                mbar_arrive(bar_full + 8 * s);
+            }
+        }
+        // the last CTA to finish fetching re-arms the chunk counter for the lane's next launch
+        if (lane == 0) {
+            __threadfence();
+            if (atomicAdd(counter + 1, 1) == (int)gridDim.x - 1) {
+                atomicExch(counter, 0);
+                atomicExch(counter + 1, 0);
+            }
         }
     } else {
-        // ------------------------------------------------ consumers: warp = KV head
-        const int g = lane >> 2;  // row of the mma tile = query head inside the group (valid if g < G)
+        // ------------------------------------------------ consumers: warp = (KV head, 8-token half)
+        const int h = warp & (kMmaHkv - 1);
+        const int half = warp >> 3;
+        const int g = lane >> 2;  // mma row = query head inside the group (real if g < G)
         const int t = lane & 3;
-        const int h = warp;
-        // ldmatrix row addresses (byte offsets inside a slab), see the layout comments above
         const int ld_row = lane & 7;
         const int ld_mat = lane >> 3;
-        // K (no transpose): matrices {tok 0-7, d lo}, {tok 0-7, d hi}, {tok 8-15, d lo}, {tok 8-15, d hi}
-        const uint32_t k_lane_off = (uint32_t)((ld_row + ((ld_mat & 2) ? 8 : 0)) * kMmaPitch + h * 256 + ((ld_mat & 1) ? 16 : 0));
-        // V (transpose): matrices {tok 0-7, d lo}, {tok 8-15, d lo}, {tok 0-7, d hi}, {tok 8-15, d hi}
-        const uint32_t v_lane_off = (uint32_t)((ld_row + ((ld_mat & 1) ? 8 : 0)) * kMmaPitch + h * 256 + ((ld_mat & 2) ? 16 : 0));
-        int n = 0;
+        // K, no transpose: token half*8 + ld_row; the four matrices are four consecutive 8-dim chunks
+        const uint32_t k_lane_off = (uint32_t)((half * 8 + ld_row) * kMmaPitch + h * 256 + ld_mat * 16);
+        // V, transposed on load: same rows and chunks, in the second slab of the stage
+        const uint32_t v_lane_off = k_lane_off + kMmaSlabBytes;
+        float* xrow = xbuf + ((h * G) + (g < G ? g : 0)) * kMmaXRow;
+
+        uint32_t qa[8][2];
+        float o[16][2];
+        float m_run = kNegBig, l_run = 0.f;
+        AttnItem item{};
+        int n = 0, n_item = 0;
         bool ok = true;
-        for (int it = item0; it < item1 && ok; ++it) {
-            const AttnItem item = batch.items[it];
-            // Q fragments of this head group: rows g < G are real, everything else is zero
-            uint32_t qa[8][2];
-            {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) qa[j][0] = qa[j][1] = 0u;
+#pragma unroll
+        for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = 0.f;
+
+        for (;; ++n) {
+            const int s = n % kMmaStages;
+            ok = mbar_wait(bar_full + 8 * s, (n / kMmaStages) & 1, abort_word, status);
+            if (!ok) break;
+            const int flags = sdesc[s].flags;
+            if (flags & kFlagEnd) break;
+            const int rows = sdesc[s].rows - 8 * half;  // valid tokens of this warp's half (may be <= 0)
+            if (flags & kFlagFirst) {
+                item = batch.items[sdesc[s].item];
                 const __nv_bfloat16* qrow = q + ((int64_t)item.b * Hq + h * G + g) * kMmaD;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     qa[j][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 2 * t) : 0u;
                     qa[j][1] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 8 + 2 * t) : 0u;
                 }
+#pragma unroll
+                for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = 0.f;
+                m_run = kNegBig;
+                l_run = 0.f;
             }
-            float o[16][4];
+            if (rows > 0) {
+                const uint32_t base = ring + s * kMmaStageBytes;
+                // scores of row g against tokens 2t, 2t+1 of this half; two accumulators shorten the chain
+                float sa0 = 0.f, sa1 = 0.f, sb0 = 0.f, sb1 = 0.f;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = o[i][2] = o[i][3] = 0.f;
-            float m_run = kNegBig, l_run = 0.f;
-
-            for (int t0 = item.t_begin; t0 < item.t_end; t0 += kMmaTileTokens, ++n) {
-                const int s = n % kMmaStages;
-                ok = mbar_wait(bar_full + 8 * s, (n / kMmaStages) & 1, abort_word, status);
-                ok = __all_sync(0xffffffffu, ok);  // the warp leaves together (full-mask shuffles below)
-                if (!ok) break;
-                const int rows = min(kMmaTileTokens, item.t_end - t0);
-                const uint32_t ks = ring + s * kMmaStageBytes;
-                const uint32_t vs = ks + kMmaSlabBytes;
-
-                // scores for 16 tokens: two n-tiles of 8 tokens
-                float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int j = 0; j < 8; ++j) {
-                    uint32_t b0, b1, b2, b3;
-                    ldsm_x4(ks + k_lane_off + 32 * j, b0, b1, b2, b3);
-                    mma_bf16(s0, qa[j][0], 0u, qa[j][1], 0u, b0, b1);
-                    mma_bf16(s1, qa[j][0], 0u, qa[j][1], 0u, b2, b3);
+                for (int jj = 0; jj < 4; ++jj) {
+                    uint32_t b0, b1, b2, b3;  // dims 32jj..+7, +8..15, +16..23, +24..31
+                    ldsm_x4(base + k_lane_off + 64 * jj, b0, b1, b2, b3);
+                    mma_k16(sa0, sa1, qa[2 * jj][0], qa[2 * jj][1], b0, b1, sa0, sa1);
+                    mma_k16(sb0, sb1, qa[2 * jj + 1][0], qa[2 * jj + 1][1], b2, b3, sb0, sb1);
                 }
-                // this lane's four tokens of row g: 2t, 2t+1, 8+2t, 9+2t
-                float x0 = s0[0] * scale_log2e, x1 = s0[1] * scale_log2e;
-                float x2 = s1[0] * scale_log2e, x3 = s1[1] * scale_log2e;
-                const bool v0 = 2 * t < rows, v1 = 2 * t + 1 < rows, v2 = 8 + 2 * t < rows, v3 = 9 + 2 * t < rows;
+                const float x0 = (sa0 + sb0) * scale_log2e, x1 = (sa1 + sb1) * scale_log2e;
+                const bool v0 = 2 * t < rows, v1 = 2 * t + 1 < rows;
                 float mx = kNegBig;
-                if (v0) mx = fmaxf(mx, x0);
+                if (v0) mx = x0;
                 if (v1) mx = fmaxf(mx, x1);
-                if (v2) mx = fmaxf(mx, x2);
-                if (v3) mx = fmaxf(mx, x3);
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
                 const float m_new = fmaxf(m_run, mx);
@@ -481,52 +567,78 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                 m_run = m_new;
                 const float p0 = v0 ? exp2f(x0 - m_new) : 0.f;
                 const float p1 = v1 ? exp2f(x1 - m_new) : 0.f;
-                const float p2 = v2 ? exp2f(x2 - m_new) : 0.f;
-                const float p3 = v3 ? exp2f(x3 - m_new) : 0.f;
-                l_run = l_run * alpha + (p0 + p1 + p2 + p3);
+                l_run = l_run * alpha + (p0 + p1);
+                const uint32_t pa = pack_bf16(p0, p1);  // A operand: row g, tokens 2t, 2t+1
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    o[i][0] *= alpha;
-                    o[i][1] *= alpha;
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t b0, b1, b2, b3;  // output dims 32c..+7, +8.., +16.., +24..
+                    ldsm_x4_t(base + v_lane_off + 64 * c, b0, b1, b2, b3);
+                    mma_k8(o[4 * c][0], o[4 * c][1], pa, b0, o[4 * c][0] * alpha, o[4 * c][1] * alpha);
+                    mma_k8(o[4 * c + 1][0], o[4 * c + 1][1], pa, b1, o[4 * c + 1][0] * alpha, o[4 * c + 1][1] * alpha);
+                    mma_k8(o[4 * c + 2][0], o[4 * c + 2][1], pa, b2, o[4 * c + 2][0] * alpha, o[4 * c + 2][1] * alpha);
+                    mma_k8(o[4 * c + 3][0], o[4 * c + 3][1], pa, b3, o[4 * c + 3][0] * alpha, o[4 * c + 3][1] * alpha);
                 }
-                const uint32_t pa0 = pack_bf16(p0, p1);  // row g, tokens 2t, 2t+1
-                const uint32_t pa2 = pack_bf16(p2, p3);  // row g, tokens 8+2t, 9+2t
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    uint32_t b0, b1, b2, b3;
-                    ldsm_x4_t(vs + v_lane_off + 32 * c, b0, b1, b2, b3);
-                    mma_bf16(o[2 * c], pa0, 0u, pa2, 0u, b0, b1);
-                    mma_bf16(o[2 * c + 1], pa0, 0u, pa2, 0u, b2, b3);
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(bar_empty + 8 * s);
             }
-            if (!ok) break;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_empty + 8 * s);
 
-            // finalise the item for row g
-            float L = l_run;
-            L += __shfl_xor_sync(0xffffffffu, L, 1);
-            L += __shfl_xor_sync(0xffffffffu, L, 2);
-            if (g < G) {
-                const int hq = h * G + g;
-                if (item.n_parts == 1) {
-                    const float inv = L > 0.f ? 1.f / L : 0.f;
-                    __nv_bfloat16* orow = out + ((int64_t)item.b * Hq + hq) * kMmaD;
+            if (flags & kFlagLast) {
+                // ---- combine the two halves of the item through shared memory, first half writes out
+                float L = l_run;
+                L += __shfl_xor_sync(0xffffffffu, L, 1);
+                L += __shfl_xor_sync(0xffffffffu, L, 2);
+                if (half == 1) {
+                    if (n_item > 0) ok = mbar_wait(bar_xfree + 8 * h, (n_item - 1) & 1, abort_word, status);
+                    if (!ok) break;
+                    if (g < G) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        *reinterpret_cast<uint32_t*>(orow + 8 * i + 2 * t) = pack_bf16(o[i][0] * inv, o[i][1] * inv);
-                    if (lse != nullptr && t == 0)
-                        lse[(int64_t)item.b * Hq + hq] = L > 0.f ? (m_run + log2f(L)) * kLn2 : -CUDART_INF_F;
-                } else {
-                    float* pr = partials + ((int64_t)item.part * Hq + hq) * (kMmaD + 2);
-#pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        *reinterpret_cast<float2*>(pr + 8 * i + 2 * t) = make_float2(o[i][0], o[i][1]);
-                    if (t == 0) {
-                        pr[kMmaD] = m_run;
-                        pr[kMmaD + 1] = L;
+                        for (int i = 0; i < 16; ++i)
+                            *reinterpret_cast<float2*>(xrow + 8 * i + 2 * t) = make_float2(o[i][0], o[i][1]);
+                        if (t == 0) {
+                            xrow[kMmaD] = m_run;
+                            xrow[kMmaD + 1] = L;
+                        }
                     }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_xfull + 8 * h);
+                } else {
+                    ok = mbar_wait(bar_xfull + 8 * h, n_item & 1, abort_word, status);
+                    if (!ok) break;
+                    if (g < G) {
+                        const float m1 = xrow[kMmaD], L1 = xrow[kMmaD + 1];
+                        const float M = fmaxf(m_run, m1);
+                        const float w0 = exp2f(m_run - M), w1 = exp2f(m1 - M);
+                        const float Lt = L * w0 + L1 * w1;
+                        const int hq = h * G + g;
+                        if (item.n_parts == 1) {
+                            const float inv = Lt > 0.f ? 1.f / Lt : 0.f;
+                            __nv_bfloat16* orow = out + ((int64_t)item.b * Hq + hq) * kMmaD;
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const float2 o1 = *reinterpret_cast<const float2*>(xrow + 8 * i + 2 * t);
+                                *reinterpret_cast<uint32_t*>(orow + 8 * i + 2 * t) =
+                                    pack_bf16((o[i][0] * w0 + o1.x * w1) * inv, (o[i][1] * w0 + o1.y * w1) * inv);
+                            }
+                            if (lse != nullptr && t == 0)
+                                lse[(int64_t)item.b * Hq + hq] = Lt > 0.f ? (M + log2f(Lt)) * kLn2 : -CUDART_INF_F;
+                        } else {
+                            float* pr = partials + ((int64_t)item.part * Hq + hq) * (kMmaD + 2);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i) {
+                                const float2 o1 = *reinterpret_cast<const float2*>(xrow + 8 * i + 2 * t);
+                                *reinterpret_cast<float2*>(pr + 8 * i + 2 * t) =
+                                    make_float2(o[i][0] * w0 + o1.x * w1, o[i][1] * w0 + o1.y * w1);
+                            }
+                            if (t == 0) {
+                                pr[kMmaD] = M;
+                                pr[kMmaD + 1] = Lt;
+                            }
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_xfree + 8 * h);
                 }
+                ++n_item;
             }
         }
     }
@@ -534,11 +646,12 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
 
 template <int G>
 cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool, const void* q, void* out, float* lse,
-                       const AttnBatch& batch, int32_t lane, float* partials, int32_t* d_status, cudaStream_t stream) {
+                       const AttnBatch& batch, int32_t lane, float* partials, int32_t* sched, int32_t* d_status,
+                       cudaStream_t stream) {
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)kMmaD);
-    decode_attn_mma_kernel<G><<<(unsigned)batch.n_cta[lane], kMmaThreads, kMmaSmemBytes, stream>>>(
+    decode_attn_mma_kernel<G><<<(unsigned)batch.n_cta[lane], kMmaThreads, mma_smem_bytes(G), stream>>>(
         (const __nv_bfloat16*)kpool, (const __nv_bfloat16*)vpool, (const __nv_bfloat16*)q, (__nv_bfloat16*)out, lse, batch,
-        batch.cta_begin[lane], sh.block_size, shift_of(sh.block_size), sh.num_blocks, partials, scale_log2e, d_status);
+        lane, sh.block_size, shift_of(sh.block_size), sh.num_blocks, partials, sched, scale_log2e, d_status);
     return cudaGetLastError();
 }
 
@@ -558,7 +671,7 @@ cudaError_t attn_init() {
     cudaError_t e;
 #define PS_MMA_ATTR(GG)                                                                                    \
     e = cudaFuncSetAttribute(decode_attn_mma_kernel<GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                             kMmaSmemBytes);                                                               \
+                             mma_smem_bytes(GG));                                                          \
     if (e != cudaSuccess) return e;
     PS_MMA_ATTR(1) PS_MMA_ATTR(2) PS_MMA_ATTR(4) PS_MMA_ATTR(8)
 #undef PS_MMA_ATTR
@@ -567,7 +680,7 @@ cudaError_t attn_init() {
 
 cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool, const void* q,
                                void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials,
-                               int32_t* d_status, cudaStream_t stream) {
+                               int32_t* sched, int32_t* d_status, cudaStream_t stream) {
     if (lane < 0 || lane > 1) return cudaErrorInvalidValue;
     const int item_begin = batch.lane_items[lane];
     const int n_items = batch.lane_items[lane + 1] - item_begin;
@@ -576,10 +689,10 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
     if (kernel == 2) {
         if (!attn_mma_supported(sh) || batch.n_cta[lane] <= 0) return cudaErrorNotSupported;
         switch (G) {
-            case 1: return launch_mma<1>(sh, kpool, vpool, q, out, lse, batch, lane, partials, d_status, stream);
-            case 2: return launch_mma<2>(sh, kpool, vpool, q, out, lse, batch, lane, partials, d_status, stream);
-            case 4: return launch_mma<4>(sh, kpool, vpool, q, out, lse, batch, lane, partials, d_status, stream);
-            case 8: return launch_mma<8>(sh, kpool, vpool, q, out, lse, batch, lane, partials, d_status, stream);
+            case 1: return launch_mma<1>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, d_status, stream);
+            case 2: return launch_mma<2>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, d_status, stream);
+            case 4: return launch_mma<4>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, d_status, stream);
+            case 8: return launch_mma<8>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, d_status, stream);
         }
         return cudaErrorNotSupported;
     }

@@ -61,7 +61,8 @@ struct AttnBatch {                 // device pointers to the per-batch metadata
     const int32_t* row_first_part; // [B] first partial slot of the row
     const int32_t* row_parts;      // [B] number of partial slots of the row
     const int32_t* row_lane;       // [B] 0 = main lane, 1 = reload lane (attention waits on reload events)
-    const int32_t* cta_begin[2];   // tensor-core kernel: per lane, [n_cta + 1] first item of every CTA
+    const int32_t* cta_begin[2];   // tensor-core kernel: per lane, [n_cta + 1]: first static item of every
+                                   // CTA; entry n_cta is where the lane's dynamic chunks start
     int32_t n_cta[2];
     int32_t lane_items[3];         // items of lane 0 are [lane_items[0], lane_items[1]), lane 1 [.. [1], [2])
     int32_t table_stride;
@@ -73,10 +74,12 @@ struct AttnBatch {                 // device pointers to the per-batch metadata
 size_t attn_partial_bytes(const AttnShape& sh, int32_t max_parts);
 
 // Launches the attention kernel for the items of one lane.  kernel: 1 = SIMT (one CTA per item and
-// KV head), 2 = MMA (CTA c of the lane walks items [cta_begin[c], cta_begin[c+1])).
+// KV head), 2 = MMA (CTA c of the lane walks items [cta_begin[c], cta_begin[c+1]), then takes dynamic
+// chunks through the counters in sched: 2 int32 per lane, zero before the first launch, re-armed by
+// the kernel itself).
 cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool, const void* q,
                                void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials,
-                               int32_t* d_status, cudaStream_t stream);
+                               int32_t* sched, int32_t* d_status, cudaStream_t stream);
 
 // Token granularity at which the tensor-core kernel splits a context.
 constexpr int kMmaTileTokens = 16;

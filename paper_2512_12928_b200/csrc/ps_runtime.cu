@@ -169,6 +169,7 @@ struct ps_ctx {
     std::deque<std::pair<uint64_t, std::pair<int64_t, int64_t>>> img_release;  // in_ticket -> (off, bytes)
     std::vector<int64_t> gated_reqs;
     float* partials = nullptr;
+    int32_t* d_sched = nullptr;  // chunk counters of the tensor-core kernel: {next, done} per lane
     int32_t max_parts = 0;
     int attn_kernel = 1;
     int32_t num_sms = 1;
@@ -586,10 +587,13 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
                 if (pass == 1) ++n_gated_rows;
             }
         } else {
-            // Tensor-core kernel: the lane's 16-token tiles form one sequence, cut into equal shares,
-            // one per CTA; an item is the part of a row that falls into one CTA's share.
+            // Tensor-core kernel: the lane's 16-token tiles form one sequence.  Its head is cut into
+            // equal static shares, one per CTA; its tail (kDynFrac of the tiles, when there are enough)
+            // into small chunks that the CTAs take dynamically.  An item is the part of a row that
+            // falls into one share or chunk.
             constexpr int kTile = ps::kMmaTileTokens;
             constexpr int64_t kMinTilesPerCta = 8;
+            constexpr int64_t kDynChunksPerCta = 6;
             int64_t total_tiles = 0;
             int32_t lane_rows = 0;
             for (int32_t b = 0; b < B; ++b)
@@ -601,9 +605,22 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
             if (lane_rows > 0)
                 n_cta = std::min<int64_t>(std::max<int64_t>((total_tiles + kMinTilesPerCta - 1) / kMinTilesPerCta, 1),
                                           ctx->num_sms);
-            const int64_t per = n_cta > 0 ? std::max<int64_t>((total_tiles + n_cta - 1) / n_cta, 1) : 1;
-            int64_t filled = 0;
+            int64_t dyn_tiles = 0, chunk = 0;
+            if (n_cta > 0 && total_tiles >= 32 * n_cta) {
+                dyn_tiles = total_tiles * 15 / 100;
+                chunk = std::max<int64_t>(kMinTilesPerCta, (dyn_tiles + kDynChunksPerCta * n_cta - 1) / (kDynChunksPerCta * n_cta));
+            }
+            const int64_t static_tiles = total_tiles - dyn_tiles;
+            const int64_t per = n_cta > 0 ? std::max<int64_t>((static_tiles + n_cta - 1) / n_cta, 1) : 1;
+            // walk the rows; `pos` is the position in the lane's tile sequence
+            int64_t pos = 0, filled = 0;       // filled: tiles in the current share or chunk
+            bool in_dyn = false;
             if (n_cta > 0) cta_begin[pass].push_back((int32_t)items.size());
+            auto close_static = [&]() {        // pad the share list and mark where the dynamic chunks start
+                while ((int64_t)cta_begin[pass].size() < n_cta + 1) cta_begin[pass].push_back((int32_t)items.size());
+                in_dyn = true;
+                filled = 0;
+            };
             for (int32_t b = 0; b < B; ++b) {
                 if (!active[b] || (gated[b] ? 1 : 0) != pass) continue;
                 const Req& r = ctx->reqs[reqs[b]];
@@ -614,33 +631,45 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
                 if (tiles_b == 0) {  // empty context: one item without tiles writes the zero row
                     ps::AttnItem it{};
                     it.b = b;
-                    it.part = parts;
                     items.push_back(it);
                 }
                 for (int64_t lo = 0; lo < tiles_b;) {
-                    if (filled == per && (int64_t)cta_begin[pass].size() < n_cta) {
-                        cta_begin[pass].push_back((int32_t)items.size());
-                        filled = 0;
+                    if (!in_dyn && pos >= static_tiles) close_static();
+                    int64_t room;
+                    if (!in_dyn) {
+                        if (filled == per && (int64_t)cta_begin[pass].size() < n_cta) {
+                            cta_begin[pass].push_back((int32_t)items.size());
+                            filled = 0;
+                        }
+                        room = std::min(per - filled, static_tiles - pos);
+                    } else {
+                        if (filled == chunk) filled = 0;
+                        room = chunk - filled;
                     }
-                    const int64_t take = std::min(tiles_b - lo, per - filled);
+                    const int64_t take = std::min(tiles_b - lo, std::max<int64_t>(room, 1));
                     ps::AttnItem it{};
                     it.b = b;
                     it.t_begin = (int32_t)(lo * kTile);
                     it.t_end = (int32_t)std::min<int64_t>(r.n_tokens, (lo + take) * kTile);
-                    it.part = parts + (int32_t)(items.size() - first_item);
                     items.push_back(it);
                     lo += take;
-                    filled += take;
+                    pos += take;
+                    // a dynamic chunk never spans two rows: every item of the tail is its own chunk
+                    filled = in_dyn ? chunk : filled + take;
+                    if (in_dyn && take < chunk && lo < tiles_b) filled = chunk;
                 }
                 const int32_t n = (int32_t)(items.size() - first_item);
-                for (size_t k = first_item; k < items.size(); ++k) items[k].n_parts = n;
+                for (size_t k = first_item; k < items.size(); ++k) {
+                    items[k].part = parts + (int32_t)(k - first_item);
+                    items[k].n_parts = n;
+                }
                 row_parts[b] = n;
                 parts += n;
                 any_multi |= n > 1;
                 lane_multi[pass] |= n > 1;
                 if (pass == 1) ++n_gated_rows;
             }
-            while (n_cta > 0 && (int64_t)cta_begin[pass].size() < n_cta + 1) cta_begin[pass].push_back((int32_t)items.size());
+            if (n_cta > 0 && !in_dyn) close_static();
         }
         if (pass == 0) n_ungated = (int32_t)items.size();
     }
@@ -735,7 +764,7 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
     if (m.n_ungated_items > 0) {
         ProfScope prof(ctx, kProfAttn, ctx->compute, ungated_bytes, layer);
         CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev, 0,
-                                  ctx->partials, ctx->d_status, ctx->compute));
+                                  ctx->partials, ctx->d_sched, ctx->d_status, ctx->compute));
         ctx->launches++;
         ++*n_launched;
     }
@@ -751,7 +780,7 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
         {
             ProfScope prof(ctx, kProfAttn, gs, bytes - ungated_bytes, 1000 + layer);
             CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev,
-                                      1, ctx->partials, ctx->d_status, gs));
+                                      1, ctx->partials, ctx->d_sched, ctx->d_status, gs));
             ctx->launches++;
             ++*n_launched;
         }
@@ -796,6 +825,7 @@ void destroy_ctx(ps_ctx* ctx) {
         if (ctx->d_kpools) cudaFree(ctx->d_kpools);
         if (ctx->d_vpools) cudaFree(ctx->d_vpools);
         if (ctx->partials) cudaFree(ctx->partials);
+        if (ctx->d_sched) cudaFree(ctx->d_sched);
         if (ctx->d_ids) cudaFree(ctx->d_ids);
         if (ctx->h_ids) cudaFreeHost(ctx->h_ids);
         if (ctx->status) cudaFreeHost(ctx->status);
@@ -982,9 +1012,12 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
             ctx->num_sms = std::max(sms, 1);
         }
         // the tensor-core kernel cuts a lane into at most num_sms shares: rows + shares parts per lane
-        max_parts = std::max<int64_t>(max_parts, max_batch + 2 * (int64_t)ctx->num_sms + 8);
+        // (static shares + at most ~6 dynamic chunks per CTA, plus one chunk boundary per row)
+        max_parts = std::max<int64_t>(max_parts, 3 * max_batch + 2 * 8 * (int64_t)ctx->num_sms + 16);
         ctx->max_parts = (int32_t)std::min<int64_t>(max_parts, 1 << 22);
         CKC(cudaMalloc((void**)&ctx->partials, ps::attn_partial_bytes(sh, ctx->max_parts)));
+        CKC(cudaMalloc((void**)&ctx->d_sched, 4 * sizeof(int32_t)));
+        CKC(cudaMemset(ctx->d_sched, 0, 4 * sizeof(int32_t)));
         const size_t meta_chunk = (size_t)max_batch * cfg->max_blocks_per_req * 4 + (size_t)max_batch * 16 +
                                   (size_t)ctx->max_parts * sizeof(ps::AttnItem) + (size_t)ctx->num_sms * 8 + 8192;
         CKR(arena_init(ctx, ctx->a_meta, meta_chunk, 3, ctx->compute));
