@@ -269,12 +269,11 @@ cudaError_t launch_simt(const AttnShape& sh, const void* kpool, const void* vpoo
 // head touches 8 different bank groups.  Rows past the end of a context are never copied (the ring
 // is zeroed once, so a stale row is always finite).
 //
-// Math: KV head h is served by two warps, one per 8-token half of the tile (16 consumer warps keep
-// enough independent instruction streams in flight to cover the mma / ldmatrix latencies).
-// Scores: mma.m16n8k16 with the G query heads of the group as the M rows (padded to 16) and the 8
-// tokens as N; softmax statistics per query head are reduced over the 4 lanes of a quad with
-// shuffles; P is re-packed in registers as the A operand of P.V (mma.m16n8k8) with V read through
-// ldmatrix.trans.  At the end of an item the two halves are combined through shared memory.
+// Math: warp w owns KV head w.  Scores: mma.m16n8k16 with the G query heads of the group as the M
+// rows (padded to 16; the padding rows of every product are dropped) and 8 tokens as N; softmax
+// statistics per query head are reduced over the 4 lanes of a quad with shuffles; P is re-packed in
+// registers as the A operand of P.V with V read through ldmatrix.trans.  (Two warps per head were
+// tried: at 17 warps the register budget drops to 96 per thread and the inner loop spills.)
 // Tensor cores keep the FMA work off the ALUs: the kernel is bound by HBM (G flop per KV byte).
 //
 // Every wait is bounded: after kSpinLimit polls a thread raises the CTA's abort word, reports
@@ -289,13 +288,12 @@ constexpr int kMmaSlabBytes = kMmaTileTokens * kMmaPitch; // one K (or V) tile i
 constexpr int kMmaStageBytes = 2 * kMmaSlabBytes;
 constexpr int kMmaRingBytes = kMmaStages * kMmaStageBytes;
 constexpr int kMmaCtrlBytes = 256;                        // barriers, stage descriptors, abort word
-constexpr int kMmaConsumerWarps = 2 * kMmaHkv;
+constexpr int kMmaConsumerWarps = kMmaHkv;
 constexpr int kMmaThreads = (kMmaConsumerWarps + 1) * 32;
-constexpr int kMmaXRow = kMmaD + 2;                       // exchange row: D outputs, max, sum
 constexpr int kSpinLimit = 1 << 22;
 constexpr int kFlagFirst = 1, kFlagLast = 2, kFlagEnd = 4;
 
-constexpr int mma_smem_bytes(int G) { return kMmaRingBytes + kMmaCtrlBytes + kMmaHkv * G * kMmaXRow * 4; }
+constexpr int mma_smem_bytes(int) { return kMmaRingBytes + kMmaCtrlBytes; }
 
 struct StageDesc {  // published by the producer next to every ring stage
     int32_t item;   // index into batch.items
@@ -366,14 +364,6 @@ __device__ __forceinline__ void mma_k16(float& d0, float& d1, uint32_t a0, uint3
         : "=f"(d0), "=f"(d1), "=f"(x2), "=f"(x3)
         : "r"(a0), "r"(0u), "r"(a2), "r"(0u), "r"(b0), "r"(b1), "f"(c0), "f"(c1), "f"(0.f), "f"(0.f));
 }
-// D = A(16x8) B(8x8) + C, same row convention.
-__device__ __forceinline__ void mma_k8(float& d0, float& d1, uint32_t a0, uint32_t b0, float c0, float c1) {
-    float x2, x3;
-    asm volatile(
-        "mma.sync.aligned.m16n8k8.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5}, {%6}, {%7,%8,%9,%10};"
-        : "=f"(d0), "=f"(d1), "=f"(x2), "=f"(x3)
-        : "r"(a0), "r"(0u), "r"(b0), "f"(c0), "f"(c1), "f"(0.f), "f"(0.f));
-}
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -392,12 +382,9 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
     unsigned char* ctrl = smem + kMmaRingBytes;
     const uint32_t bar_full = ring + kMmaRingBytes;         // [kMmaStages]
     const uint32_t bar_empty = bar_full + 8 * kMmaStages;   // [kMmaStages]
-    const uint32_t bar_xfull = bar_empty + 8 * kMmaStages;  // [kMmaHkv] second half has published its state
-    const uint32_t bar_xfree = bar_xfull + 8 * kMmaHkv;     // [kMmaHkv] first half has read it
-    // 8 * (3 + 3 + 8 + 8) = 176 bytes of barriers, then the stage descriptors and the abort word
-    volatile StageDesc* sdesc = reinterpret_cast<volatile StageDesc*>(ctrl + 176);
-    volatile int32_t* abort_word = reinterpret_cast<volatile int32_t*>(ctrl + 176 + 16 * kMmaStages);
-    float* xbuf = reinterpret_cast<float*>(smem + kMmaRingBytes + kMmaCtrlBytes);  // [Hkv][G][kMmaXRow]
+    // 48 bytes of barriers, then the stage descriptors and the abort word
+    volatile StageDesc* sdesc = reinterpret_cast<volatile StageDesc*>(ctrl + 64);
+    volatile int32_t* abort_word = reinterpret_cast<volatile int32_t*>(ctrl + 64 + 16 * kMmaStages);
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
@@ -405,10 +392,6 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
         for (int s = 0; s < kMmaStages; ++s) {
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, kMmaConsumerWarps);
-        }
-        for (int h = 0; h < kMmaHkv; ++h) {
-            mbar_init(bar_xfull + 8 * h, 1);
-            mbar_init(bar_xfree + 8 * h, 1);
         }
         *abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -500,40 +483,41 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             }
         }
     } else {
-        // ------------------------------------------------ consumers: warp = (KV head, 8-token half)
-        const int h = warp & (kMmaHkv - 1);
-        const int half = warp >> 3;
+        // ------------------------------------------------ consumers: warp = KV head
+        const int h = warp;
         const int g = lane >> 2;  // mma row = query head inside the group (real if g < G)
         const int t = lane & 3;
         const int ld_row = lane & 7;
         const int ld_mat = lane >> 3;
-        // K, no transpose: token half*8 + ld_row; the four matrices are four consecutive 8-dim chunks
-        const uint32_t k_lane_off = (uint32_t)((half * 8 + ld_row) * kMmaPitch + h * 256 + ld_mat * 16);
-        // V, transposed on load: same rows and chunks, in the second slab of the stage
-        const uint32_t v_lane_off = k_lane_off + kMmaSlabBytes;
-        float* xrow = xbuf + ((h * G) + (g < G ? g : 0)) * kMmaXRow;
-
+        // K, no transpose: matrices {tok 0-7, d lo}, {tok 0-7, d hi}, {tok 8-15, d lo}, {tok 8-15, d hi}
+        const uint32_t k_lane_off =
+            (uint32_t)((ld_row + ((ld_mat & 2) ? 8 : 0)) * kMmaPitch + h * 256 + ((ld_mat & 1) ? 16 : 0));
+        // V, transposed on load: matrices {tok 0-7, d lo}, {tok 8-15, d lo}, {tok 0-7, d hi}, {tok 8-15, d hi}
+        const uint32_t v_lane_off = (uint32_t)(kMmaSlabBytes + (ld_row + ((ld_mat & 1) ? 8 : 0)) * kMmaPitch + h * 256 +
+                                               ((ld_mat & 2) ? 16 : 0));
         uint32_t qa[8][2];
         float o[16][2];
         float m_run = kNegBig, l_run = 0.f;
-        AttnItem item{};
-        int n = 0, n_item = 0;
+        int item_b = 0, item_part = 0, item_nparts = 1;
         bool ok = true;
 #pragma unroll
         for (int j = 0; j < 8; ++j) qa[j][0] = qa[j][1] = 0u;
 #pragma unroll
         for (int i = 0; i < 16; ++i) o[i][0] = o[i][1] = 0.f;
 
-        for (;; ++n) {
+        for (int n = 0;; ++n) {
             const int s = n % kMmaStages;
             ok = mbar_wait(bar_full + 8 * s, (n / kMmaStages) & 1, abort_word, status);
             if (!ok) break;
             const int flags = sdesc[s].flags;
             if (flags & kFlagEnd) break;
-            const int rows = sdesc[s].rows - 8 * half;  // valid tokens of this warp's half (may be <= 0)
+            const int rows = sdesc[s].rows;
             if (flags & kFlagFirst) {
-                item = batch.items[sdesc[s].item];
-                const __nv_bfloat16* qrow = q + ((int64_t)item.b * Hq + h * G + g) * kMmaD;
+                const AttnItem* ip = batch.items + sdesc[s].item;
+                item_b = ip->b;
+                item_part = ip->part;
+                item_nparts = ip->n_parts;
+                const __nv_bfloat16* qrow = q + ((int64_t)item_b * Hq + h * G + g) * kMmaD;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     qa[j][0] = g < G ? *reinterpret_cast<const uint32_t*>(qrow + 16 * j + 2 * t) : 0u;
@@ -546,20 +530,23 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             }
             if (rows > 0) {
                 const uint32_t base = ring + s * kMmaStageBytes;
-                // scores of row g against tokens 2t, 2t+1 of this half; two accumulators shorten the chain
-                float sa0 = 0.f, sa1 = 0.f, sb0 = 0.f, sb1 = 0.f;
+                // scores of row g: s0 -> tokens 2t, 2t+1; s1 -> tokens 8+2t, 9+2t
+                float s00 = 0.f, s01 = 0.f, s10 = 0.f, s11 = 0.f;
 #pragma unroll
-                for (int jj = 0; jj < 4; ++jj) {
-                    uint32_t b0, b1, b2, b3;  // dims 32jj..+7, +8..15, +16..23, +24..31
-                    ldsm_x4(base + k_lane_off + 64 * jj, b0, b1, b2, b3);
-                    mma_k16(sa0, sa1, qa[2 * jj][0], qa[2 * jj][1], b0, b1, sa0, sa1);
-                    mma_k16(sb0, sb1, qa[2 * jj + 1][0], qa[2 * jj + 1][1], b2, b3, sb0, sb1);
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4(base + k_lane_off + 32 * j, b0, b1, b2, b3);
+                    mma_k16(s00, s01, qa[j][0], qa[j][1], b0, b1, s00, s01);
+                    mma_k16(s10, s11, qa[j][0], qa[j][1], b2, b3, s10, s11);
                 }
-                const float x0 = (sa0 + sb0) * scale_log2e, x1 = (sa1 + sb1) * scale_log2e;
-                const bool v0 = 2 * t < rows, v1 = 2 * t + 1 < rows;
+                const float x0 = s00 * scale_log2e, x1 = s01 * scale_log2e;
+                const float x2 = s10 * scale_log2e, x3 = s11 * scale_log2e;
+                const bool v0 = 2 * t < rows, v1 = 2 * t + 1 < rows, v2 = 8 + 2 * t < rows, v3 = 9 + 2 * t < rows;
                 float mx = kNegBig;
                 if (v0) mx = x0;
                 if (v1) mx = fmaxf(mx, x1);
+                if (v2) mx = fmaxf(mx, x2);
+                if (v3) mx = fmaxf(mx, x3);
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
                 mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
                 const float m_new = fmaxf(m_run, mx);
@@ -567,78 +554,48 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                 m_run = m_new;
                 const float p0 = v0 ? exp2f(x0 - m_new) : 0.f;
                 const float p1 = v1 ? exp2f(x1 - m_new) : 0.f;
-                l_run = l_run * alpha + (p0 + p1);
-                const uint32_t pa = pack_bf16(p0, p1);  // A operand: row g, tokens 2t, 2t+1
+                const float p2 = v2 ? exp2f(x2 - m_new) : 0.f;
+                const float p3 = v3 ? exp2f(x3 - m_new) : 0.f;
+                l_run = l_run * alpha + (p0 + p1 + p2 + p3);
+                const uint32_t pa0 = pack_bf16(p0, p1);  // A operand: row g, tokens 2t, 2t+1
+                const uint32_t pa2 = pack_bf16(p2, p3);  // row g, tokens 8+2t, 9+2t
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t b0, b1, b2, b3;  // output dims 32c..+7, +8.., +16.., +24..
-                    ldsm_x4_t(base + v_lane_off + 64 * c, b0, b1, b2, b3);
-                    mma_k8(o[4 * c][0], o[4 * c][1], pa, b0, o[4 * c][0] * alpha, o[4 * c][1] * alpha);
-                    mma_k8(o[4 * c + 1][0], o[4 * c + 1][1], pa, b1, o[4 * c + 1][0] * alpha, o[4 * c + 1][1] * alpha);
-                    mma_k8(o[4 * c + 2][0], o[4 * c + 2][1], pa, b2, o[4 * c + 2][0] * alpha, o[4 * c + 2][1] * alpha);
-                    mma_k8(o[4 * c + 3][0], o[4 * c + 3][1], pa, b3, o[4 * c + 3][0] * alpha, o[4 * c + 3][1] * alpha);
+                for (int c = 0; c < 8; ++c) {
+                    uint32_t b0, b1, b2, b3;
+                    ldsm_x4_t(base + v_lane_off + 32 * c, b0, b1, b2, b3);
+                    mma_k16(o[2 * c][0], o[2 * c][1], pa0, pa2, b0, b1, o[2 * c][0] * alpha, o[2 * c][1] * alpha);
+                    mma_k16(o[2 * c + 1][0], o[2 * c + 1][1], pa0, pa2, b2, b3, o[2 * c + 1][0] * alpha,
+                            o[2 * c + 1][1] * alpha);
                 }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
 
             if (flags & kFlagLast) {
-                // ---- combine the two halves of the item through shared memory, first half writes out
                 float L = l_run;
                 L += __shfl_xor_sync(0xffffffffu, L, 1);
                 L += __shfl_xor_sync(0xffffffffu, L, 2);
-                if (half == 1) {
-                    if (n_item > 0) ok = mbar_wait(bar_xfree + 8 * h, (n_item - 1) & 1, abort_word, status);
-                    if (!ok) break;
-                    if (g < G) {
+                if (g < G) {
+                    const int hq = h * G + g;
+                    if (item_nparts == 1) {
+                        const float inv = L > 0.f ? 1.f / L : 0.f;
+                        __nv_bfloat16* orow = out + ((int64_t)item_b * Hq + hq) * kMmaD;
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
-                            *reinterpret_cast<float2*>(xrow + 8 * i + 2 * t) = make_float2(o[i][0], o[i][1]);
+                            *reinterpret_cast<uint32_t*>(orow + 8 * i + 2 * t) = pack_bf16(o[i][0] * inv, o[i][1] * inv);
+                        if (lse != nullptr && t == 0)
+                            lse[(int64_t)item_b * Hq + hq] = L > 0.f ? (m_run + log2f(L)) * kLn2 : -CUDART_INF_F;
+                    } else {
+                        float* pr = partials + ((int64_t)item_part * Hq + hq) * (kMmaD + 2);
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            *reinterpret_cast<float2*>(pr + 8 * i + 2 * t) = make_float2(o[i][0], o[i][1]);
                         if (t == 0) {
-                            xrow[kMmaD] = m_run;
-                            xrow[kMmaD + 1] = L;
+                            pr[kMmaD] = m_run;
+                            pr[kMmaD + 1] = L;
                         }
                     }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_xfull + 8 * h);
-                } else {
-                    ok = mbar_wait(bar_xfull + 8 * h, n_item & 1, abort_word, status);
-                    if (!ok) break;
-                    if (g < G) {
-                        const float m1 = xrow[kMmaD], L1 = xrow[kMmaD + 1];
-                        const float M = fmaxf(m_run, m1);
-                        const float w0 = exp2f(m_run - M), w1 = exp2f(m1 - M);
-                        const float Lt = L * w0 + L1 * w1;
-                        const int hq = h * G + g;
-                        if (item.n_parts == 1) {
-                            const float inv = Lt > 0.f ? 1.f / Lt : 0.f;
-                            __nv_bfloat16* orow = out + ((int64_t)item.b * Hq + hq) * kMmaD;
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const float2 o1 = *reinterpret_cast<const float2*>(xrow + 8 * i + 2 * t);
-                                *reinterpret_cast<uint32_t*>(orow + 8 * i + 2 * t) =
-                                    pack_bf16((o[i][0] * w0 + o1.x * w1) * inv, (o[i][1] * w0 + o1.y * w1) * inv);
-                            }
-                            if (lse != nullptr && t == 0)
-                                lse[(int64_t)item.b * Hq + hq] = Lt > 0.f ? (M + log2f(Lt)) * kLn2 : -CUDART_INF_F;
-                        } else {
-                            float* pr = partials + ((int64_t)item.part * Hq + hq) * (kMmaD + 2);
-#pragma unroll
-                            for (int i = 0; i < 16; ++i) {
-                                const float2 o1 = *reinterpret_cast<const float2*>(xrow + 8 * i + 2 * t);
-                                *reinterpret_cast<float2*>(pr + 8 * i + 2 * t) =
-                                    make_float2(o[i][0] * w0 + o1.x * w1, o[i][1] * w0 + o1.y * w1);
-                            }
-                            if (t == 0) {
-                                pr[kMmaD] = M;
-                                pr[kMmaD + 1] = Lt;
-                            }
-                        }
-                    }
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(bar_xfree + 8 * h);
                 }
-                ++n_item;
             }
         }
     }
