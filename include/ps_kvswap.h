@@ -227,6 +227,52 @@ int32_t ps_missing_blocks(ps_ctx* ctx, int64_t req, int32_t* out);
 int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, float* lse,
                        const int64_t* reqs, int32_t batch);
 
+/* ---- decode attention without any allocation ---------------------------------------------- */
+
+/* The paper has no counterpart to this call; it exists for hosts that may not allocate.
+ *
+ * Some users of this library cannot call cudaMalloc (or anything that does so for them) when they
+ * need attention: an inference engine that gave all device memory to its own pool allocator at
+ * start-up, code living inside another program's memory budget, a latency-critical loop in which
+ * an allocation, which can synchronise the whole device, is not allowed.  ps_decode_attn above
+ * needs a context, and ps_create allocates that context's split-KV scratch.  This entry point
+ * computes the same attention with no context and no allocation: its scratch is a fixed array of
+ * PS_STATIC_SCRATCH_BYTES that is part of the library image (every GPU that loads the library
+ * holds it until the process exits), and everything else is the caller's memory.
+ *
+ *   kpool, vpool : device, bf16 [num_gpu_blocks][block_size][num_kv_heads][head_dim], one layer
+ *   q, out       : device, bf16 [batch][num_q_heads][head_dim]
+ *   lse          : device, fp32 [batch][num_q_heads], or NULL
+ *   block_tables : device, int32 [batch][table_stride]; row b lists the blocks of request b
+ *   ctx_lens     : HOST, int32 [batch]; tokens of request b (0 gives a zero row, lse = -inf)
+ *   kv_split_tokens : tokens per split-KV work item, 0 = chosen from the batch
+ *   status_word  : device int32 the kernels set to 2 when they meet a block id outside
+ *                  [0, num_gpu_blocks) (the access is skipped), or NULL to ignore
+ *   stream       : cudaStream_t on which everything is enqueued (asynchronous)
+ *   err_buf      : host buffer of err_cap bytes that receives the error text, or NULL
+ *
+ * Limits (PS_ERR_INVALID with a message naming the limit when exceeded): batch <=
+ * PS_STATIC_MAX_BATCH; at most 4096 work items (sum over requests of ceil(ctx / split)); their
+ * partial results, num_q_heads * (head_dim + 2) floats per item, must fit in the scratch less
+ * 192 KiB.  Shapes as for ps_decode_attn: head_dim 64 or 128, num_q_heads / num_kv_heads in
+ * {1, 2, 4, 8}.  Results equal those of ps_decode_attn with the CUDA-core kernel.
+ *
+ * The first call on a device looks up the scratch's device address (cudaGetSymbolAddress, with that
+ * device current) and caches it; make that first call before any stream capture begins.  All calls
+ * on a device share the one array, which still holds the previous call's contents: every call
+ * rewrites all metadata and the status word it owns before use, and partial results are written
+ * before they are read, so back-to-back calls on one stream are independent.  Calls whose kernels
+ * can overlap on the GPU (different streams with no ordering between them, or several host threads
+ * doing so) race on the array and give wrong results: order them.
+ * Errors: PS_ERR_INVALID, PS_ERR_CUDA.  Calls no cudaMalloc / cudaFree and no allocating routine. */
+#define PS_STATIC_MAX_BATCH 256
+#define PS_STATIC_SCRATCH_BYTES (16 * 1024 * 1024)
+int32_t ps_decode_attn_static(const void* kpool, const void* vpool, const void* q, void* out, float* lse,
+                              const int32_t* block_tables, int32_t table_stride, const int32_t* ctx_lens,
+                              int32_t batch, int32_t num_kv_heads, int32_t num_q_heads, int32_t head_dim,
+                              int32_t block_size, int32_t num_gpu_blocks, int32_t kv_split_tokens,
+                              int32_t* status_word, void* stream, char* err_buf, int32_t err_cap);
+
 /* ---- one engine step under the copy budget (Section 4.3 "Put it Together"; Alg. 1) -------- */
 
 /* In order: reaps finished offloads; turns copy_budget_bytes into blocks (floor(bytes /

@@ -30,6 +30,7 @@ EXPORTS = [
     "ps_num_free_blocks", "ps_swap_out", "ps_host_image", "ps_swap_in_begin", "ps_swap_in_cancel",
     "ps_swap_in_layer", "ps_missing_blocks", "ps_decode_attn", "ps_step", "ps_poll", "ps_sync",
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
+    "ps_decode_attn_static",
 ]
 
 
@@ -121,6 +122,8 @@ def load() -> C.CDLL:
         "ps_copy_blocks": (i32, [vp, i32, p32, i32, vp, i32]),
         "ps_trace": (i32, [vp, i32]),
         "ps_trace_read": (i32, [vp, C.POINTER(PsTraceSpan), i32, p32]),
+        "ps_decode_attn_static": (i32, [vp, vp, vp, vp, vp, vp, i32, p32, i32, i32, i32, i32, i32, i32, i32, vp, vp,
+                                        C.c_char_p, i32]),
     }
     for name, (res, args) in proto.items():
         fn = getattr(lib, name)
@@ -137,6 +140,32 @@ def ps_link_probe(nbytes: int, direction: int, iters: int = 10) -> float:
     if rc != PS_OK:
         raise PsError(rc, "ps_link_probe", load().ps_last_error(None).decode())
     return out.value
+
+
+PS_STATIC_MAX_BATCH = 256
+PS_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+
+def ps_decode_attn_static(kpool, vpool, q, out, block_tables, ctx_lens: Sequence[int], *, num_kv_heads: int,
+                          num_q_heads: int, head_dim: int, block_size: int, num_gpu_blocks: int,
+                          kv_split_tokens: int = 0, lse=None, status_word=None, stream: Optional[int] = None):
+    """Decode attention with no context and no allocation (scratch is a fixed array inside the library).
+
+    kpool, vpool, q, out, block_tables (int32 [batch][stride]), lse, status_word: device tensors;
+    ctx_lens: host integers.  Returns (status, error text).  See ps_decode_attn_static in the header:
+    calls on one device share the scratch, so overlapping calls on unordered streams race."""
+    if stream is None:
+        import torch
+        stream = torch.cuda.current_stream().cuda_stream
+    batch = len(ctx_lens)
+    arr = (C.c_int32 * max(batch, 1))(*[int(v) for v in ctx_lens])
+    err = C.create_string_buffer(512)
+    ptr = lambda t: C.c_void_p(t.data_ptr()) if t is not None else None
+    stride = int(block_tables.shape[-1]) if block_tables is not None and block_tables.dim() > 1 else 1
+    rc = load().ps_decode_attn_static(ptr(kpool), ptr(vpool), ptr(q), ptr(out), ptr(lse), ptr(block_tables), stride,
+                                      arr, batch, num_kv_heads, num_q_heads, head_dim, block_size, num_gpu_blocks,
+                                      kv_split_tokens, ptr(status_word), C.c_void_p(stream or None), err, 512)
+    return rc, err.value.decode()
 
 
 def _i64_array(vals: Sequence[int]):

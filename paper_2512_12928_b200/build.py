@@ -16,7 +16,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB_DIR = os.path.join(PKG, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libps_kvswap.so")
-SOURCES = ["ps_runtime.cu", "ps_copy_kernels.cu", "ps_attn_kernels.cu"]
+SOURCES = ["ps_runtime.cu", "ps_copy_kernels.cu", "ps_attn_kernels.cu", "ps_static_scratch.cu"]
 HEADERS = [os.path.join(CSRC, "ps_internal.h"), os.path.join(ROOT, "include", "ps_kvswap.h")]
 
 
