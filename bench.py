@@ -52,13 +52,22 @@ def read_peaks():
 
 
 def read_traffic_ratio():
-    """DRAM bytes per algorithmic byte of the attention kernel, from the committed ncu summary."""
-    path = os.path.join(ROOT, "profiles", "attn_traffic.json")
-    if os.path.exists(path):
-        try:
-            return float(json.load(open(path))["dram_bytes_per_algorithmic_byte"])
-        except Exception:
-            return None
+    """DRAM bytes per algorithmic byte of the attention kernel from the committed ncu summary, or None when
+    the kernel source has changed since that capture (the counters then describe another kernel)."""
+    import glob
+    import hashlib
+    import re
+    src = os.path.join(ROOT, "paper_2512_12928_b200", "csrc", "ps_attn_kernels.cu")
+    try:
+        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+    except OSError:
+        return None
+    for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "decode_attn_mma_*.md"))):
+        text = open(path).read()
+        m_sha = re.search(r"^kernel_source_sha256:\s*([0-9a-f]{64})", text, re.M)
+        m_ratio = re.search(r"^dram_bytes_per_algorithmic_byte:\s*([0-9.]+)", text, re.M)
+        if m_sha and m_ratio and m_sha.group(1) == sha:
+            return float(m_ratio.group(1))
     return None
 
 
@@ -295,8 +304,28 @@ def time_decode_steps(torch, lib, reqs, q, out, n):
     return e0.elapsed_time(e1) / n
 
 
+def kv_bytes_per_layer(sh, ctx_lens, reqs):
+    """K and V bytes one layer of decode attention addresses for these requests (the algorithmic bytes)."""
+    return sum(ctx_lens[r] for r in reqs) * 2 * sh.num_kv_heads * sh.head_dim * 2
+
+
+def decode_roofline(torch, lib, sh, ctx_lens, reqs, q, out, steps=5):
+    """Decode-only steps (nothing to reload): average duration of one attention launch, CUDA events around
+    `steps` whole steps on the compute stream (no per-launch events), and the HBM rate that implies."""
+    n0 = lib.launch_count()
+    step_ms = time_decode_steps(torch, lib, reqs, q, out, steps)
+    launches = (lib.launch_count() - n0) / steps
+    alg = kv_bytes_per_layer(sh, ctx_lens, reqs)
+    us = step_ms * 1e3 / sh.num_layers
+    return {"us_per_layer": us, "launches_per_layer": launches / sh.num_layers, "algorithmic_bytes_per_launch": alg,
+            "gbs": alg / us / 1e3, "step_us": step_ms * 1e3}
+
+
 def overlap_sweep(torch, B, K, V, peaks_hbm):
-    """Overlap workload: decode batch 128 + 8 preempted requests reloading under 16/64/256 MiB budgets."""
+    """Overlap workload: decode batch 128 + 8 preempted requests reloading under 16/64/256 MiB budgets.
+
+    Contexts carry no per-launch profiling events: under host-link load those events delay the compute
+    stream's commands and would be charged to the reload."""
     w = wl.overlap()
     sh = w.shape
     nb = sh.num_gpu_blocks
@@ -304,7 +333,7 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
     res = {"workload": "overlap: decode batch 128, lognormal contexts (mean 2k, cap 8k), 8 preempted requests"}
     stream = torch.cuda.current_stream()
     for mode in ("pipelined", "sync_reload"):
-        flags = B.PS_FLAG_PROFILE | (B.PS_FLAG_SYNC_RELOAD if mode == "sync_reload" else 0)
+        flags = B.PS_FLAG_SYNC_RELOAD if mode == "sync_reload" else 0
         lib = make_ctx(B, w, K, V, nb, max_batch=len(w.ctx_lens), host_pool_bytes=host_bytes, flags=flags)
         for r, n in wl.build_order_round_robin(w):
             assert lib.kv_alloc(r, n) == 0, lib.last_error()
@@ -318,6 +347,13 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
         reload_bytes = sum(sh.blocks_for(w.ctx_lens[r]) for r in w.victims) * sh.block_bytes
         budgets = w.budgets + [-1] if mode == "pipelined" else [256 * wl.MiB, -1]
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if mode == "pipelined":
+            for _ in range(3):
+                time_decode_steps(torch, lib, batch, sub_batch(q, len(batch)), sub_batch(out, len(batch)), 1)
+            rf = decode_roofline(torch, lib, sh, w.ctx_lens, batch, sub_batch(q, len(batch)), sub_batch(out, len(batch)))
+            res["attn_gbs"] = rf["gbs"]
+            res["attn_frac_of_hbm"] = rf["gbs"] / peaks_hbm
+            res["attn_us_per_layer"] = rf["us_per_layer"]
         for r in w.victims:
             assert lib.swap_out(r) == 0, lib.last_error()
         assert lib.sync() == 0
@@ -376,39 +412,41 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
             for r in w.victims:
                 assert lib.swap_out(r) == 0
             assert lib.sync() == 0
-        prof = lib.get_profile()
-        if mode == "pipelined" and prof["attn_ms"] > 0:
-            gbs = prof["attn_kv_bytes"] / prof["attn_ms"] / 1e6
-            res["attn_gbs"] = gbs
-            res["attn_frac_of_hbm"] = gbs / peaks_hbm
-            res["attn_us_per_launch"] = prof["attn_ms"] / prof["attn_launches"] * 1e3
         lib.destroy()
     return res
 
 
-def kernel_rates(torch, B, lib, sh, nb, n_blocks=2048, iters=10):
-    """Gather / scatter kernels alone (no host link): payload read once + written once per launch."""
+def kernel_rates(torch, B, lib, sh, nb, n_blocks=2048, iters=20):
+    """Gather / scatter kernels alone (no host link): payload read once + written once per launch.
+
+    The launches are enqueued back to back (the ids are marshalled once), so the GPU never waits for the
+    host; the time per launch includes the small upload kernel that carries the ids."""
+    import ctypes as C
     rng = np.random.default_rng(3)
-    ids = [int(v) for v in rng.permutation(nb)[:n_blocks]]
+    ids = (C.c_int32 * n_blocks)(*[int(v) for v in rng.permutation(nb)[:n_blocks]])
     stage = torch.empty((n_blocks, 2, sh.block_size, sh.num_kv_heads, sh.head_dim), dtype=torch.bfloat16, device="cuda")
-    # the scatter writes blocks: use free ones only
     res = {}
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     payload = n_blocks * sh.layer_block_bytes
+
+    def launch(i, direction):
+        rc = lib.lib.ps_copy_blocks(lib.h, i % sh.num_layers, ids, n_blocks, C.c_void_p(stage.data_ptr()), direction)
+        assert rc == 0, lib.last_error()
+
     for name, direction in (("gather", 0), ("scatter", 1)):   # the scatter overwrites pool blocks: run last
-        best = None
-        for it in range(iters + 2):
-            layer = it % sh.num_layers
-            e0.record()
-            assert lib.copy_blocks(layer, ids, stage, direction) == 0, lib.last_error()
-            e1.record(); e1.synchronize()
-            ms = e0.elapsed_time(e1)
-            if it >= 2:
-                best = ms if best is None else min(best, ms)
-        res[name + "_gbs_rw"] = 2 * payload / best / 1e6
-        res[name + "_us"] = best * 1e3
+        for i in range(3):
+            launch(i, direction)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(iters):
+            launch(i, direction)
+        e1.record(); e1.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        res[name + "_gbs_rw"] = 2 * payload / ms / 1e6
+        res[name + "_us"] = ms * 1e3
     res["blocks_per_launch"] = n_blocks
     res["payload_bytes_per_launch"] = payload
+    res["launches_timed"] = iters
     return res
 
 
@@ -444,10 +482,6 @@ def run_gpu(args):
     torch.cuda.synchronize()
 
     victim_bytes = sum(sh.blocks_for(w.ctx_lens[r]) for r in w.victims) * sh.block_bytes
-    lib = make_ctx(B, w, K, V, sh.num_gpu_blocks, max_batch=len(w.ctx_lens),
-                   host_pool_bytes=victim_bytes + (256 << 20), flags=B.PS_FLAG_PROFILE)
-    for r, n in wl.build_order_round_robin(w):
-        assert lib.kv_alloc(r, n) == 0, lib.last_error()
     nreq = len(w.ctx_lens)
     g = torch.Generator(device="cuda")
     g.manual_seed(w.seed)
@@ -456,13 +490,21 @@ def run_gpu(args):
     out = torch.zeros_like(q)
     budget = args.budget_mib * wl.MiB if args.budget_mib >= 0 else -1
     e2e_bufs = {"q_host": q.cpu().pin_memory(), "out_host": torch.zeros_like(q, device="cpu").pin_memory()}
-
     n_res = nreq - len(w.victims)
     q_res = sub_batch(q, n_res).clone()
     out_res = torch.zeros_like(q_res)
+
+    def fresh_ctx(flags):
+        lib = make_ctx(B, w, K, V, sh.num_gpu_blocks, max_batch=nreq, host_pool_bytes=victim_bytes + (256 << 20),
+                       flags=flags)
+        for r, n in wl.build_order_round_robin(w):
+            assert lib.kv_alloc(r, n) == 0, lib.last_error()
+        return lib
+
+    # ---- the timed region: no per-launch events (they delay the compute stream under host-link load)
+    lib = fresh_ctx(0)
     for _ in range(args.warmup):
         swap_workload_step(torch, B, lib, w, q, out, q_res, out_res, budget)
-    lib.get_profile(reset=True)
     launches0 = lib.launch_count()
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -475,9 +517,7 @@ def run_gpu(args):
     if world > 1:
         dist.barrier()
     wall_ms = (time.perf_counter() - t_wall0) * 1e3
-    clocks = sampler.stop()
     launches = lib.launch_count() - launches0
-    prof = lib.get_profile(reset=True)
 
     out_ms = sum(r["out_ms"] for r in recs)
     in_ms = sum(r["in_ms"] for r in recs)
@@ -489,7 +529,17 @@ def run_gpu(args):
     moved = 2 * victim_bytes * args.steps * world
     value = moved / total_ms / 1e6
 
-    # end-to-end arm: queries from pinned host memory and outputs back to it, every decode step
+    # ---- the dominant kernel, live, in the launch configuration of the step: decode-only steps of the
+    # whole batch between two CUDA events on the compute stream (still inside the clock-sampled region)
+    all_reqs = list(range(nreq))
+    residents = [r for r in all_reqs if r not in set(w.victims)]
+    time_decode_steps(torch, lib, all_reqs, q, out, 2)
+    rf_all = decode_roofline(torch, lib, sh, w.ctx_lens, all_reqs, q, out, steps=5)
+    time_decode_steps(torch, lib, residents, q_res, out_res, 2)
+    rf_res = decode_roofline(torch, lib, sh, w.ctx_lens, residents, q_res, out_res, steps=5)
+    clocks = sampler.stop()
+
+    # ---- end-to-end arm: queries from pinned host memory and outputs back to it, every decode step
     e2e_recs = [swap_workload_step(torch, B, lib, w, q, out, q_res, out_res, budget, e2e_bufs)
                 for _ in range(max(1, min(args.steps, 2)))]
     e2e_ms = sum(r["out_ms"] + r["in_ms"] for r in e2e_recs)
@@ -504,7 +554,6 @@ def run_gpu(args):
            "d2h_bytes_per_step": int(victim_bytes + e2e_steps * q_bytes),
            "note": "host images live in pinned host memory by definition; this arm adds the per-decode-step "
                    "upload of the queries from pinned host memory and the download of the attention output"}
-    lib.get_profile(reset=True)
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -514,43 +563,55 @@ def run_gpu(args):
                    "q_heads": sh.num_q_heads, "head_dim": sh.head_dim, "block_size": sh.block_size,
                    "gpu_blocks": sh.num_gpu_blocks, "resident_requests": nreq, "victims": len(w.victims),
                    "victim_bytes": victim_bytes, "copy_budget_mib_per_step": args.budget_mib,
-                   "l2": "inputs larger than L2 (5 GiB swapped, ~0.4 GiB of KV read per attention launch)",
+                   "l2": "inputs larger than L2 (6 GiB swapped each way, ~0.6 GiB of KV read per attention launch)",
                    "parallelism": "independent replicas" if world > 1 else "single GPU"},
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "wall_ms": wall_ms,
     }
     if rank == 0:
-        attn_ms = prof["attn_ms"]
-        attn_gbs = prof["attn_kv_bytes"] / attn_ms / 1e6 if attn_ms > 0 else None
         ratio = read_traffic_ratio()
-        per_launch_bytes = prof["attn_kv_bytes"] / max(prof["attn_launches"], 1)
         result["roofline"] = {
-            "kernel": "decode_attn (paged GQA decode attention)", "bound": "hbm", "achieved": attn_gbs,
-            "peak": hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth", "unit": "GB/s",
-            "frac": attn_gbs / hbm_peak if attn_gbs else None,
-            "traffic": ratio * per_launch_bytes if ratio else None,
-            "algorithmic_bytes_per_launch": per_launch_bytes,
-            "us_per_launch": attn_ms / max(prof["attn_launches"], 1) * 1e3, "launches": prof["attn_launches"],
-            "frac_of_nominal_8TBs": attn_gbs / 8000.0 if attn_gbs else None,
+            "kernel": "decode_attn_mma_kernel (paged GQA decode attention, split-KV combined in the kernel)",
+            "bound": "hbm", "achieved": rf_all["gbs"], "peak": hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth",
+            "unit": "GB/s", "frac": rf_all["gbs"] / hbm_peak,
+            "traffic": ratio * rf_all["algorithmic_bytes_per_launch"] if ratio else None,
+            "algorithmic_bytes_per_launch": rf_all["algorithmic_bytes_per_launch"],
+            "us_per_launch": rf_all["us_per_layer"], "launches_per_layer": rf_all["launches_per_layer"],
+            "how": "CUDA events around 5 decode-only steps (32 launches each, all 64 requests) on the compute "
+                   "stream; duration per launch includes the launch gap",
+            "frac_of_nominal_8TBs": rf_all["gbs"] / 8000.0,
+            "batch_of_48_residents": {"gbs": rf_res["gbs"], "us_per_launch": rf_res["us_per_layer"],
+                                      "frac": rf_res["gbs"] / hbm_peak},
         }
-        gather_gbs = 2 * prof["gather_bytes"] / prof["gather_ms"] / 1e6 if prof["gather_ms"] > 0 else None
-        scatter_gbs = 2 * prof["scatter_bytes"] / prof["scatter_ms"] / 1e6 if prof["scatter_ms"] > 0 else None
         result["swap"] = {
             "swap_out_gbs": victim_bytes * args.steps / out_ms / 1e6, "swap_in_gbs": victim_bytes * args.steps / in_ms / 1e6,
             "swap_out_frac_of_link": victim_bytes * args.steps / out_ms / 1e6 / link["d2h_gbs"],
             "swap_in_frac_of_link": victim_bytes * args.steps / in_ms / 1e6 / link["h2d_gbs"],
-            "d2h_engine_gbs": prof["d2h_bytes"] / prof["d2h_ms"] / 1e6 if prof["d2h_ms"] > 0 else None,
-            "h2d_engine_gbs": prof["h2d_bytes"] / prof["h2d_ms"] / 1e6 if prof["h2d_ms"] > 0 else None,
-            "gather_in_step_gbs_rw": gather_gbs, "scatter_in_step_gbs_rw": scatter_gbs,
             "decode_steps_during_out": recs[-1]["steps_out"], "decode_steps_during_in": recs[-1]["steps_in"],
+            "decode_step_us_during_out": recs[-1]["out_ms"] / recs[-1]["steps_out"] * 1e3,
+            "decode_step_us_no_swap": rf_res["step_us"],
             "link": link,
         }
-        kr = kernel_rates(torch, B, lib, sh, sh.num_gpu_blocks)
+    lib.destroy()
+    del lib
+    if rank == 0:
+        # diagnostics pass with per-launch events (not part of any reported rate above): engine and kernel
+        # rates inside a step; the events themselves slow this pass down
+        plib = fresh_ctx(B.PS_FLAG_PROFILE)
+        swap_workload_step(torch, B, plib, w, q, out, q_res, out_res, budget)
+        prof = plib.get_profile(reset=True)
+        result["swap"].update({
+            "d2h_engine_gbs": prof["d2h_bytes"] / prof["d2h_ms"] / 1e6 if prof["d2h_ms"] > 0 else None,
+            "h2d_engine_gbs": prof["h2d_bytes"] / prof["h2d_ms"] / 1e6 if prof["h2d_ms"] > 0 else None,
+            "gather_in_step_gbs_rw": 2 * prof["gather_bytes"] / prof["gather_ms"] / 1e6 if prof["gather_ms"] > 0 else None,
+            "scatter_in_step_gbs_rw": 2 * prof["scatter_bytes"] / prof["scatter_ms"] / 1e6 if prof["scatter_ms"] > 0 else None,
+        })
+        kr = kernel_rates(torch, B, plib, sh, sh.num_gpu_blocks)
         kr["gather_frac_of_hbm"] = kr["gather_gbs_rw"] / hbm_peak
         kr["scatter_frac_of_hbm"] = kr["scatter_gbs_rw"] / hbm_peak
         result["gather_scatter_alone"] = kr
-    lib.destroy()
-    del lib
+        plib.destroy()
+        del plib
     if rank == 0 and not args.no_overlap:
         result["overlap"] = overlap_sweep(torch, B, K, V, hbm_peak)
     if rank == 0 and world == 1:

@@ -70,7 +70,9 @@ enum ps_flags {
        ps_decode_attn and the q/out arguments of ps_step are rejected in this mode. */
     PS_FLAG_BOOKKEEPING_ONLY = 1,
     /* Record CUDA events around every kernel and transfer so that ps_get_profile can report
-       per-kind device times.  Costs two event records per launch. */
+       per-kind device times.  Costs two event records per launch; while a host transfer saturates
+       the link these records delay the compute stream's commands noticeably (a decode step grew
+       from 3.8 to 6.4 ms in one measurement), so use it for diagnosis, not inside timed runs. */
     PS_FLAG_PROFILE = 2,
     /* Ablation (Section 5, block-management ablation "w/o async"): ps_step finishes the whole
        reload before the first attention launch instead of pipelining it layer by layer. */
@@ -253,7 +255,7 @@ int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, flo
  *
  * Limits (PS_ERR_INVALID with a message naming the limit when exceeded): batch <=
  * PS_STATIC_MAX_BATCH; at most 4096 work items (sum over requests of ceil(ctx / split)); their
- * partial results, num_q_heads * (head_dim + 2) floats per item, must fit in the scratch less
+ * partial results, num_q_heads * (head_dim + 4) floats per item, must fit in the scratch less
  * 192 KiB.  Shapes as for ps_decode_attn: head_dim 64 or 128, num_q_heads / num_kv_heads in
  * {1, 2, 4, 8}.  Results equal those of ps_decode_attn with the CUDA-core kernel.
  *
@@ -280,9 +282,9 @@ int32_t ps_decode_attn_static(const void* kpool, const void* vpool, const void* 
  * a request whose missing blocks fit is taken whole, the first that does not fit gets what is
  * left; then for each layer issues that layer's reload (as ps_swap_in_layer) and launches that
  * layer's attention for the requests of `reqs` that are RESIDENT once this step's reload is
- * issued.  Requests complete before the step run without waiting; requests completed by this
- * step run in a second launch that waits on the layer's reload event.  Everything is enqueued
- * asynchronously.
+ * issued.  When the batch holds requests completed by this step, each layer's attention launch
+ * waits on that layer's reload event (and on nothing later), so the reload of layer i+1 runs
+ * under the attention of layer i.  Everything is enqueued asynchronously.
  *   q_all_layers, out_all_layers : device, bf16 [num_layers][batch][num_q_heads][head_dim]; rows of
  *                                  requests that do not decode are left untouched.  Both may be
  *                                  NULL with batch 0 for a copy-only step.

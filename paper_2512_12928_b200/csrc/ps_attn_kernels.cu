@@ -287,9 +287,11 @@ constexpr int kMmaPitch = kMmaRowBytes + 16;              // 2064: breaks the 2 
 constexpr int kMmaSlabBytes = kMmaTileTokens * kMmaPitch; // one K (or V) tile in shared memory
 constexpr int kMmaStageBytes = 2 * kMmaSlabBytes;
 constexpr int kMmaRingBytes = kMmaStages * kMmaStageBytes;
-constexpr int kMmaCtrlBytes = 256;                        // barriers, stage descriptors, abort word
+constexpr int kMmaMaxPending = 14;                        // rows a warp may note for combining after its last tile
+constexpr int kMmaCtrlBytes = 128 + 8 * 16 * 4;           // barriers, stage descriptors, abort word; pending-row lists
 constexpr int kMmaConsumerWarps = kMmaHkv;
 constexpr int kMmaThreads = (kMmaConsumerWarps + 1) * 32;
+constexpr int kMmaPartStride = kMmaD + 4;                 // floats per (part, query head): 16-byte aligned rows
 constexpr int kSpinLimit = 1 << 22;
 constexpr int kFlagFirst = 1, kFlagLast = 2, kFlagEnd = 4;
 
@@ -340,10 +342,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     return __all_sync(0xffffffffu, ok);
 }
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
+// KV rows are read once per launch: they are marked evict-first in L2 so that the split-KV partials (written and
+// re-read within the launch) and the batch metadata stay resident under the stream.
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
+        "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+        : "memory");
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
@@ -369,13 +379,94 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// Combines the parts of batch row b for the G query heads of KV head h (one warp; every part has been
+// delivered and fenced).  Parts are combined in part order, whoever calls.  The loads of all G heads
+// are issued together, two parts at a time.  Re-arms the row's arrival counter.
+template <int G>
+__device__ __forceinline__ void merge_row(int b, int h, int lane, const AttnBatch& batch,
+                                          const float* __restrict__ partials, __nv_bfloat16* __restrict__ out,
+                                          float* __restrict__ lse, int32_t* __restrict__ row_done) {
+    constexpr int Hq = kMmaHkv * G;
+    __threadfence();
+    const int n = batch.row_parts[b];
+    const float* base = partials + ((int64_t)batch.row_first_part[b] * Hq + h * G) * kMmaPartStride;
+    const int64_t stride = (int64_t)Hq * kMmaPartStride;   // floats between parts
+    // pass 1: per head the maximum over the parts (lanes stride over the parts)
+    float M[G];
+#pragma unroll
+    for (int gg = 0; gg < G; ++gg) M[gg] = kNegBig;
+    for (int i = lane; i < n; i += 32)
+#pragma unroll
+        for (int gg = 0; gg < G; ++gg) M[gg] = fmaxf(M[gg], __ldcg(base + i * stride + gg * kMmaPartStride + kMmaD));
+#pragma unroll
+    for (int gg = 0; gg < G; ++gg)
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) M[gg] = fmaxf(M[gg], __shfl_xor_sync(0xffffffffu, M[gg], off));
+    // pass 2: lane owns dims [4 lane, 4 lane + 4) of every head
+    float4 acc[G];
+    float Ls[G];
+#pragma unroll
+    for (int gg = 0; gg < G; ++gg) {
+        acc[gg] = make_float4(0.f, 0.f, 0.f, 0.f);
+        Ls[gg] = 0.f;
+    }
+    for (int i0 = 0; i0 < n; i0 += 2) {
+        const bool two = i0 + 1 < n;
+        float4 va[G], vb[G];
+        float ma[G], la[G], mb[G], lb[G];
+#pragma unroll
+        for (int gg = 0; gg < G; ++gg) {
+            const float* pa = base + i0 * stride + gg * kMmaPartStride;
+            va[gg] = __ldcg(reinterpret_cast<const float4*>(pa) + lane);
+            ma[gg] = __ldcg(pa + kMmaD);
+            la[gg] = __ldcg(pa + kMmaD + 1);
+            vb[gg] = make_float4(0.f, 0.f, 0.f, 0.f);
+            mb[gg] = kNegBig;
+            lb[gg] = 0.f;
+            if (two) {
+                vb[gg] = __ldcg(reinterpret_cast<const float4*>(pa + stride) + lane);
+                mb[gg] = __ldcg(pa + stride + kMmaD);
+                lb[gg] = __ldcg(pa + stride + kMmaD + 1);
+            }
+        }
+#pragma unroll
+        for (int gg = 0; gg < G; ++gg) {
+            const float wa = exp2f(ma[gg] - M[gg]);
+            const float wb = two ? exp2f(mb[gg] - M[gg]) : 0.f;
+            Ls[gg] = fmaf(la[gg], wa, Ls[gg]);
+            acc[gg].x = fmaf(va[gg].x, wa, acc[gg].x);
+            acc[gg].y = fmaf(va[gg].y, wa, acc[gg].y);
+            acc[gg].z = fmaf(va[gg].z, wa, acc[gg].z);
+            acc[gg].w = fmaf(va[gg].w, wa, acc[gg].w);
+            Ls[gg] = fmaf(lb[gg], wb, Ls[gg]);
+            acc[gg].x = fmaf(vb[gg].x, wb, acc[gg].x);
+            acc[gg].y = fmaf(vb[gg].y, wb, acc[gg].y);
+            acc[gg].z = fmaf(vb[gg].z, wb, acc[gg].z);
+            acc[gg].w = fmaf(vb[gg].w, wb, acc[gg].w);
+        }
+    }
+#pragma unroll
+    for (int gg = 0; gg < G; ++gg) {
+        const int hq = h * G + gg;
+        const float inv = Ls[gg] > 0.f ? 1.f / Ls[gg] : 0.f;
+        __nv_bfloat16* orow = out + ((int64_t)b * Hq + hq) * kMmaD;
+        uint2 packed;
+        packed.x = pack_bf16(acc[gg].x * inv, acc[gg].y * inv);
+        packed.y = pack_bf16(acc[gg].z * inv, acc[gg].w * inv);
+        *reinterpret_cast<uint2*>(orow + 4 * lane) = packed;
+        if (lse != nullptr && lane == 0)
+            lse[(int64_t)b * Hq + hq] = Ls[gg] > 0.f ? (M[gg] + log2f(Ls[gg])) * kLn2 : -CUDART_INF_F;
+    }
+    if (lane == 0) row_done[b * kMmaHkv + h] = 0;  // every part has arrived: re-arm for the next launch
+}
+
 template <int G>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloat16* __restrict__ vpool,
                        const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
                        AttnBatch batch, int32_t sched_lane, int32_t block_size, int32_t block_shift,
                        int32_t num_blocks, float* __restrict__ partials, int32_t* __restrict__ sched,
-                       float scale_log2e, int32_t* status) {
+                       int32_t* __restrict__ row_done, float scale_log2e, int32_t* status) {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int Hq = kMmaHkv * G;
     const uint32_t ring = smem_u32(smem);
@@ -409,6 +500,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
 
     if (warp == kMmaConsumerWarps) {
         // ------------------------------------------------ producer warp
+        const uint64_t kv_policy = l2_evict_first_policy();
         int n = 0;
         bool ok = true;
         int32_t* counter = sched + 2 * sched_lane;
@@ -460,7 +552,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                     if (r < rows) {
                         const int64_t off = ((int64_t)id * block_size + slot + r) * (kMmaRowBytes / 2);  // elements
                         const uint32_t dst = ring + s * kMmaStageBytes + (lane < 16 ? 0 : kMmaSlabBytes) + r * kMmaPitch;
-                        bulk_g2s(dst, (lane < 16 ? kpool : vpool) + off, kMmaRowBytes, full);
+                        bulk_g2s(dst, (lane < 16 ? kpool : vpool) + off, kMmaRowBytes, full, kv_policy);
                     }
                 }
             }
@@ -499,6 +591,8 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
         float o[16][2];
         float m_run = kNegBig, l_run = 0.f;
         int item_b = 0, item_part = 0, item_nparts = 1;
+        volatile int32_t* pending = reinterpret_cast<volatile int32_t*>(ctrl + 128) + warp * 16;
+        int n_pend = 0;
         bool ok = true;
 #pragma unroll
         for (int j = 0; j < 8; ++j) qa[j][0] = qa[j][1] = 0u;
@@ -586,7 +680,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                         if (lse != nullptr && t == 0)
                             lse[(int64_t)item_b * Hq + hq] = L > 0.f ? (m_run + log2f(L)) * kLn2 : -CUDART_INF_F;
                     } else {
-                        float* pr = partials + ((int64_t)item_part * Hq + hq) * (kMmaD + 2);
+                        float* pr = partials + ((int64_t)item_part * Hq + hq) * kMmaPartStride;
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
                             *reinterpret_cast<float2*>(pr + 8 * i + 2 * t) = make_float2(o[i][0], o[i][1]);
@@ -596,26 +690,48 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                         }
                     }
                 }
+                if (item_nparts > 1) {
+                    // Split-KV fix-up: the warp that delivers the last part of a (row, KV head) combines the
+                    // parts.  Combining costs a few round trips to L2 during which this warp would hold up the
+                    // CTA's ring, so the row is only noted here and combined after the CTA's last tile.
+                    __threadfence();
+                    __syncwarp();
+                    int prev = 0;
+                    if (lane == 0) prev = atomicAdd(row_done + item_b * kMmaHkv + h, 1);
+                    prev = __shfl_sync(0xffffffffu, prev, 0);
+                    if (prev == item_nparts - 1) {
+                        if (n_pend < kMmaMaxPending) {
+                            if (lane == 0) pending[n_pend] = item_b;
+                            ++n_pend;
+                        } else {
+                            merge_row<G>(item_b, h, lane, batch, partials, out, lse, row_done);
+                        }
+                    }
+                }
             }
+        }
+        if (ok) {
+            __syncwarp();
+            for (int p = 0; p < n_pend; ++p) merge_row<G>(pending[p], h, lane, batch, partials, out, lse, row_done);
         }
     }
 }
 
 template <int G>
 cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool, const void* q, void* out, float* lse,
-                       const AttnBatch& batch, int32_t lane, float* partials, int32_t* sched, int32_t* d_status,
-                       cudaStream_t stream) {
+                       const AttnBatch& batch, int32_t lane, float* partials, int32_t* sched, int32_t* row_done,
+                       int32_t* d_status, cudaStream_t stream) {
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)kMmaD);
     decode_attn_mma_kernel<G><<<(unsigned)batch.n_cta[lane], kMmaThreads, mma_smem_bytes(G), stream>>>(
         (const __nv_bfloat16*)kpool, (const __nv_bfloat16*)vpool, (const __nv_bfloat16*)q, (__nv_bfloat16*)out, lse, batch,
-        lane, sh.block_size, shift_of(sh.block_size), sh.num_blocks, partials, sched, scale_log2e, d_status);
+        lane, sh.block_size, shift_of(sh.block_size), sh.num_blocks, partials, sched, row_done, scale_log2e, d_status);
     return cudaGetLastError();
 }
 
 }  // namespace
 
 size_t attn_partial_bytes(const AttnShape& sh, int32_t max_parts) {
-    return (size_t)max_parts * sh.num_q_heads * (sh.head_dim + 2) * sizeof(float);
+    return (size_t)max_parts * sh.num_q_heads * (sh.head_dim + 4) * sizeof(float);
 }
 
 bool attn_mma_supported(const AttnShape& sh) {
@@ -637,19 +753,24 @@ cudaError_t attn_init() {
 
 cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool, const void* q,
                                void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials,
-                               int32_t* sched, int32_t* d_status, cudaStream_t stream) {
+                               int32_t* sched, int32_t* row_done, int32_t* d_status, cudaStream_t stream) {
     if (lane < 0 || lane > 1) return cudaErrorInvalidValue;
     const int item_begin = batch.lane_items[lane];
     const int n_items = batch.lane_items[lane + 1] - item_begin;
     if (n_items <= 0) return cudaSuccess;
     const int G = sh.num_q_heads / sh.num_kv_heads;
     if (kernel == 2) {
-        if (!attn_mma_supported(sh) || batch.n_cta[lane] <= 0) return cudaErrorNotSupported;
+        if (!attn_mma_supported(sh) || batch.n_cta[lane] <= 0 || sched == nullptr || row_done == nullptr)
+            return cudaErrorNotSupported;
         switch (G) {
-            case 1: return launch_mma<1>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, d_status, stream);
-            case 2: return launch_mma<2>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, d_status, stream);
-            case 4: return launch_mma<4>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, d_status, stream);
-            case 8: return launch_mma<8>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, d_status, stream);
+            case 1: return launch_mma<1>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+                                       stream);
+            case 2: return launch_mma<2>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+                                       stream);
+            case 4: return launch_mma<4>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+                                       stream);
+            case 8: return launch_mma<8>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+                                       stream);
         }
         return cudaErrorNotSupported;
     }

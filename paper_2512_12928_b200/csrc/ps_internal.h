@@ -70,16 +70,20 @@ struct AttnBatch {                 // device pointers to the per-batch metadata
 };
 
 // Partial results: per (part, q head): D floats of unnormalised output, then the running max
-// (log2 units) and the running sum.  Row stride D + 2 floats.
+// (log2 units) and the running sum.  The CUDA-core kernel and the merge kernel use a row stride of
+// D + 2 floats, the tensor-core kernel D + 4 (16-byte aligned rows); the buffer is sized for D + 4.
 size_t attn_partial_bytes(const AttnShape& sh, int32_t max_parts);
 
 // Launches the attention kernel for the items of one lane.  kernel: 1 = SIMT (one CTA per item and
-// KV head), 2 = MMA (CTA c of the lane walks items [cta_begin[c], cta_begin[c+1]), then takes dynamic
-// chunks through the counters in sched: 2 int32 per lane, zero before the first launch, re-armed by
-// the kernel itself).
+// KV head; rows with several parts need launch_attn_merge afterwards), 2 = MMA (CTA c of the lane walks
+// items [cta_begin[c], cta_begin[c+1]), then takes dynamic chunks through the counters in sched: 2 int32
+// per lane, zero before the first launch, re-armed by the kernel itself; rows with several parts are
+// combined inside the kernel by whichever warp delivers the last part, counted in row_done:
+// batch x num_kv_heads int32, zero before the first launch, re-armed by the kernel).  sched and
+// row_done may be null for the SIMT kernel.
 cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool, const void* q,
                                void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials,
-                               int32_t* sched, int32_t* d_status, cudaStream_t stream);
+                               int32_t* sched, int32_t* row_done, int32_t* d_status, cudaStream_t stream);
 
 // Token granularity at which the tensor-core kernel splits a context.
 constexpr int kMmaTileTokens = 16;

@@ -4,7 +4,8 @@
 //
 // Streams (Appendix B: a copy stream per direction, independent of the compute stream; one
 // completion event per layer chunk):
-//   compute  : the caller's stream; attention runs here.
+//   compute  : the caller's stream; attention runs here (a layer's launch waits on that layer's reload
+//              event when the batch holds requests whose reload is landing in this step).
 //   s_gather : gather kernels of swap-out.           s_d2h : staging -> pinned host copies.
 //   s_h2d    : pinned host -> staging copies.        s_scatter : scatter kernels of swap-in.
 // Each direction owns kSlots staging slots; two events per slot hand a slot back and forth between
@@ -148,8 +149,7 @@ struct ps_ctx {
     char* host_pool = nullptr;
     bool own_host_pool = false;
     HostPool hpool;
-    cudaStream_t compute = nullptr, s_gather = nullptr, s_d2h = nullptr, s_h2d = nullptr, s_scatter = nullptr,
-                 s_lane = nullptr;
+    cudaStream_t compute = nullptr, s_gather = nullptr, s_d2h = nullptr, s_h2d = nullptr, s_scatter = nullptr;
     char* stage_out = nullptr;
     char* stage_in = nullptr;
     int64_t slot_bytes = 0;
@@ -157,19 +157,17 @@ struct ps_ctx {
     bool out_used[kSlots]{}, in_used[kSlots]{};
     uint64_t out_next = 0, in_next = 0;
     std::vector<cudaEvent_t> ev_in;  // per layer
-    cudaEvent_t e_mark = nullptr, e_mark2 = nullptr, e_ids = nullptr, e_fork = nullptr, e_join = nullptr;
-    bool ids_fenced = false;
-    int32_t* h_ids = nullptr;
-    int32_t* d_ids = nullptr;
+    cudaEvent_t e_mark = nullptr, e_mark2 = nullptr;
     int32_t* status = nullptr;  // mapped pinned word written by kernels on a bad block id
     int32_t* d_status = nullptr;
     Tracker t_d2h, t_scatter, t_compute;
-    Arena a_gather, a_meta;
+    Arena a_gather, a_meta, a_ids;
     std::vector<cudaEvent_t> ev_pool, ev_pool_timing;
     std::deque<std::pair<uint64_t, std::pair<int64_t, int64_t>>> img_release;  // in_ticket -> (off, bytes)
     std::vector<int64_t> gated_reqs;
     float* partials = nullptr;
     int32_t* d_sched = nullptr;  // chunk counters of the tensor-core kernel: {next, done} per lane
+    int32_t* d_row_done = nullptr;  // its split-KV arrival counters: max_batch x num_kv_heads
     int32_t max_parts = 0;
     int attn_kernel = 1;
     int32_t num_sms = 1;
@@ -539,7 +537,8 @@ int32_t choose_split(const ps_ctx* ctx, int64_t total_tokens) {
 
 // Builds (or reuses) the device metadata for a decode batch.  Row b of the metadata is position b of
 // the caller's request array (q / out rows are addressed by that position); rows with active[b] == 0
-// get no work item.  gated[b] != 0 puts the row's items behind the reload-event wait.
+// get no work item.  gated[b] != 0 marks rows whose reload is still landing (the launch then waits on
+// the layer's reload event).
 int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::vector<char>& active,
                       const std::vector<char>& gated) {
     BatchMeta& m = ctx->meta;
@@ -562,11 +561,11 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     bool any_multi = false, lane_multi[2] = {false, false};
     const bool mma = ctx->attn_kernel == PS_ATTN_MMA;
     const int32_t split = mma ? 0 : choose_split(ctx, total_tokens);
-    for (int pass = 0; pass < 2; ++pass) {  // lane 0: rows that need no wait; lane 1: gated rows
+    for (int pass = 0; pass < 1; ++pass) {  // a single work list (lane 0) holds every active row
         if (!mma) {
             // SIMT kernel: one CTA per (item, KV head); items are fixed-size token ranges of a row
             for (int32_t b = 0; b < B; ++b) {
-                if (!active[b] || (gated[b] ? 1 : 0) != pass) continue;
+                if (!active[b]) continue;
                 const Req& r = ctx->reqs[reqs[b]];
                 const int32_t n = std::max(1, (r.n_tokens + split - 1) / split);
                 row_first[b] = parts;
@@ -584,7 +583,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
                     items.push_back(it);
                 }
                 parts += n;
-                if (pass == 1) ++n_gated_rows;
+                if (gated[b]) ++n_gated_rows;
             }
         } else {
             // Tensor-core kernel: the lane's 16-token tiles form one sequence.  Its head is cut into
@@ -597,7 +596,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
             int64_t total_tiles = 0;
             int32_t lane_rows = 0;
             for (int32_t b = 0; b < B; ++b)
-                if (active[b] && (gated[b] ? 1 : 0) == pass) {
+                if (active[b]) {
                     total_tiles += (ctx->reqs[reqs[b]].n_tokens + kTile - 1) / kTile;
                     ++lane_rows;
                 }
@@ -622,7 +621,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
                 filled = 0;
             };
             for (int32_t b = 0; b < B; ++b) {
-                if (!active[b] || (gated[b] ? 1 : 0) != pass) continue;
+                if (!active[b]) continue;
                 const Req& r = ctx->reqs[reqs[b]];
                 const int64_t tiles_b = (r.n_tokens + kTile - 1) / kTile;
                 const size_t first_item = items.size();
@@ -667,12 +666,12 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
                 parts += n;
                 any_multi |= n > 1;
                 lane_multi[pass] |= n > 1;
-                if (pass == 1) ++n_gated_rows;
+                if (gated[b]) ++n_gated_rows;
             }
             if (n_cta > 0 && !in_dyn) close_static();
         }
-        if (pass == 0) n_ungated = (int32_t)items.size();
     }
+    n_ungated = (int32_t)items.size();
     if (parts > ctx->max_parts) return ctx->fail(PS_ERR_INVALID, "split-KV scratch too small for this batch");
 
     const size_t sz_tables = (size_t)round_up((int64_t)B * stride * 4, 256);
@@ -701,7 +700,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     memcpy(h + sz_tables + 2 * sz_vec, row_parts.data(), (size_t)B * 4);
     {
         int32_t* lane = (int32_t*)(h + sz_tables + 3 * sz_vec);
-        for (int32_t b = 0; b < B; ++b) lane[b] = gated[b] ? 1 : 0;
+        for (int32_t b = 0; b < B; ++b) lane[b] = 0;
     }
     if (!items.empty()) memcpy(h + sz_tables + 4 * sz_vec, items.data(), items.size() * sizeof(ps::AttnItem));
     {
@@ -749,49 +748,25 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     return PS_OK;
 }
 
-// Launches one layer of attention for the prepared batch.  wait_event: the layer's reload event for
-// the gated rows (nullptr = no wait).  lanes == false: everything on the compute stream (main rows,
-// wait, gated rows, one merge).  lanes == true: the gated rows run on the reload-lane stream behind
-// the wait, with their own merge, so the main rows of the next layer never queue behind them.
+// Launches one layer of attention for the prepared batch on the compute stream.  wait_event: the
+// layer's reload event when rows of the batch are still being reloaded (Appendix B: the compute stream
+// synchronises on a layer chunk's event only before it executes that chunk); nullptr = no wait.
 int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, float* lse, cudaEvent_t wait_event,
-                          bool lanes, int32_t* n_launched) {
+                          int32_t* n_launched) {
     BatchMeta& m = ctx->meta;
+    if (m.n_items == 0) return PS_OK;
     ps::AttnShape sh{ctx->cfg.num_kv_heads, ctx->cfg.num_q_heads, ctx->cfg.head_dim, ctx->cfg.block_size,
                      ctx->cfg.num_gpu_blocks};
-    const int64_t bytes = m.kv_bytes_per_layer;
-    const int64_t ungated_bytes = m.n_items ? bytes * m.n_ungated_items / m.n_items : 0;
-    const bool have_gated = m.n_items > m.n_ungated_items;
-    if (m.n_ungated_items > 0) {
-        ProfScope prof(ctx, kProfAttn, ctx->compute, ungated_bytes, layer);
+    if (wait_event) CK(cudaStreamWaitEvent(ctx->compute, wait_event, 0));
+    {
+        ProfScope prof(ctx, kProfAttn, ctx->compute, m.kv_bytes_per_layer, wait_event ? 1000 + layer : layer);
         CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev, 0,
-                                  ctx->partials, ctx->d_sched, ctx->d_status, ctx->compute));
+                                  ctx->partials, ctx->d_sched, ctx->d_row_done, ctx->d_status, ctx->compute));
         ctx->launches++;
         ++*n_launched;
     }
-    if (lanes && have_gated && m.lane_multi[0]) {
-        ProfScope prof(ctx, kProfMerge, ctx->compute, 0, layer);
-        CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials, 0, ctx->compute));
-        ctx->launches++;
-        ++*n_launched;
-    }
-    if (have_gated) {
-        cudaStream_t gs = lanes ? ctx->s_lane : ctx->compute;
-        if (wait_event) CK(cudaStreamWaitEvent(gs, wait_event, 0));
-        {
-            ProfScope prof(ctx, kProfAttn, gs, bytes - ungated_bytes, 1000 + layer);
-            CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev,
-                                      1, ctx->partials, ctx->d_sched, ctx->d_status, gs));
-            ctx->launches++;
-            ++*n_launched;
-        }
-        if (lanes && m.lane_multi[1]) {
-            ProfScope prof(ctx, kProfMerge, gs, 0, 1000 + layer);
-            CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials, 1, gs));
-            ctx->launches++;
-            ++*n_launched;
-        }
-    }
-    if (!(lanes && have_gated) && m.any_multi) {
+    // the tensor-core kernel combines split rows itself; the CUDA-core kernel needs the merge pass
+    if (ctx->attn_kernel != PS_ATTN_MMA && m.any_multi) {
         ProfScope prof(ctx, kProfMerge, ctx->compute, 0, layer);
         CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials, -1, ctx->compute));
         ctx->launches++;
@@ -802,13 +777,13 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
 
 void destroy_ctx(ps_ctx* ctx) {
     if (!ctx->bk) {
-        for (cudaStream_t s : {ctx->s_gather, ctx->s_d2h, ctx->s_h2d, ctx->s_scatter, ctx->s_lane})
+        for (cudaStream_t s : {ctx->s_gather, ctx->s_d2h, ctx->s_h2d, ctx->s_scatter})
             if (s) cudaStreamDestroy(s);
         for (int i = 0; i < kSlots; ++i)
             for (cudaEvent_t e : {ctx->e_gathered[i], ctx->e_drained[i], ctx->e_loaded[i], ctx->e_scattered[i]})
                 if (e) cudaEventDestroy(e);
         for (cudaEvent_t e : ctx->ev_in) cudaEventDestroy(e);
-        for (cudaEvent_t e : {ctx->e_mark, ctx->e_mark2, ctx->e_ids, ctx->e_fork, ctx->e_join, ctx->trace_base})
+        for (cudaEvent_t e : {ctx->e_mark, ctx->e_mark2, ctx->trace_base})
             if (e) cudaEventDestroy(e);
         for (auto& t : {&ctx->t_d2h, &ctx->t_scatter, &ctx->t_compute})
             for (auto& p : t->pending) cudaEventDestroy(p.second);
@@ -820,14 +795,14 @@ void destroy_ctx(ps_ctx* ctx) {
         }
         arena_free(ctx->a_gather);
         arena_free(ctx->a_meta);
+        arena_free(ctx->a_ids);
         if (ctx->stage_out) cudaFree(ctx->stage_out);
         if (ctx->stage_in) cudaFree(ctx->stage_in);
         if (ctx->d_kpools) cudaFree(ctx->d_kpools);
         if (ctx->d_vpools) cudaFree(ctx->d_vpools);
         if (ctx->partials) cudaFree(ctx->partials);
         if (ctx->d_sched) cudaFree(ctx->d_sched);
-        if (ctx->d_ids) cudaFree(ctx->d_ids);
-        if (ctx->h_ids) cudaFreeHost(ctx->h_ids);
+        if (ctx->d_row_done) cudaFree(ctx->d_row_done);
         if (ctx->status) cudaFreeHost(ctx->status);
         if (ctx->own_host_pool && ctx->host_pool) cudaFreeHost(ctx->host_pool);
         cudaGetLastError();
@@ -952,8 +927,6 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     CKC(cudaStreamCreateWithPriority(&ctx->s_d2h, cudaStreamNonBlocking, prio_hi));
     CKC(cudaStreamCreateWithPriority(&ctx->s_h2d, cudaStreamNonBlocking, prio_hi));
     CKC(cudaStreamCreateWithPriority(&ctx->s_scatter, cudaStreamNonBlocking, prio_hi));
-    // the reload lane: attention of requests whose reload is landing in this step (same priority as compute)
-    CKC(cudaStreamCreateWithPriority(&ctx->s_lane, cudaStreamNonBlocking, prio_lo));
     ctx->t_d2h.s = ctx->s_d2h;
     ctx->t_scatter.s = ctx->s_scatter;
     ctx->t_compute.s = ctx->compute;
@@ -972,20 +945,16 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     for (int l = 0; l < L; ++l) CKC(cudaEventCreateWithFlags(&ctx->ev_in[(size_t)l], cudaEventDisableTiming));
     CKC(cudaEventCreateWithFlags(&ctx->e_mark, cudaEventDisableTiming));
     CKC(cudaEventCreateWithFlags(&ctx->e_mark2, cudaEventDisableTiming));
-    CKC(cudaEventCreateWithFlags(&ctx->e_ids, cudaEventDisableTiming));
-    CKC(cudaEventCreateWithFlags(&ctx->e_fork, cudaEventDisableTiming));
-    CKC(cudaEventCreateWithFlags(&ctx->e_join, cudaEventDisableTiming));
     CKC(cudaHostAlloc((void**)&ctx->status, 64, cudaHostAllocMapped));
     memset(ctx->status, 0, 64);
     CKC(cudaHostGetDevicePointer((void**)&ctx->d_status, ctx->status, 0));
-    CKC(cudaHostAlloc((void**)&ctx->h_ids, sizeof(int32_t) * (size_t)cfg->num_gpu_blocks, cudaHostAllocDefault));
-    CKC(cudaMalloc((void**)&ctx->d_ids, sizeof(int32_t) * (size_t)cfg->num_gpu_blocks));
 
     // descriptor arenas: a table per swap-out; one decode batch per chunk (scatter ids travel as
     // kernel parameters).  Uploads are done by a kernel reading the mapped pinned side, so the copy
     // engines carry bulk KV traffic only.
     const size_t desc_chunk = std::max<size_t>((size_t)cfg->max_blocks_per_req * 4 * 8, 1 << 20);
     CKR(arena_init(ctx, ctx->a_gather, desc_chunk, 4, ctx->s_gather));
+    CKR(arena_init(ctx, ctx->a_ids, (size_t)cfg->num_gpu_blocks * 4, 4, ctx->compute));  // ps_copy_blocks
 
     // split-KV scratch
     ctx->attn_kernel = PS_ATTN_SIMT;
@@ -1018,6 +987,9 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
         CKC(cudaMalloc((void**)&ctx->partials, ps::attn_partial_bytes(sh, ctx->max_parts)));
         CKC(cudaMalloc((void**)&ctx->d_sched, 4 * sizeof(int32_t)));
         CKC(cudaMemset(ctx->d_sched, 0, 4 * sizeof(int32_t)));
+        const size_t done_bytes = (size_t)max_batch * cfg->num_kv_heads * sizeof(int32_t);
+        CKC(cudaMalloc((void**)&ctx->d_row_done, done_bytes));
+        CKC(cudaMemset(ctx->d_row_done, 0, done_bytes));
         const size_t meta_chunk = (size_t)max_batch * cfg->max_blocks_per_req * 4 + (size_t)max_batch * 16 +
                                   (size_t)ctx->max_parts * sizeof(ps::AttnItem) + (size_t)ctx->num_sms * 8 + 8192;
         CKR(arena_init(ctx, ctx->a_meta, meta_chunk, 3, ctx->compute));
@@ -1290,7 +1262,7 @@ int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, flo
     if (rc != PS_OK) return rc;
     int32_t launched = 0;
     return launch_layer_attn(ctx, layer, q, out, lse, ctx->meta.n_gated_rows ? ctx->ev_in[(size_t)layer] : nullptr,
-                             /*lanes=*/false, &launched);
+                             &launched);
 }
 
 int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs, int32_t batch,
@@ -1356,11 +1328,6 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
     if (attn) {
         const int64_t layer_bytes = (int64_t)batch * ctx->cfg.num_q_heads * ctx->cfg.head_dim * 2;
         const bool any_gated = ctx->meta.n_gated_rows > 0;
-        const bool lanes = any_gated && !sync_reload;
-        if (lanes) {  // the reload lane starts where the compute stream stands now (metadata uploaded)
-            CK(cudaEventRecord(ctx->e_fork, ctx->compute));
-            CK(cudaStreamWaitEvent(ctx->s_lane, ctx->e_fork, 0));
-        }
         for (int l = 0; l < L; ++l) {
             if (!sync_reload) {
                 rc = issue_reload_layer(ctx, l, plan);
@@ -1375,12 +1342,8 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
             }
             int32_t launched = 0;
             rc = launch_layer_attn(ctx, l, (const char*)q_all_layers + l * layer_bytes,
-                                   (char*)out_all_layers + l * layer_bytes, nullptr, wait, lanes, &launched);
+                                   (char*)out_all_layers + l * layer_bytes, nullptr, wait, &launched);
             if (rc != PS_OK) return rc;
-        }
-        if (lanes) {  // the step is complete on the compute stream only when the reload lane is
-            CK(cudaEventRecord(ctx->e_join, ctx->s_lane));
-            CK(cudaStreamWaitEvent(ctx->compute, ctx->e_join, 0));
         }
     }
 
@@ -1500,22 +1463,23 @@ int32_t ps_copy_blocks(ps_ctx* ctx, int32_t layer, const int32_t* ids, int32_t n
     if (n_blocks == 0) return PS_OK;
     for (int32_t i = 0; i < n_blocks; ++i)
         if (ids[i] < 0 || ids[i] >= ctx->cfg.num_gpu_blocks) return ctx->fail(PS_ERR_INVALID, "ps_copy_blocks: bad block id");
-    if (ctx->ids_fenced) {
-        CK(cudaEventSynchronize(ctx->e_ids));
-        ctx->ids_fenced = false;
-    }
-    memcpy(ctx->h_ids, ids, (size_t)n_blocks * 4);
-    CK(cudaMemcpyAsync(ctx->d_ids, ctx->h_ids, (size_t)n_blocks * 4, cudaMemcpyHostToDevice, ctx->compute));
-    CK(cudaEventRecord(ctx->e_ids, ctx->compute));
-    ctx->ids_fenced = true;
+    // the ids travel through a descriptor ring on the compute stream: no host wait between calls
+    size_t ioff = 0;
+    int32_t rc = arena_alloc(ctx, ctx->a_ids, (size_t)n_blocks * 4, &ioff);
+    if (rc != PS_OK) return rc;
+    memcpy(ctx->a_ids.h + ioff, ids, (size_t)n_blocks * 4);
+    CK(ps::launch_upload(ctx->a_ids.d + ioff, ctx->a_ids.hd + ioff, (size_t)round_up((int64_t)n_blocks * 4, 16),
+                         ctx->compute));
+    ctx->launches++;
+    const int32_t* d_ids = (const int32_t*)(ctx->a_ids.d + ioff);
     const int64_t bytes = (int64_t)n_blocks * ctx->layer_block_bytes;
     if (direction == 0) {
         ProfScope prof(ctx, kProfGather, ctx->compute, bytes);
-        CK(ps::launch_gather_layer(ctx->kpools[(size_t)layer], ctx->vpools[(size_t)layer], ctx->d_ids, n_blocks, staging,
+        CK(ps::launch_gather_layer(ctx->kpools[(size_t)layer], ctx->vpools[(size_t)layer], d_ids, n_blocks, staging,
                                    ctx->slab_vec, ctx->cfg.num_gpu_blocks, ctx->d_status, ctx->compute));
     } else {
         ProfScope prof(ctx, kProfScatter, ctx->compute, bytes);
-        CK(ps::launch_scatter_layer(ctx->kpools[(size_t)layer], ctx->vpools[(size_t)layer], ctx->d_ids, n_blocks, staging,
+        CK(ps::launch_scatter_layer(ctx->kpools[(size_t)layer], ctx->vpools[(size_t)layer], d_ids, n_blocks, staging,
                                     ctx->slab_vec, ctx->cfg.num_gpu_blocks, ctx->d_status, ctx->compute));
     }
     ctx->launches++;
