@@ -1084,7 +1084,12 @@ int32_t ps_swap_out(ps_ctx* ctx, int64_t req) {
     if (r.state != PS_REQ_RESIDENT) return ctx->fail(PS_ERR_STATE, "ps_swap_out: request is not resident");
     const int64_t n_blk = (int64_t)r.table.size();
     const int64_t bytes = n_blk * ctx->block_bytes;
-    const int64_t off = ctx->hpool.alloc(bytes);
+    int64_t off = ctx->hpool.alloc(bytes);
+    if (off < 0) {  // images of reloads that have landed since the last poll may still be held
+        int32_t rc = do_poll(ctx, nullptr);
+        if (rc != PS_OK) return rc;
+        off = ctx->hpool.alloc(bytes);
+    }
     if (off < 0) return ctx->fail(PS_ERR_HOST_NOMEM, "ps_swap_out: host pool cannot hold the image");
 
     if (!ctx->bk && n_blk > 0) {
