@@ -452,21 +452,18 @@ def kernel_rates(torch, B, lib, sh, nb, n_blocks=2048, iters=20):
 
 def run_gpu(args):
     import torch
-    import torch.distributed as dist
 
     from paper_2512_12928_b200 import binding as B
     from paper_2512_12928_b200 import build as ps_build
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    from paper_2512_12928_b200 import replicas
+
+    rank, world, local_rank = replicas.env()
     torch.cuda.set_device(local_rank)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    group = replicas.Group("nccl", torch.device("cuda", local_rank))
     if rank == 0:
         ps_build.build()
-    if world > 1:
-        dist.barrier()
+    group.barrier()
     B.load()
     hbm_peak, peak_kind = read_peaks()
 
@@ -478,7 +475,8 @@ def run_gpu(args):
     sh = w.shape
     w3 = wl.overlap()
     nb_alloc = max(sh.num_gpu_blocks, w3.shape.num_gpu_blocks) if not args.no_overlap else sh.num_gpu_blocks
-    K, V = fill_pools(torch, sh.num_layers, nb_alloc, sh.block_size, sh.num_kv_heads, sh.head_dim, w.seed + 1000 * rank)
+    K, V = fill_pools(torch, sh.num_layers, nb_alloc, sh.block_size, sh.num_kv_heads, sh.head_dim,
+                      replicas.replica_seed(w.seed, rank))
     torch.cuda.synchronize()
 
     victim_bytes = sum(sh.blocks_for(w.ctx_lens[r]) for r in w.victims) * sh.block_bytes
@@ -508,25 +506,20 @@ def run_gpu(args):
     launches0 = lib.launch_count()
     sampler = ClockSampler(local_rank)
     sampler.start()
-    if world > 1:
-        dist.barrier()
+    group.barrier()
     torch.cuda.synchronize()
     t_wall0 = time.perf_counter()
     recs = [swap_workload_step(torch, B, lib, w, q, out, q_res, out_res, budget) for _ in range(args.steps)]
     torch.cuda.synchronize()
-    if world > 1:
-        dist.barrier()
+    group.barrier()
     wall_ms = (time.perf_counter() - t_wall0) * 1e3
     launches = lib.launch_count() - launches0
 
     out_ms = sum(r["out_ms"] for r in recs)
     in_ms = sum(r["in_ms"] for r in recs)
     total_ms = out_ms + in_ms
-    if world > 1:
-        t = torch.tensor([total_ms, out_ms, in_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, out_ms, in_ms = [float(x) for x in t.tolist()]
-    moved = 2 * victim_bytes * args.steps * world
+    total_ms, out_ms, in_ms = group.max_over_ranks([total_ms, out_ms, in_ms])
+    (moved,) = group.sum_over_ranks([2 * victim_bytes * args.steps])
     value = moved / total_ms / 1e6
 
     # ---- the dominant kernel, live, in the launch configuration of the step: decode-only steps of the
@@ -544,10 +537,7 @@ def run_gpu(args):
                 for _ in range(max(1, min(args.steps, 2)))]
     e2e_ms = sum(r["out_ms"] + r["in_ms"] for r in e2e_recs)
     e2e_steps = sum(r["steps_out"] + r["steps_in"] for r in e2e_recs) / len(e2e_recs)
-    if world > 1:
-        t = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    (e2e_ms,) = group.max_over_ranks([e2e_ms])
     q_bytes = q.numel() * 2
     e2e = {"value": 2 * victim_bytes * len(e2e_recs) * world / e2e_ms / 1e6, "unit": UNIT,
            "h2d_bytes_per_step": int(victim_bytes + e2e_steps * q_bytes),
@@ -617,9 +607,7 @@ def run_gpu(args):
     if rank == 0 and world == 1:
         del K, V
         result["cpu_baseline"] = time_oracle(args.cpu_seconds)
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    group.close()
     if rank == 0:
         print(json.dumps(result))
 

@@ -23,7 +23,7 @@ PS_OK, PS_ERR_INVALID, PS_ERR_NOMEM, PS_ERR_HOST_NOMEM = 0, -1, -2, -3
 PS_ERR_STATE, PS_ERR_BUSY, PS_ERR_TIMEOUT, PS_ERR_CUDA, PS_ERR_BOUNDS = -4, -5, -6, -7, -8
 PS_REQ_NONE, PS_REQ_RESIDENT, PS_REQ_SWAPPING_OUT, PS_REQ_HOST, PS_REQ_SWAPPING_IN = 0, 1, 2, 3, 4
 PS_FLAG_BOOKKEEPING_ONLY, PS_FLAG_PROFILE, PS_FLAG_SYNC_RELOAD = 1, 2, 4
-PS_ATTN_AUTO, PS_ATTN_SIMT, PS_ATTN_MMA = 0, 1, 2
+PS_ATTN_AUTO, PS_ATTN_SIMT, PS_ATTN_MMA, PS_ATTN_MMA_ROWS = 0, 1, 2, 3
 
 EXPORTS = [
     "ps_create", "ps_destroy", "ps_last_error", "ps_kv_alloc", "ps_kv_free", "ps_block_table",

@@ -11,7 +11,9 @@
 // The kernel is HBM-bound (G flop per KV byte), so the SIMT kernel below spends its effort on
 // 16-byte coalesced loads with many of them in flight; softmax statistics are reduced with warp
 // shuffles inside the group of lanes that shares a token.
+#include <cuda.h>
 #include <cuda_bf16.h>
+#include <cstring>
 #include <math_constants.h>
 
 #include "ps_internal.h"
@@ -295,7 +297,16 @@ constexpr int kMmaPartStride = kMmaD + 4;                 // floats per (part, q
 constexpr int kSpinLimit = 1 << 22;
 constexpr int kFlagFirst = 1, kFlagLast = 2, kFlagEnd = 4;
 
-constexpr int mma_smem_bytes(int) { return kMmaRingBytes + kMmaCtrlBytes; }
+// Tensor-map mode: a K (or V) tile is one 32 KiB box copy, laid out [16 chunks of 128 B][16 tokens][128 B] with
+// the 128-byte swizzle (16-byte units XORed with the token index mod 8), so no row padding is needed.
+constexpr int kTmaTileBytes = kMmaTileTokens * kMmaRowBytes;   // 32768
+constexpr int kTmaStageBytes = 2 * kTmaTileBytes;              // 65536
+constexpr int kTmaRingBytes = kMmaStages * kTmaStageBytes;
+constexpr int kTmaAlign = 1024;                                // the swizzle pattern repeats every 1 KiB
+
+constexpr int mma_smem_bytes(bool tma) {
+    return tma ? kTmaRingBytes + kTmaAlign + kMmaCtrlBytes : kMmaRingBytes + kMmaCtrlBytes;
+}
 
 struct StageDesc {  // published by the producer next to every ring stage
     int32_t item;   // index into batch.items
@@ -353,6 +364,15 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
     asm volatile(
         "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(dst),
         "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+        : "memory");
+}
+// One box of a rank-3 tensor map (element, token row, 128-byte chunk) into shared memory.
+__device__ __forceinline__ void tensor_g2s(uint32_t dst, const void* map, int32_t token_row, uint32_t bar,
+                                           uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3, %4}], [%5], %6;" ::"r"(dst),
+        "l"(map), "r"(0), "r"(token_row), "r"(0), "r"(bar), "l"(policy)
         : "memory");
 }
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
@@ -460,18 +480,25 @@ __device__ __forceinline__ void merge_row(int b, int h, int lane, const AttnBatc
     if (lane == 0) row_done[b * kMmaHkv + h] = 0;  // every part has arrived: re-arm for the next launch
 }
 
-template <int G>
+template <int G, bool kTma>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloat16* __restrict__ vpool,
+                       const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
                        const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
                        AttnBatch batch, int32_t sched_lane, int32_t block_size, int32_t block_shift,
                        int32_t num_blocks, float* __restrict__ partials, int32_t* __restrict__ sched,
                        int32_t* __restrict__ row_done, float scale_log2e, int32_t* status) {
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
     constexpr int Hq = kMmaHkv * G;
-    const uint32_t ring = smem_u32(smem);
-    unsigned char* ctrl = smem + kMmaRingBytes;
-    const uint32_t bar_full = ring + kMmaRingBytes;         // [kMmaStages]
+    constexpr int kStageBytes = kTma ? kTmaStageBytes : kMmaStageBytes;
+    constexpr int kRingBytes = kTma ? kTmaRingBytes : kMmaRingBytes;
+    constexpr int kVOff = kTma ? kTmaTileBytes : kMmaSlabBytes;   // V tile inside a stage
+    // the swizzled layout needs the ring on a 1 KiB boundary of the shared address space
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t ring = kTma ? (raw + kTmaAlign - 1) & ~(uint32_t)(kTmaAlign - 1) : raw;
+    unsigned char* smem = smem_raw + (ring - raw);
+    unsigned char* ctrl = smem + kRingBytes;
+    const uint32_t bar_full = ring + kRingBytes;            // [kMmaStages]
     const uint32_t bar_empty = bar_full + 8 * kMmaStages;   // [kMmaStages]
     // 48 bytes of barriers, then the stage descriptors and the abort word
     volatile StageDesc* sdesc = reinterpret_cast<volatile StageDesc*>(ctrl + 64);
@@ -487,9 +514,11 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
         *abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    for (int i = threadIdx.x; i < kMmaRingBytes / 16; i += kMmaThreads)
-        reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy zeroes before async-proxy writes
+    if (!kTma) {  // row copies skip the rows past a context's end: a stale row must at least be finite
+        for (int i = threadIdx.x; i < kRingBytes / 16; i += kMmaThreads)
+            reinterpret_cast<uint4*>(smem)[i] = make_uint4(0, 0, 0, 0);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy zeroes before async-proxy writes
+    }
     __syncthreads();
 
     const int32_t* cta_begin = batch.cta_begin[sched_lane];
@@ -518,20 +547,31 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             const AttnItem item = batch.items[it];
             const int32_t* table = batch.block_tables + (int64_t)item.b * batch.table_stride;
             const int ntiles = max(1, (item.t_end - item.t_begin + kMmaTileTokens - 1) / kMmaTileTokens);
+            // Block ids are read 32 at a time, one per lane, a window ahead of their use: the table read
+            // never sits between a freed stage and the copies that refill it.
+            const int last_blk = (max(item.t_end, 1) - 1) / block_size;
+            int win = block_shift >= 0 ? (item.t_begin >> block_shift) : (item.t_begin / block_size);
+            int ids = win + lane <= last_blk ? __ldg(table + win + lane) : 0;
+            int ids_next = win + 32 + lane <= last_blk ? __ldg(table + win + 32 + lane) : 0;
             for (int ti = 0; ti < ntiles; ++ti, ++n) {
                 const int s = n % kMmaStages;
-                if (n >= kMmaStages) ok = mbar_wait(bar_empty + 8 * s, ((n / kMmaStages) - 1) & 1, abort_word, status);
-                if (!ok) break;
                 const int t0 = item.t_begin + ti * kMmaTileTokens;
                 const int rows = max(0, min(kMmaTileTokens, item.t_end - t0));
+                const int blk = block_shift >= 0 ? (t0 >> block_shift) : (t0 / block_size);
+                if (blk >= win + 32) {  // tiles advance by at most one block: the next window is the one ahead
+                    win += 32;
+                    ids = ids_next;
+                    ids_next = win + 32 + lane <= last_blk ? __ldg(table + win + 32 + lane) : 0;
+                }
+                if (n >= kMmaStages) ok = mbar_wait(bar_empty + 8 * s, ((n / kMmaStages) - 1) & 1, abort_word, status);
+                if (!ok) break;
                 const uint32_t full = bar_full + 8 * s;
-                int id = 0, slot = 0;
+                int id = __shfl_sync(0xffffffffu, ids, (blk - win) & 31);
+                int slot = 0;
                 bool copy = rows > 0;
                 if (copy) {
-                    const int blk = block_shift >= 0 ? (t0 >> block_shift) : (t0 / block_size);
                     slot = t0 - blk * block_size;
-                    id = table[blk];
-                    if ((unsigned)id >= (unsigned)num_blocks) {  // the stage keeps its old, finite contents
+                    if ((unsigned)id >= (unsigned)num_blocks) {  // nothing is copied and the tile is skipped
                         *(volatile int32_t*)status = 2;
                         copy = false;
                     }
@@ -539,20 +579,28 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                 if (lane == 0) {
                     sdesc[s].item = it;
                     sdesc[s].t0 = t0;
-                    sdesc[s].rows = rows;
+                    sdesc[s].rows = copy ? rows : 0;
                     sdesc[s].flags = (ti == 0 ? kFlagFirst : 0) | (ti == ntiles - 1 ? kFlagLast : 0);
                     if (copy)
-                        mbar_expect_tx(full, (uint32_t)rows * 2u * kMmaRowBytes);
+                        mbar_expect_tx(full, kTma ? (uint32_t)kTmaStageBytes : (uint32_t)rows * 2u * kMmaRowBytes);
                     else
                         mbar_arrive(full);
                 }
                 __syncwarp();  // descriptor and expected byte count are posted before any copy can complete
                 if (copy) {
-                    const int r = lane & 15;
-                    if (r < rows) {
-                        const int64_t off = ((int64_t)id * block_size + slot + r) * (kMmaRowBytes / 2);  // elements
-                        const uint32_t dst = ring + s * kMmaStageBytes + (lane < 16 ? 0 : kMmaSlabBytes) + r * kMmaPitch;
-                        bulk_g2s(dst, (lane < 16 ? kpool : vpool) + off, kMmaRowBytes, full, kv_policy);
+                    if (kTma) {
+                        // whole boxes of 16 token rows: the tile lies inside one block, so rows past the context's
+                        // end are in bounds (the consumers clear them in V and mask them in the scores)
+                        if (lane < 2)
+                            tensor_g2s(ring + s * kStageBytes + lane * kVOff, lane == 0 ? &kmap : &vmap,
+                                       id * block_size + slot, full, kv_policy);
+                    } else {
+                        const int r = lane & 15;
+                        if (r < rows) {
+                            const int64_t off = ((int64_t)id * block_size + slot + r) * (kMmaRowBytes / 2);  // elements
+                            const uint32_t dst = ring + s * kStageBytes + (lane < 16 ? 0 : kVOff) + r * kMmaPitch;
+                            bulk_g2s(dst, (lane < 16 ? kpool : vpool) + off, kMmaRowBytes, full, kv_policy);
+                        }
                     }
                 }
             }
@@ -582,11 +630,22 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
         const int ld_row = lane & 7;
         const int ld_mat = lane >> 3;
         // K, no transpose: matrices {tok 0-7, d lo}, {tok 0-7, d hi}, {tok 8-15, d lo}, {tok 8-15, d hi}
-        const uint32_t k_lane_off =
-            (uint32_t)((ld_row + ((ld_mat & 2) ? 8 : 0)) * kMmaPitch + h * 256 + ((ld_mat & 1) ? 16 : 0));
         // V, transposed on load: matrices {tok 0-7, d lo}, {tok 8-15, d lo}, {tok 0-7, d hi}, {tok 8-15, d hi}
-        const uint32_t v_lane_off = (uint32_t)(kMmaSlabBytes + (ld_row + ((ld_mat & 1) ? 8 : 0)) * kMmaPitch + h * 256 +
-                                               ((ld_mat & 2) ? 16 : 0));
+        const int k_tok = ld_row + ((ld_mat & 2) ? 8 : 0), k_half = ld_mat & 1;
+        const int v_tok = ld_row + ((ld_mat & 1) ? 8 : 0), v_half = (ld_mat & 2) ? 1 : 0;
+        // Row-copy mode: token rows at a 2064-byte pitch, head h at byte 256 h.  Tensor-map mode: head h is the
+        // 128-byte chunks 2h and 2h + 1, each [16 tokens][128 B]; the 16-byte unit u of a token row sits at
+        // unit u ^ (token mod 8).  k_x[u] / v_x[u]: byte offset of the lane's unit for dims 32 u .. 32 u + 15.
+        const uint32_t k_lane_off = kTma ? (uint32_t)(2 * h * 2048 + k_tok * 128)
+                                         : (uint32_t)(k_tok * kMmaPitch + h * 256 + k_half * 16);
+        const uint32_t v_lane_off = kTma ? (uint32_t)(kVOff + 2 * h * 2048 + v_tok * 128)
+                                         : (uint32_t)(kVOff + v_tok * kMmaPitch + h * 256 + v_half * 16);
+        uint32_t k_x[4], v_x[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            k_x[u] = kTma ? (uint32_t)(((2 * u + k_half) ^ ld_row) << 4) : (uint32_t)(64 * u);
+            v_x[u] = kTma ? (uint32_t)(((2 * u + v_half) ^ ld_row) << 4) : (uint32_t)(64 * u);
+        }
         uint32_t qa[8][2];
         float o[16][2];
         float m_run = kNegBig, l_run = 0.f;
@@ -623,13 +682,24 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                 l_run = 0.f;
             }
             if (rows > 0) {
-                const uint32_t base = ring + s * kMmaStageBytes;
+                const uint32_t base = ring + s * kStageBytes;
+                if (kTma && rows < kMmaTileTokens) {
+                    // the box brought whole token rows past the context's end: clear this head's part of them in V
+                    // (a zero weight times a non-finite leftover would poison the row's output)
+                    if (lane < 16)
+                        for (int r = rows; r < kMmaTileTokens; ++r)
+                            *reinterpret_cast<uint4*>(smem + s * kStageBytes + kVOff + (2 * h + (lane >> 3)) * 2048 + r * 128 +
+                                                      (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // before the stage is refilled
+                    __syncwarp();
+                }
                 // scores of row g: s0 -> tokens 2t, 2t+1; s1 -> tokens 8+2t, 9+2t
                 float s00 = 0.f, s01 = 0.f, s10 = 0.f, s11 = 0.f;
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     uint32_t b0, b1, b2, b3;
-                    ldsm_x4(base + k_lane_off + 32 * j, b0, b1, b2, b3);
+                    ldsm_x4(base + k_lane_off + (kTma ? (j >> 2) * 2048 : (j >> 2) * 128) + (kTma ? k_x[j & 3] : 32 * (j & 3)),
+                            b0, b1, b2, b3);
                     mma_k16(s00, s01, qa[j][0], qa[j][1], b0, b1, s00, s01);
                     mma_k16(s10, s11, qa[j][0], qa[j][1], b2, b3, s10, s11);
                 }
@@ -656,7 +726,8 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {
                     uint32_t b0, b1, b2, b3;
-                    ldsm_x4_t(base + v_lane_off + 32 * c, b0, b1, b2, b3);
+                    ldsm_x4_t(base + v_lane_off + (kTma ? (c >> 2) * 2048 : (c >> 2) * 128) + (kTma ? v_x[c & 3] : 32 * (c & 3)),
+                              b0, b1, b2, b3);
                     mma_k16(o[2 * c][0], o[2 * c][1], pa0, pa2, b0, b1, o[2 * c][0] * alpha, o[2 * c][1] * alpha);
                     mma_k16(o[2 * c + 1][0], o[2 * c + 1][1], pa0, pa2, b2, b3, o[2 * c + 1][0] * alpha,
                             o[2 * c + 1][1] * alpha);
@@ -718,13 +789,27 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
 }
 
 template <int G>
-cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool, const void* q, void* out, float* lse,
-                       const AttnBatch& batch, int32_t lane, float* partials, int32_t* sched, int32_t* row_done,
-                       int32_t* d_status, cudaStream_t stream) {
+cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool, const AttnTensorMaps* maps, const void* q,
+                       void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials, int32_t* sched,
+                       int32_t* row_done, int32_t* d_status, cudaStream_t stream) {
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)kMmaD);
-    decode_attn_mma_kernel<G><<<(unsigned)batch.n_cta[lane], kMmaThreads, mma_smem_bytes(G), stream>>>(
-        (const __nv_bfloat16*)kpool, (const __nv_bfloat16*)vpool, (const __nv_bfloat16*)q, (__nv_bfloat16*)out, lse, batch,
-        lane, sh.block_size, shift_of(sh.block_size), sh.num_blocks, partials, sched, row_done, scale_log2e, d_status);
+    static_assert(sizeof(CUtensorMap) == sizeof(maps->k), "AttnTensorMaps must hold driver tensor maps");
+    if (maps != nullptr) {
+        CUtensorMap km, vm;
+        memcpy(&km, maps->k, sizeof km);
+        memcpy(&vm, maps->v, sizeof vm);
+        decode_attn_mma_kernel<G, true><<<(unsigned)batch.n_cta[lane], kMmaThreads, mma_smem_bytes(true), stream>>>(
+            (const __nv_bfloat16*)kpool, (const __nv_bfloat16*)vpool, km, vm, (const __nv_bfloat16*)q, (__nv_bfloat16*)out,
+            lse, batch, lane, sh.block_size, shift_of(sh.block_size), sh.num_blocks, partials, sched, row_done,
+            scale_log2e, d_status);
+    } else {
+        CUtensorMap none;
+        memset(&none, 0, sizeof none);
+        decode_attn_mma_kernel<G, false><<<(unsigned)batch.n_cta[lane], kMmaThreads, mma_smem_bytes(false), stream>>>(
+            (const __nv_bfloat16*)kpool, (const __nv_bfloat16*)vpool, none, none, (const __nv_bfloat16*)q,
+            (__nv_bfloat16*)out, lse, batch, lane, sh.block_size, shift_of(sh.block_size), sh.num_blocks, partials, sched,
+            row_done, scale_log2e, d_status);
+    }
     return cudaGetLastError();
 }
 
@@ -742,18 +827,56 @@ bool attn_mma_supported(const AttnShape& sh) {
 
 cudaError_t attn_init() {
     cudaError_t e;
-#define PS_MMA_ATTR(GG)                                                                                    \
-    e = cudaFuncSetAttribute(decode_attn_mma_kernel<GG>, cudaFuncAttributeMaxDynamicSharedMemorySize, \
-                             mma_smem_bytes(GG));                                                          \
+#define PS_MMA_ATTR(GG)                                                                                           \
+    e = cudaFuncSetAttribute(decode_attn_mma_kernel<GG, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
+                             mma_smem_bytes(false));                                                              \
+    if (e != cudaSuccess) return e;                                                                               \
+    e = cudaFuncSetAttribute(decode_attn_mma_kernel<GG, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
+                             mma_smem_bytes(true));                                                               \
     if (e != cudaSuccess) return e;
     PS_MMA_ATTR(1) PS_MMA_ATTR(2) PS_MMA_ATTR(4) PS_MMA_ATTR(8)
 #undef PS_MMA_ATTR
     return cudaSuccess;
 }
 
-cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool, const void* q,
-                               void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials,
-                               int32_t* sched, int32_t* row_done, int32_t* d_status, cudaStream_t stream) {
+// Tensor maps over one layer's pools, seen as rank-3 tensors (64 elements = 128 bytes, token row, 128-byte chunk
+// of the row): strides 2 KiB per token row and 128 bytes per chunk, box 64 x 16 token rows x 16 chunks, 128-byte
+// swizzle.  The driver entry point is looked up at run time (the library does not link against the driver).
+cudaError_t attn_make_tensor_maps(const AttnShape& sh, const void* kpool, const void* vpool, AttnTensorMaps* out) {
+    if (!attn_mma_supported(sh)) return cudaErrorNotSupported;
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                 const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                 CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    static EncodeFn encode = nullptr;
+    if (encode == nullptr) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+        if (e != cudaSuccess) return e;
+        if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
+        encode = (EncodeFn)fn;
+    }
+    const cuuint64_t dims[3] = {64, (cuuint64_t)sh.num_blocks * (cuuint64_t)sh.block_size, (cuuint64_t)(kMmaRowBytes / 128)};
+    const cuuint64_t strides[2] = {(cuuint64_t)kMmaRowBytes, 128};   // bytes: token row, then chunk of the row
+    const cuuint32_t box[3] = {64, (cuuint32_t)kMmaTileTokens, (cuuint32_t)(kMmaRowBytes / 128)};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const void* pools[2] = {kpool, vpool};
+    unsigned char* dst[2] = {out->k, out->v};
+    for (int t = 0; t < 2; ++t) {
+        CUtensorMap m;
+        const CUresult r = encode(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(pools[t]), dims, strides, box,
+                                  estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) return cudaErrorInvalidValue;
+        memcpy(dst[t], &m, sizeof m);
+    }
+    return cudaSuccess;
+}
+
+cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool,
+                               const AttnTensorMaps* maps, const void* q, void* out, float* lse, const AttnBatch& batch,
+                               int32_t lane, float* partials, int32_t* sched, int32_t* row_done, int32_t* d_status,
+                               cudaStream_t stream) {
     if (lane < 0 || lane > 1) return cudaErrorInvalidValue;
     const int item_begin = batch.lane_items[lane];
     const int n_items = batch.lane_items[lane + 1] - item_begin;
@@ -763,13 +886,13 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
         if (!attn_mma_supported(sh) || batch.n_cta[lane] <= 0 || sched == nullptr || row_done == nullptr)
             return cudaErrorNotSupported;
         switch (G) {
-            case 1: return launch_mma<1>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 1: return launch_mma<1>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        stream);
-            case 2: return launch_mma<2>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 2: return launch_mma<2>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        stream);
-            case 4: return launch_mma<4>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 4: return launch_mma<4>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        stream);
-            case 8: return launch_mma<8>(sh, kpool, vpool, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 8: return launch_mma<8>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        stream);
         }
         return cudaErrorNotSupported;

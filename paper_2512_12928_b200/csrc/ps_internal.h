@@ -81,9 +81,17 @@ size_t attn_partial_bytes(const AttnShape& sh, int32_t max_parts);
 // combined inside the kernel by whichever warp delivers the last part, counted in row_done:
 // batch x num_kv_heads int32, zero before the first launch, re-armed by the kernel).  sched and
 // row_done may be null for the SIMT kernel.
-cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool, const void* q,
-                               void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials,
-                               int32_t* sched, int32_t* row_done, int32_t* d_status, cudaStream_t stream);
+// maps: the layer's tensor maps (attn_make_tensor_maps) for the tensor-core kernel, whose tiles then arrive as
+// two 32 KiB box copies; null = one 2 KiB bulk copy per token row.
+struct AttnTensorMaps {
+    alignas(64) unsigned char k[128];
+    alignas(64) unsigned char v[128];
+};
+cudaError_t attn_make_tensor_maps(const AttnShape& sh, const void* kpool, const void* vpool, AttnTensorMaps* out);
+cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool,
+                               const AttnTensorMaps* maps, const void* q, void* out, float* lse, const AttnBatch& batch,
+                               int32_t lane, float* partials, int32_t* sched, int32_t* row_done, int32_t* d_status,
+                               cudaStream_t stream);
 
 // Token granularity at which the tensor-core kernel splits a context.
 constexpr int kMmaTileTokens = 16;

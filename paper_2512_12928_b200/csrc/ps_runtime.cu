@@ -168,6 +168,7 @@ struct ps_ctx {
     float* partials = nullptr;
     int32_t* d_sched = nullptr;  // chunk counters of the tensor-core kernel: {next, done} per lane
     int32_t* d_row_done = nullptr;  // its split-KV arrival counters: max_batch x num_kv_heads
+    std::vector<ps::AttnTensorMaps> tmaps;  // per layer; empty = the kernel copies row by row
     int32_t max_parts = 0;
     int attn_kernel = 1;
     int32_t num_sms = 1;
@@ -760,7 +761,8 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
     if (wait_event) CK(cudaStreamWaitEvent(ctx->compute, wait_event, 0));
     {
         ProfScope prof(ctx, kProfAttn, ctx->compute, m.kv_bytes_per_layer, wait_event ? 1000 + layer : layer);
-        CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], q, out, lse, m.dev, 0,
+        const ps::AttnTensorMaps* maps = ctx->tmaps.empty() ? nullptr : &ctx->tmaps[(size_t)layer];
+        CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], maps, q, out, lse, m.dev, 0,
                                   ctx->partials, ctx->d_sched, ctx->d_row_done, ctx->d_status, ctx->compute));
         ctx->launches++;
         ++*n_launched;
@@ -960,12 +962,24 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     ctx->attn_kernel = PS_ATTN_SIMT;
     {
         ps::AttnShape sh{cfg->num_kv_heads, cfg->num_q_heads, cfg->head_dim, cfg->block_size, cfg->num_gpu_blocks};
-        if (cfg->attn_kernel == PS_ATTN_MMA && !ps::attn_mma_supported(sh)) {
+        if ((cfg->attn_kernel == PS_ATTN_MMA || cfg->attn_kernel == PS_ATTN_MMA_ROWS) && !ps::attn_mma_supported(sh)) {
             ctx->err = "the tensor-core attention kernel does not support this shape";
             return create_fail(ctx, PS_ERR_INVALID);
         }
-        if (cfg->attn_kernel == PS_ATTN_MMA || (cfg->attn_kernel == PS_ATTN_AUTO && ps::attn_mma_supported(sh)))
+        if (cfg->attn_kernel == PS_ATTN_MMA || cfg->attn_kernel == PS_ATTN_MMA_ROWS ||
+            (cfg->attn_kernel == PS_ATTN_AUTO && ps::attn_mma_supported(sh)))
             ctx->attn_kernel = PS_ATTN_MMA;
+        if (ctx->attn_kernel == PS_ATTN_MMA && cfg->attn_kernel != PS_ATTN_MMA_ROWS) {
+            // tiles by tensor-map box copies when the driver accepts the maps, else row by row
+            ctx->tmaps.resize((size_t)L);
+            for (int l = 0; l < L; ++l)
+                if (ps::attn_make_tensor_maps(sh, ctx->kpools[(size_t)l], ctx->vpools[(size_t)l], &ctx->tmaps[(size_t)l]) !=
+                    cudaSuccess) {
+                    ctx->tmaps.clear();
+                    cudaGetLastError();
+                    break;
+                }
+        }
         const int64_t max_batch = std::max(cfg->max_batch, 1);
         int64_t max_parts;
         if (cfg->kv_split_tokens > 0) {

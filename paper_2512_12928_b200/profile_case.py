@@ -1,6 +1,6 @@
 """Small, self-contained cases of the three kernels for profilers and quick timing.
 
-    python -m paper_2512_12928_b200.profile_case attn    [--iters N] [--batch B] [--ctx T] [--q-heads H] [--simt]
+    python -m paper_2512_12928_b200.profile_case attn    [--iters N] [--batch B] [--ctx T] [--q-heads H] [--simt | --rows]
     python -m paper_2512_12928_b200.profile_case gather  [--iters N] [--blocks K]
     python -m paper_2512_12928_b200.profile_case scatter [--iters N] [--blocks K]
 
@@ -31,6 +31,7 @@ def main():
     ap.add_argument("--q-heads", type=int, default=32)
     ap.add_argument("--blocks", type=int, default=2048)
     ap.add_argument("--simt", action="store_true")
+    ap.add_argument("--rows", action="store_true", help="tensor-core kernel fed by per-row bulk copies")
     args = ap.parse_args()
 
     L, Hkv, D, S = 2, 8, 128, 16
@@ -45,7 +46,7 @@ def main():
     lib = B.KVSwap(num_layers=L, num_kv_heads=Hkv, num_q_heads=args.q_heads, head_dim=D, block_size=S,
                    num_gpu_blocks=nb, max_blocks_per_req=nblk_req + 1, max_batch=args.batch, host_pool_bytes=1 << 20,
                    initial_free_order=order, k_pools=[K[l] for l in range(L)], v_pools=[V[l] for l in range(L)],
-                   attn_kernel=B.PS_ATTN_SIMT if args.simt else B.PS_ATTN_AUTO)
+                   attn_kernel=B.PS_ATTN_SIMT if args.simt else B.PS_ATTN_MMA_ROWS if args.rows else B.PS_ATTN_AUTO)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     res = {"case": args.case}
     if args.case == "attn":
@@ -68,7 +69,7 @@ def main():
         ms = e0.elapsed_time(e1) / args.iters
         kv_bytes = args.batch * args.ctx * 2 * Hkv * D * 2
         res.update(us_per_launch=ms * 1e3, kv_bytes_per_launch=kv_bytes, gb_per_s=kv_bytes / ms / 1e6,
-                   batch=args.batch, ctx=args.ctx, q_heads=args.q_heads, kernel="simt" if args.simt else "auto")
+                   batch=args.batch, ctx=args.ctx, q_heads=args.q_heads, kernel="simt" if args.simt else "mma_rows" if args.rows else "auto")
     else:
         direction = 0 if args.case == "gather" else 1
         ids = np.random.default_rng(2).permutation(nb)[: args.blocks].astype(np.int32)

@@ -122,6 +122,10 @@ SHAPES = [
     (8, 64, 128, 16, B.PS_ATTN_MMA, 0),
     (8, 64, 128, 32, B.PS_ATTN_MMA, 0),
     (8, 32, 128, 48, B.PS_ATTN_MMA, 0),
+    # the same kernel fed by one bulk copy per token row instead of tensor-map boxes
+    (8, 32, 128, 16, B.PS_ATTN_MMA_ROWS, 0),
+    (8, 64, 128, 32, B.PS_ATTN_MMA_ROWS, 0),
+    (8, 8, 128, 48, B.PS_ATTN_MMA_ROWS, 0),
 ]
 
 
