@@ -506,6 +506,11 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
+    // Programmatic dependent launch: the next layer's launch (same kernel, the other set of scratch buffers,
+    // independent inputs) may start filling SMs as the CTAs of this one retire, which hides its launch latency
+    // and prologue under this launch's tail.  A no-op for ordinary launches.
+    if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMmaStages; ++s) {
             mbar_init(bar_full + 8 * s, 1);
@@ -786,31 +791,45 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             for (int p = 0; p < n_pend; ++p) merge_row<G>(pending[p], h, lane, batch, partials, out, lse, row_done);
         }
     }
+    // A launch does not complete before the launch it was made programmatically dependent on has completed:
+    // work enqueued after this launch may rely on both.  (Returns at once for ordinary launches.)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 template <int G>
 cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool, const AttnTensorMaps* maps, const void* q,
                        void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials, int32_t* sched,
-                       int32_t* row_done, int32_t* d_status, cudaStream_t stream) {
+                       int32_t* row_done, int32_t* d_status, bool after_own_launch, cudaStream_t stream) {
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)kMmaD);
     static_assert(sizeof(CUtensorMap) == sizeof(maps->k), "AttnTensorMaps must hold driver tensor maps");
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)batch.n_cta[lane]);
+    cfg.blockDim = dim3(kMmaThreads);
+    cfg.dynamicSmemBytes = (size_t)mma_smem_bytes(maps != nullptr);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = after_own_launch ? 1 : 0;
+    CUtensorMap km, vm;
     if (maps != nullptr) {
-        CUtensorMap km, vm;
         memcpy(&km, maps->k, sizeof km);
         memcpy(&vm, maps->v, sizeof vm);
-        decode_attn_mma_kernel<G, true><<<(unsigned)batch.n_cta[lane], kMmaThreads, mma_smem_bytes(true), stream>>>(
-            (const __nv_bfloat16*)kpool, (const __nv_bfloat16*)vpool, km, vm, (const __nv_bfloat16*)q, (__nv_bfloat16*)out,
-            lse, batch, lane, sh.block_size, shift_of(sh.block_size), sh.num_blocks, partials, sched, row_done,
-            scale_log2e, d_status);
     } else {
-        CUtensorMap none;
-        memset(&none, 0, sizeof none);
-        decode_attn_mma_kernel<G, false><<<(unsigned)batch.n_cta[lane], kMmaThreads, mma_smem_bytes(false), stream>>>(
-            (const __nv_bfloat16*)kpool, (const __nv_bfloat16*)vpool, none, none, (const __nv_bfloat16*)q,
-            (__nv_bfloat16*)out, lse, batch, lane, sh.block_size, shift_of(sh.block_size), sh.num_blocks, partials, sched,
-            row_done, scale_log2e, d_status);
+        memset(&km, 0, sizeof km);
+        memset(&vm, 0, sizeof vm);
     }
-    return cudaGetLastError();
+    const __nv_bfloat16* kp = (const __nv_bfloat16*)kpool;
+    const __nv_bfloat16* vp = (const __nv_bfloat16*)vpool;
+    const __nv_bfloat16* qp = (const __nv_bfloat16*)q;
+    __nv_bfloat16* op = (__nv_bfloat16*)out;
+    const int32_t shift = shift_of(sh.block_size);
+    if (maps != nullptr)
+        return cudaLaunchKernelEx(&cfg, decode_attn_mma_kernel<G, true>, kp, vp, km, vm, qp, op, lse, batch, lane,
+                                  sh.block_size, shift, sh.num_blocks, partials, sched, row_done, scale_log2e, d_status);
+    return cudaLaunchKernelEx(&cfg, decode_attn_mma_kernel<G, false>, kp, vp, km, vm, qp, op, lse, batch, lane,
+                              sh.block_size, shift, sh.num_blocks, partials, sched, row_done, scale_log2e, d_status);
 }
 
 }  // namespace
@@ -876,7 +895,7 @@ cudaError_t attn_make_tensor_maps(const AttnShape& sh, const void* kpool, const 
 cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool,
                                const AttnTensorMaps* maps, const void* q, void* out, float* lse, const AttnBatch& batch,
                                int32_t lane, float* partials, int32_t* sched, int32_t* row_done, int32_t* d_status,
-                               cudaStream_t stream) {
+                               bool after_own_launch, cudaStream_t stream) {
     if (lane < 0 || lane > 1) return cudaErrorInvalidValue;
     const int item_begin = batch.lane_items[lane];
     const int n_items = batch.lane_items[lane + 1] - item_begin;
@@ -887,13 +906,13 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
             return cudaErrorNotSupported;
         switch (G) {
             case 1: return launch_mma<1>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       stream);
+                                       after_own_launch, stream);
             case 2: return launch_mma<2>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       stream);
+                                       after_own_launch, stream);
             case 4: return launch_mma<4>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       stream);
+                                       after_own_launch, stream);
             case 8: return launch_mma<8>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       stream);
+                                       after_own_launch, stream);
         }
         return cudaErrorNotSupported;
     }

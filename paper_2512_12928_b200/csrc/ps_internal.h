@@ -91,7 +91,11 @@ cudaError_t attn_make_tensor_maps(const AttnShape& sh, const void* kpool, const 
 cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool,
                                const AttnTensorMaps* maps, const void* q, void* out, float* lse, const AttnBatch& batch,
                                int32_t lane, float* partials, int32_t* sched, int32_t* row_done, int32_t* d_status,
-                               cudaStream_t stream);
+                               bool after_own_launch, cudaStream_t stream);
+// after_own_launch (tensor-core kernel only): the previous kernel on `stream` is a launch of the same kernel
+// that filled every SM, used the OTHER set of partials / sched / row_done, and shares no data with this one;
+// the launch is then made programmatically dependent on it, so its CTAs start as that launch's CTAs retire.
+// With one CTA per SM and full grids at most two consecutive launches overlap, hence two sets of scratch.
 
 // Token granularity at which the tensor-core kernel splits a context.
 constexpr int kMmaTileTokens = 16;

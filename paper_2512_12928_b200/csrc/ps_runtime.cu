@@ -165,9 +165,11 @@ struct ps_ctx {
     std::vector<cudaEvent_t> ev_pool, ev_pool_timing;
     std::deque<std::pair<uint64_t, std::pair<int64_t, int64_t>>> img_release;  // in_ticket -> (off, bytes)
     std::vector<int64_t> gated_reqs;
-    float* partials = nullptr;
-    int32_t* d_sched = nullptr;  // chunk counters of the tensor-core kernel: {next, done} per lane
-    int32_t* d_row_done = nullptr;  // its split-KV arrival counters: max_batch x num_kv_heads
+    // split-KV scratch, two sets used alternately: consecutive attention launches of a step may overlap
+    float* partials[2] = {nullptr, nullptr};
+    int32_t* d_sched[2] = {nullptr, nullptr};     // chunk counters of the tensor-core kernel: {next, done} per lane
+    int32_t* d_row_done[2] = {nullptr, nullptr};  // its split-KV arrival counters: max_batch x num_kv_heads
+    int scratch_set = 0;
     std::vector<ps::AttnTensorMaps> tmaps;  // per layer; empty = the kernel copies row by row
     int32_t max_parts = 0;
     int attn_kernel = 1;
@@ -752,25 +754,32 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
 // Launches one layer of attention for the prepared batch on the compute stream.  wait_event: the
 // layer's reload event when rows of the batch are still being reloaded (Appendix B: the compute stream
 // synchronises on a layer chunk's event only before it executes that chunk); nullptr = no wait.
+// follows_own: the previous kernel on the compute stream is this function's launch for the previous layer
+// of the same step (independent data); full-grid tensor-core launches then overlap head to tail.
 int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, float* lse, cudaEvent_t wait_event,
-                          int32_t* n_launched) {
+                          bool follows_own, int32_t* n_launched) {
     BatchMeta& m = ctx->meta;
     if (m.n_items == 0) return PS_OK;
     ps::AttnShape sh{ctx->cfg.num_kv_heads, ctx->cfg.num_q_heads, ctx->cfg.head_dim, ctx->cfg.block_size,
                      ctx->cfg.num_gpu_blocks};
     if (wait_event) CK(cudaStreamWaitEvent(ctx->compute, wait_event, 0));
+    const bool mma = ctx->attn_kernel == PS_ATTN_MMA;
+    const bool overlap = follows_own && mma && !ctx->profile && m.dev.n_cta[0] == ctx->num_sms;
+    const int set = ctx->scratch_set;
+    ctx->scratch_set ^= 1;
     {
         ProfScope prof(ctx, kProfAttn, ctx->compute, m.kv_bytes_per_layer, wait_event ? 1000 + layer : layer);
         const ps::AttnTensorMaps* maps = ctx->tmaps.empty() ? nullptr : &ctx->tmaps[(size_t)layer];
         CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], maps, q, out, lse, m.dev, 0,
-                                  ctx->partials, ctx->d_sched, ctx->d_row_done, ctx->d_status, ctx->compute));
+                                  ctx->partials[set], ctx->d_sched[set], ctx->d_row_done[set], ctx->d_status, overlap,
+                                  ctx->compute));
         ctx->launches++;
         ++*n_launched;
     }
     // the tensor-core kernel combines split rows itself; the CUDA-core kernel needs the merge pass
-    if (ctx->attn_kernel != PS_ATTN_MMA && m.any_multi) {
+    if (!mma && m.any_multi) {
         ProfScope prof(ctx, kProfMerge, ctx->compute, 0, layer);
-        CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials, -1, ctx->compute));
+        CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials[set], -1, ctx->compute));
         ctx->launches++;
         ++*n_launched;
     }
@@ -802,9 +811,11 @@ void destroy_ctx(ps_ctx* ctx) {
         if (ctx->stage_in) cudaFree(ctx->stage_in);
         if (ctx->d_kpools) cudaFree(ctx->d_kpools);
         if (ctx->d_vpools) cudaFree(ctx->d_vpools);
-        if (ctx->partials) cudaFree(ctx->partials);
-        if (ctx->d_sched) cudaFree(ctx->d_sched);
-        if (ctx->d_row_done) cudaFree(ctx->d_row_done);
+        for (int i = 0; i < 2; ++i) {
+            if (ctx->partials[i]) cudaFree(ctx->partials[i]);
+            if (ctx->d_sched[i]) cudaFree(ctx->d_sched[i]);
+            if (ctx->d_row_done[i]) cudaFree(ctx->d_row_done[i]);
+        }
         if (ctx->status) cudaFreeHost(ctx->status);
         if (ctx->own_host_pool && ctx->host_pool) cudaFreeHost(ctx->host_pool);
         cudaGetLastError();
@@ -998,12 +1009,14 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
         // (static shares + at most ~6 dynamic chunks per CTA, plus one chunk boundary per row)
         max_parts = std::max<int64_t>(max_parts, 3 * max_batch + 2 * 8 * (int64_t)ctx->num_sms + 16);
         ctx->max_parts = (int32_t)std::min<int64_t>(max_parts, 1 << 22);
-        CKC(cudaMalloc((void**)&ctx->partials, ps::attn_partial_bytes(sh, ctx->max_parts)));
-        CKC(cudaMalloc((void**)&ctx->d_sched, 4 * sizeof(int32_t)));
-        CKC(cudaMemset(ctx->d_sched, 0, 4 * sizeof(int32_t)));
         const size_t done_bytes = (size_t)max_batch * cfg->num_kv_heads * sizeof(int32_t);
-        CKC(cudaMalloc((void**)&ctx->d_row_done, done_bytes));
-        CKC(cudaMemset(ctx->d_row_done, 0, done_bytes));
+        for (int i = 0; i < 2; ++i) {
+            CKC(cudaMalloc((void**)&ctx->partials[i], ps::attn_partial_bytes(sh, ctx->max_parts)));
+            CKC(cudaMalloc((void**)&ctx->d_sched[i], 4 * sizeof(int32_t)));
+            CKC(cudaMemset(ctx->d_sched[i], 0, 4 * sizeof(int32_t)));
+            CKC(cudaMalloc((void**)&ctx->d_row_done[i], done_bytes));
+            CKC(cudaMemset(ctx->d_row_done[i], 0, done_bytes));
+        }
         const size_t meta_chunk = (size_t)max_batch * cfg->max_blocks_per_req * 4 + (size_t)max_batch * 16 +
                                   (size_t)ctx->max_parts * sizeof(ps::AttnItem) + (size_t)ctx->num_sms * 8 + 8192;
         CKR(arena_init(ctx, ctx->a_meta, meta_chunk, 3, ctx->compute));
@@ -1281,7 +1294,7 @@ int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, flo
     if (rc != PS_OK) return rc;
     int32_t launched = 0;
     return launch_layer_attn(ctx, layer, q, out, lse, ctx->meta.n_gated_rows ? ctx->ev_in[(size_t)layer] : nullptr,
-                             &launched);
+                             /*follows_own=*/false, &launched);
 }
 
 int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs, int32_t batch,
@@ -1361,7 +1374,7 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
             }
             int32_t launched = 0;
             rc = launch_layer_attn(ctx, l, (const char*)q_all_layers + l * layer_bytes,
-                                   (char*)out_all_layers + l * layer_bytes, nullptr, wait, &launched);
+                                   (char*)out_all_layers + l * layer_bytes, nullptr, wait, /*follows_own=*/l > 0, &launched);
             if (rc != PS_OK) return rc;
         }
     }

@@ -209,7 +209,7 @@ extern "C" int32_t ps_decode_attn_static(const void* kpool, const void* vpool, c
     float* partials = reinterpret_cast<float*>(scratch + kMetaBytes);
     int32_t* status = status_word ? status_word : reinterpret_cast<int32_t*>(scratch + kOffStatus);
     if (e == cudaSuccess)
-        e = ps::launch_decode_attn(/*SIMT kernel*/ 1, sh, kpool, vpool, nullptr, q, out, lse, ab, 0, partials, nullptr, nullptr, status, s);
+        e = ps::launch_decode_attn(/*SIMT kernel*/ 1, sh, kpool, vpool, nullptr, q, out, lse, ab, 0, partials, nullptr, nullptr, status, false, s);
     if (e == cudaSuccess && any_multi) e = ps::launch_attn_merge(sh, out, lse, ab, partials, -1, s);
     if (e != cudaSuccess) {
         snprintf(msg, sizeof msg, "ps_decode_attn_static: kernel launch: %s", cudaGetErrorString(e));
