@@ -284,9 +284,12 @@ int32_t ps_decode_attn_static(const void* kpool, const void* vpool, const void* 
  * a request whose missing blocks fit is taken whole, the first that does not fit gets what is
  * left; then for each layer issues that layer's reload (as ps_swap_in_layer) and launches that
  * layer's attention for the requests of `reqs` that are RESIDENT once this step's reload is
- * issued.  When the batch holds requests completed by this step, each layer's attention launch
- * waits on that layer's reload event (and on nothing later), so the reload of layer i+1 runs
- * under the attention of layer i.  Everything is enqueued asynchronously.
+ * issued.  Requests completed by this step have each layer's attention wait on that layer's
+ * reload event (and on nothing later), so the reload of layer i+1 runs under the attention of
+ * layer i; with the tensor-core kernel they run in a launch of their own on a side stream, so
+ * that the other requests never wait, and the compute stream joins that stream at the end of the
+ * step.  The queries of all layers are inputs, so consecutive layers are independent and their
+ * launches may overlap head to tail.  Everything is enqueued asynchronously.
  *   q_all_layers, out_all_layers : device, bf16 [num_layers][batch][num_q_heads][head_dim]; rows of
  *                                  requests that do not decode are left untouched.  Both may be
  *                                  NULL with batch 0 for a copy-only step.

@@ -4,8 +4,9 @@
 //
 // Streams (Appendix B: a copy stream per direction, independent of the compute stream; one
 // completion event per layer chunk):
-//   compute  : the caller's stream; attention runs here (a layer's launch waits on that layer's reload
-//              event when the batch holds requests whose reload is landing in this step).
+//   compute  : the caller's stream; attention runs here.
+//   s_lane   : attention of the requests whose reload lands in this step, layer by layer behind that
+//              layer's reload event (tensor-core kernel; other kernels make the whole launch wait instead).
 //   s_gather : gather kernels of swap-out.           s_d2h : staging -> pinned host copies.
 //   s_h2d    : pinned host -> staging copies.        s_scatter : scatter kernels of swap-in.
 // Each direction owns kSlots staging slots; two events per slot hand a slot back and forth between
@@ -123,6 +124,7 @@ struct BatchMeta {  // cached device metadata of the last prepared decode batch
     int32_t n_items = 0, n_ungated_items = 0, n_parts = 0;
     int32_t n_gated_rows = 0;
     bool any_multi = false, lane_multi[2] = {false, false};
+    bool two_lanes = false;
     int64_t kv_bytes_per_layer = 0;
 };
 
@@ -149,7 +151,8 @@ struct ps_ctx {
     char* host_pool = nullptr;
     bool own_host_pool = false;
     HostPool hpool;
-    cudaStream_t compute = nullptr, s_gather = nullptr, s_d2h = nullptr, s_h2d = nullptr, s_scatter = nullptr;
+    cudaStream_t compute = nullptr, s_gather = nullptr, s_d2h = nullptr, s_h2d = nullptr, s_scatter = nullptr,
+                 s_lane = nullptr;
     char* stage_out = nullptr;
     char* stage_in = nullptr;
     int64_t slot_bytes = 0;
@@ -157,7 +160,7 @@ struct ps_ctx {
     bool out_used[kSlots]{}, in_used[kSlots]{};
     uint64_t out_next = 0, in_next = 0;
     std::vector<cudaEvent_t> ev_in;  // per layer
-    cudaEvent_t e_mark = nullptr, e_mark2 = nullptr;
+    cudaEvent_t e_mark = nullptr, e_mark2 = nullptr, e_fork = nullptr, e_join = nullptr;
     int32_t* status = nullptr;  // mapped pinned word written by kernels on a bad block id
     int32_t* d_status = nullptr;
     Tracker t_d2h, t_scatter, t_compute;
@@ -165,10 +168,11 @@ struct ps_ctx {
     std::vector<cudaEvent_t> ev_pool, ev_pool_timing;
     std::deque<std::pair<uint64_t, std::pair<int64_t, int64_t>>> img_release;  // in_ticket -> (off, bytes)
     std::vector<int64_t> gated_reqs;
-    // split-KV scratch, two sets used alternately: consecutive attention launches of a step may overlap
-    float* partials[2] = {nullptr, nullptr};
-    int32_t* d_sched[2] = {nullptr, nullptr};     // chunk counters of the tensor-core kernel: {next, done} per lane
-    int32_t* d_row_done[2] = {nullptr, nullptr};  // its split-KV arrival counters: max_batch x num_kv_heads
+    // split-KV scratch: sets 0 and 1 are used alternately by the launches on the compute stream (consecutive
+    // launches of a step may overlap), set 2 by the launches on the reload lane
+    float* partials[3] = {nullptr, nullptr, nullptr};
+    int32_t* d_sched[3] = {nullptr, nullptr, nullptr};     // chunk counters of the tensor-core kernel: {next, done} per lane
+    int32_t* d_row_done[3] = {nullptr, nullptr, nullptr};  // its split-KV arrival counters: max_batch x num_kv_heads
     int scratch_set = 0;
     std::vector<ps::AttnTensorMaps> tmaps;  // per layer; empty = the kernel copies row by row
     int32_t max_parts = 0;
@@ -540,12 +544,17 @@ int32_t choose_split(const ps_ctx* ctx, int64_t total_tokens) {
 
 // Builds (or reuses) the device metadata for a decode batch.  Row b of the metadata is position b of
 // the caller's request array (q / out rows are addressed by that position); rows with active[b] == 0
-// get no work item.  gated[b] != 0 marks rows whose reload is still landing (the launch then waits on
-// the layer's reload event).
+// get no work item.  gated[b] != 0 marks rows whose reload is still landing: their attention waits on
+// the layer's reload event.  With want_lanes they get a work list of their own (lane 1), launched on
+// the reload-lane stream behind the event, so that the launches of the other rows never wait.
 int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::vector<char>& active,
-                      const std::vector<char>& gated) {
+                      const std::vector<char>& gated, bool want_lanes) {
     BatchMeta& m = ctx->meta;
-    if (m.valid && m.epoch == ctx->table_epoch && (int32_t)m.reqs.size() == B &&
+    // two work lists (lanes) only for the tensor-core kernel and only when some row is gated
+    bool two_lanes = false;
+    if (want_lanes && ctx->attn_kernel == PS_ATTN_MMA)
+        for (int32_t b = 0; b < B; ++b) two_lanes |= active[b] && gated[b];
+    if (m.valid && m.epoch == ctx->table_epoch && (int32_t)m.reqs.size() == B && m.two_lanes == two_lanes &&
         std::equal(m.reqs.begin(), m.reqs.end(), reqs) && m.gated == gated && m.active == active)
         return PS_OK;
 
@@ -564,11 +573,11 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     bool any_multi = false, lane_multi[2] = {false, false};
     const bool mma = ctx->attn_kernel == PS_ATTN_MMA;
     const int32_t split = mma ? 0 : choose_split(ctx, total_tokens);
-    for (int pass = 0; pass < 1; ++pass) {  // a single work list (lane 0) holds every active row
+    for (int pass = 0; pass < (two_lanes ? 2 : 1); ++pass) {  // lane 0: rows that need no wait (or all rows); lane 1: gated rows
         if (!mma) {
             // SIMT kernel: one CTA per (item, KV head); items are fixed-size token ranges of a row
             for (int32_t b = 0; b < B; ++b) {
-                if (!active[b]) continue;
+                if (!active[b] || (two_lanes && (gated[b] ? 1 : 0) != pass)) continue;
                 const Req& r = ctx->reqs[reqs[b]];
                 const int32_t n = std::max(1, (r.n_tokens + split - 1) / split);
                 row_first[b] = parts;
@@ -599,7 +608,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
             int64_t total_tiles = 0;
             int32_t lane_rows = 0;
             for (int32_t b = 0; b < B; ++b)
-                if (active[b]) {
+                if (active[b] && !(two_lanes && (gated[b] ? 1 : 0) != pass)) {
                     total_tiles += (ctx->reqs[reqs[b]].n_tokens + kTile - 1) / kTile;
                     ++lane_rows;
                 }
@@ -624,7 +633,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
                 filled = 0;
             };
             for (int32_t b = 0; b < B; ++b) {
-                if (!active[b]) continue;
+                if (!active[b] || (two_lanes && (gated[b] ? 1 : 0) != pass)) continue;
                 const Req& r = ctx->reqs[reqs[b]];
                 const int64_t tiles_b = (r.n_tokens + kTile - 1) / kTile;
                 const size_t first_item = items.size();
@@ -673,8 +682,8 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
             }
             if (n_cta > 0 && !in_dyn) close_static();
         }
+        if (pass == 0) n_ungated = (int32_t)items.size();
     }
-    n_ungated = (int32_t)items.size();
     if (parts > ctx->max_parts) return ctx->fail(PS_ERR_INVALID, "split-KV scratch too small for this batch");
 
     const size_t sz_tables = (size_t)round_up((int64_t)B * stride * 4, 256);
@@ -703,7 +712,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     memcpy(h + sz_tables + 2 * sz_vec, row_parts.data(), (size_t)B * 4);
     {
         int32_t* lane = (int32_t*)(h + sz_tables + 3 * sz_vec);
-        for (int32_t b = 0; b < B; ++b) lane[b] = 0;
+        for (int32_t b = 0; b < B; ++b) lane[b] = two_lanes && gated[b] ? 1 : 0;
     }
     if (!items.empty()) memcpy(h + sz_tables + 4 * sz_vec, items.data(), items.size() * sizeof(ps::AttnItem));
     {
@@ -720,6 +729,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     m.reqs.assign(reqs, reqs + B);
     m.gated = gated;
     m.active = active;
+    m.two_lanes = two_lanes;
     m.epoch = ctx->table_epoch;
     m.valid = true;
     m.dev.block_tables = (const int32_t*)d;
@@ -751,35 +761,50 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     return PS_OK;
 }
 
-// Launches one layer of attention for the prepared batch on the compute stream.  wait_event: the
-// layer's reload event when rows of the batch are still being reloaded (Appendix B: the compute stream
-// synchronises on a layer chunk's event only before it executes that chunk); nullptr = no wait.
-// follows_own: the previous kernel on the compute stream is this function's launch for the previous layer
-// of the same step (independent data); full-grid tensor-core launches then overlap head to tail.
+// Launches one layer of attention for the prepared batch.  wait_event: the layer's reload event when rows
+// of the batch are still being reloaded (Appendix B: the computation synchronises on a layer chunk's event
+// only before it executes that chunk); nullptr = no wait.  With two work lists the rows that need no wait
+// run on the compute stream and the gated rows on the reload lane behind the event; with one list the
+// whole launch waits.  follows_own: the previous kernel on the compute stream is this function's launch
+// for the previous layer of the same step (independent data); full-grid tensor-core launches then overlap
+// head to tail.
 int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, float* lse, cudaEvent_t wait_event,
                           bool follows_own, int32_t* n_launched) {
     BatchMeta& m = ctx->meta;
     if (m.n_items == 0) return PS_OK;
     ps::AttnShape sh{ctx->cfg.num_kv_heads, ctx->cfg.num_q_heads, ctx->cfg.head_dim, ctx->cfg.block_size,
                      ctx->cfg.num_gpu_blocks};
-    if (wait_event) CK(cudaStreamWaitEvent(ctx->compute, wait_event, 0));
     const bool mma = ctx->attn_kernel == PS_ATTN_MMA;
-    const bool overlap = follows_own && mma && !ctx->profile && m.dev.n_cta[0] == ctx->num_sms;
-    const int set = ctx->scratch_set;
-    ctx->scratch_set ^= 1;
-    {
-        ProfScope prof(ctx, kProfAttn, ctx->compute, m.kv_bytes_per_layer, wait_event ? 1000 + layer : layer);
-        const ps::AttnTensorMaps* maps = ctx->tmaps.empty() ? nullptr : &ctx->tmaps[(size_t)layer];
-        CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], maps, q, out, lse, m.dev, 0,
-                                  ctx->partials[set], ctx->d_sched[set], ctx->d_row_done[set], ctx->d_status, overlap,
-                                  ctx->compute));
-        ctx->launches++;
-        ++*n_launched;
+    const ps::AttnTensorMaps* maps = ctx->tmaps.empty() ? nullptr : &ctx->tmaps[(size_t)layer];
+    const bool lanes = m.two_lanes && m.n_items > m.n_ungated_items;
+    if (wait_event && !lanes) CK(cudaStreamWaitEvent(ctx->compute, wait_event, 0));
+    if (m.n_ungated_items > 0) {
+        const bool overlap = follows_own && mma && !ctx->profile && m.dev.n_cta[0] == ctx->num_sms;
+        const int set = ctx->scratch_set;
+        ctx->scratch_set ^= 1;
+        const int64_t bytes = m.kv_bytes_per_layer * m.n_ungated_items / m.n_items;
+        {
+            ProfScope prof(ctx, kProfAttn, ctx->compute, bytes, wait_event && !lanes ? 1000 + layer : layer);
+            CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], maps, q, out, lse, m.dev,
+                                      0, ctx->partials[set], ctx->d_sched[set], ctx->d_row_done[set], ctx->d_status,
+                                      overlap, ctx->compute));
+            ctx->launches++;
+            ++*n_launched;
+        }
+        // the tensor-core kernel combines split rows itself; the CUDA-core kernel needs the merge pass
+        if (!mma && m.any_multi) {
+            ProfScope prof(ctx, kProfMerge, ctx->compute, 0, layer);
+            CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials[set], -1, ctx->compute));
+            ctx->launches++;
+            ++*n_launched;
+        }
     }
-    // the tensor-core kernel combines split rows itself; the CUDA-core kernel needs the merge pass
-    if (!mma && m.any_multi) {
-        ProfScope prof(ctx, kProfMerge, ctx->compute, 0, layer);
-        CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials[set], -1, ctx->compute));
+    if (lanes) {
+        if (wait_event) CK(cudaStreamWaitEvent(ctx->s_lane, wait_event, 0));
+        const int64_t bytes = m.kv_bytes_per_layer * (m.n_items - m.n_ungated_items) / m.n_items;
+        ProfScope prof(ctx, kProfAttn, ctx->s_lane, bytes, 1000 + layer);
+        CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], maps, q, out, lse, m.dev, 1,
+                                  ctx->partials[2], ctx->d_sched[2], ctx->d_row_done[2], ctx->d_status, false, ctx->s_lane));
         ctx->launches++;
         ++*n_launched;
     }
@@ -788,13 +813,13 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
 
 void destroy_ctx(ps_ctx* ctx) {
     if (!ctx->bk) {
-        for (cudaStream_t s : {ctx->s_gather, ctx->s_d2h, ctx->s_h2d, ctx->s_scatter})
+        for (cudaStream_t s : {ctx->s_gather, ctx->s_d2h, ctx->s_h2d, ctx->s_scatter, ctx->s_lane})
             if (s) cudaStreamDestroy(s);
         for (int i = 0; i < kSlots; ++i)
             for (cudaEvent_t e : {ctx->e_gathered[i], ctx->e_drained[i], ctx->e_loaded[i], ctx->e_scattered[i]})
                 if (e) cudaEventDestroy(e);
         for (cudaEvent_t e : ctx->ev_in) cudaEventDestroy(e);
-        for (cudaEvent_t e : {ctx->e_mark, ctx->e_mark2, ctx->trace_base})
+        for (cudaEvent_t e : {ctx->e_mark, ctx->e_mark2, ctx->e_fork, ctx->e_join, ctx->trace_base})
             if (e) cudaEventDestroy(e);
         for (auto& t : {&ctx->t_d2h, &ctx->t_scatter, &ctx->t_compute})
             for (auto& p : t->pending) cudaEventDestroy(p.second);
@@ -811,7 +836,7 @@ void destroy_ctx(ps_ctx* ctx) {
         if (ctx->stage_in) cudaFree(ctx->stage_in);
         if (ctx->d_kpools) cudaFree(ctx->d_kpools);
         if (ctx->d_vpools) cudaFree(ctx->d_vpools);
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < 3; ++i) {
             if (ctx->partials[i]) cudaFree(ctx->partials[i]);
             if (ctx->d_sched[i]) cudaFree(ctx->d_sched[i]);
             if (ctx->d_row_done[i]) cudaFree(ctx->d_row_done[i]);
@@ -940,6 +965,9 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     CKC(cudaStreamCreateWithPriority(&ctx->s_d2h, cudaStreamNonBlocking, prio_hi));
     CKC(cudaStreamCreateWithPriority(&ctx->s_h2d, cudaStreamNonBlocking, prio_hi));
     CKC(cudaStreamCreateWithPriority(&ctx->s_scatter, cudaStreamNonBlocking, prio_hi));
+    // the reload lane: attention of the requests whose reload lands in this step, behind the per-layer events;
+    // its few CTAs should get an SM as soon as one frees up
+    CKC(cudaStreamCreateWithPriority(&ctx->s_lane, cudaStreamNonBlocking, prio_hi));
     ctx->t_d2h.s = ctx->s_d2h;
     ctx->t_scatter.s = ctx->s_scatter;
     ctx->t_compute.s = ctx->compute;
@@ -958,6 +986,8 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     for (int l = 0; l < L; ++l) CKC(cudaEventCreateWithFlags(&ctx->ev_in[(size_t)l], cudaEventDisableTiming));
     CKC(cudaEventCreateWithFlags(&ctx->e_mark, cudaEventDisableTiming));
     CKC(cudaEventCreateWithFlags(&ctx->e_mark2, cudaEventDisableTiming));
+    CKC(cudaEventCreateWithFlags(&ctx->e_fork, cudaEventDisableTiming));
+    CKC(cudaEventCreateWithFlags(&ctx->e_join, cudaEventDisableTiming));
     CKC(cudaHostAlloc((void**)&ctx->status, 64, cudaHostAllocMapped));
     memset(ctx->status, 0, 64);
     CKC(cudaHostGetDevicePointer((void**)&ctx->d_status, ctx->status, 0));
@@ -1010,7 +1040,7 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
         max_parts = std::max<int64_t>(max_parts, 3 * max_batch + 2 * 8 * (int64_t)ctx->num_sms + 16);
         ctx->max_parts = (int32_t)std::min<int64_t>(max_parts, 1 << 22);
         const size_t done_bytes = (size_t)max_batch * cfg->num_kv_heads * sizeof(int32_t);
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < 3; ++i) {
             CKC(cudaMalloc((void**)&ctx->partials[i], ps::attn_partial_bytes(sh, ctx->max_parts)));
             CKC(cudaMalloc((void**)&ctx->d_sched[i], 4 * sizeof(int32_t)));
             CKC(cudaMemset(ctx->d_sched[i], 0, 4 * sizeof(int32_t)));
@@ -1290,7 +1320,7 @@ int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, flo
     }
     std::vector<char> active((size_t)batch, 1), gated((size_t)batch, 0);
     for (int32_t b = 0; b < batch; ++b) gated[(size_t)b] = ctx->reqs[reqs[b]].gated ? 1 : 0;
-    int32_t rc = prepare_batch(ctx, reqs, batch, active, gated);
+    int32_t rc = prepare_batch(ctx, reqs, batch, active, gated, /*want_lanes=*/false);
     if (rc != PS_OK) return rc;
     int32_t launched = 0;
     return launch_layer_attn(ctx, layer, q, out, lse, ctx->meta.n_gated_rows ? ctx->ev_in[(size_t)layer] : nullptr,
@@ -1341,7 +1371,7 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
     }
     const bool attn = want_attn && st.decoded > 0;
     if (attn) {
-        rc = prepare_batch(ctx, reqs, batch, active, gated);
+        rc = prepare_batch(ctx, reqs, batch, active, gated, (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) == 0);
         if (rc != PS_OK) return rc;
         st.gated = ctx->meta.n_gated_rows;
     }
@@ -1360,6 +1390,11 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
     if (attn) {
         const int64_t layer_bytes = (int64_t)batch * ctx->cfg.num_q_heads * ctx->cfg.head_dim * 2;
         const bool any_gated = ctx->meta.n_gated_rows > 0;
+        const bool lanes = ctx->meta.two_lanes;
+        if (lanes) {  // the reload lane starts where the compute stream stands now (metadata uploaded)
+            CK(cudaEventRecord(ctx->e_fork, ctx->compute));
+            CK(cudaStreamWaitEvent(ctx->s_lane, ctx->e_fork, 0));
+        }
         for (int l = 0; l < L; ++l) {
             if (!sync_reload) {
                 rc = issue_reload_layer(ctx, l, plan);
@@ -1376,6 +1411,10 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
             rc = launch_layer_attn(ctx, l, (const char*)q_all_layers + l * layer_bytes,
                                    (char*)out_all_layers + l * layer_bytes, nullptr, wait, /*follows_own=*/l > 0, &launched);
             if (rc != PS_OK) return rc;
+        }
+        if (lanes) {  // the step is complete on the compute stream only when the reload lane is
+            CK(cudaEventRecord(ctx->e_join, ctx->s_lane));
+            CK(cudaStreamWaitEvent(ctx->compute, ctx->e_join, 0));
         }
     }
 
