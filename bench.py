@@ -321,6 +321,23 @@ def decode_roofline(torch, lib, sh, ctx_lens, reqs, q, out, steps=5):
             "gbs": alg / us / 1e3, "step_us": step_ms * 1e3}
 
 
+def single_launch_rate(torch, lib, sh, ctx_lens, reqs, q, out, rounds=3):
+    """The same kernel through ps_decode_attn, one layer per call (what an engine that computes the next
+    layer's queries from this layer's output can use): launches back to back, no overlap between layers."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for l in range(sh.num_layers):
+        assert lib.decode_attn(l, q[l], out[l], reqs) == 0, lib.last_error()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(rounds):
+        for l in range(sh.num_layers):
+            assert lib.decode_attn(l, q[l], out[l], reqs) == 0, lib.last_error()
+    e1.record(); e1.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / (rounds * sh.num_layers)
+    alg = kv_bytes_per_layer(sh, ctx_lens, reqs)
+    return {"us_per_launch": us, "gbs": alg / us / 1e3}
+
+
 def overlap_sweep(torch, B, K, V, peaks_hbm):
     """Overlap workload: decode batch 128 + 8 preempted requests reloading under 16/64/256 MiB budgets.
 
@@ -530,6 +547,7 @@ def run_gpu(args):
     rf_all = decode_roofline(torch, lib, sh, w.ctx_lens, all_reqs, q, out, steps=5)
     time_decode_steps(torch, lib, residents, q_res, out_res, 2)
     rf_res = decode_roofline(torch, lib, sh, w.ctx_lens, residents, q_res, out_res, steps=5)
+    rf_single = single_launch_rate(torch, lib, sh, w.ctx_lens, all_reqs, q, out)
     clocks = sampler.stop()
 
     # ---- end-to-end arm: queries from pinned host memory and outputs back to it, every decode step
@@ -568,7 +586,11 @@ def run_gpu(args):
             "algorithmic_bytes_per_launch": rf_all["algorithmic_bytes_per_launch"],
             "us_per_launch": rf_all["us_per_layer"], "launches_per_layer": rf_all["launches_per_layer"],
             "how": "CUDA events around 5 decode-only steps (32 launches each, all 64 requests) on the compute "
-                   "stream; duration per launch includes the launch gap",
+                   "stream, as ps_step issues them: the queries of all layers are inputs, so the launches of "
+                   "consecutive layers are independent and overlap head to tail (programmatic dependent launch)",
+            "single_launch": {"gbs": rf_single["gbs"], "us_per_launch": rf_single["us_per_launch"],
+                              "frac": rf_single["gbs"] / hbm_peak,
+                              "how": "ps_decode_attn, one layer per call, back to back, no overlap between layers"},
             "frac_of_nominal_8TBs": rf_all["gbs"] / 8000.0,
             "batch_of_48_residents": {"gbs": rf_res["gbs"], "us_per_launch": rf_res["us_per_layer"],
                                       "frac": rf_res["gbs"] / hbm_peak},

@@ -165,6 +165,8 @@ struct ps_ctx {
     int32_t* d_status = nullptr;
     Tracker t_d2h, t_scatter, t_compute;
     Arena a_gather, a_meta, a_ids;
+    std::vector<int32_t> ids_cache;  // ids of the last ps_copy_blocks upload and where they sit in a_ids
+    size_t ids_cache_off = 0;
     std::vector<cudaEvent_t> ev_pool, ev_pool_timing;
     std::deque<std::pair<uint64_t, std::pair<int64_t, int64_t>>> img_release;  // in_ticket -> (off, bytes)
     std::vector<int64_t> gated_reqs;
@@ -1534,14 +1536,19 @@ int32_t ps_copy_blocks(ps_ctx* ctx, int32_t layer, const int32_t* ids, int32_t n
     if (n_blocks == 0) return PS_OK;
     for (int32_t i = 0; i < n_blocks; ++i)
         if (ids[i] < 0 || ids[i] >= ctx->cfg.num_gpu_blocks) return ctx->fail(PS_ERR_INVALID, "ps_copy_blocks: bad block id");
-    // the ids travel through a descriptor ring on the compute stream: no host wait between calls
-    size_t ioff = 0;
-    int32_t rc = arena_alloc(ctx, ctx->a_ids, (size_t)n_blocks * 4, &ioff);
-    if (rc != PS_OK) return rc;
-    memcpy(ctx->a_ids.h + ioff, ids, (size_t)n_blocks * 4);
-    CK(ps::launch_upload(ctx->a_ids.d + ioff, ctx->a_ids.hd + ioff, (size_t)round_up((int64_t)n_blocks * 4, 16),
-                         ctx->compute));
-    ctx->launches++;
+    // the ids travel through a descriptor ring on the compute stream (no host wait between calls); a call with
+    // the same ids as the previous one reuses that upload
+    size_t ioff = ctx->ids_cache_off;
+    if (ctx->ids_cache.size() != (size_t)n_blocks || memcmp(ctx->ids_cache.data(), ids, (size_t)n_blocks * 4) != 0) {
+        int32_t rc = arena_alloc(ctx, ctx->a_ids, (size_t)n_blocks * 4, &ioff);
+        if (rc != PS_OK) return rc;
+        memcpy(ctx->a_ids.h + ioff, ids, (size_t)n_blocks * 4);
+        CK(ps::launch_upload(ctx->a_ids.d + ioff, ctx->a_ids.hd + ioff, (size_t)round_up((int64_t)n_blocks * 4, 16),
+                             ctx->compute));
+        ctx->launches++;
+        ctx->ids_cache.assign(ids, ids + n_blocks);
+        ctx->ids_cache_off = ioff;
+    }
     const int32_t* d_ids = (const int32_t*)(ctx->a_ids.d + ioff);
     const int64_t bytes = (int64_t)n_blocks * ctx->layer_block_bytes;
     if (direction == 0) {
