@@ -362,7 +362,10 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
                         dtype=torch.float32).to(torch.bfloat16)
         out = torch.zeros_like(q)
         reload_bytes = sum(sh.blocks_for(w.ctx_lens[r]) for r in w.victims) * sh.block_bytes
-        budgets = w.budgets + [-1] if mode == "pipelined" else [256 * wl.MiB, -1]
+        # "adaptive": B_copy chosen every step by ps_copy_budget (Section 4.3) from the measured decode time per
+        # token and the measured copy time per block (no latency budget: case 2 of the procedure)
+        budgets = w.budgets + ["adaptive", -1] if mode == "pipelined" else [256 * wl.MiB, -1]
+        model = None
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         if mode == "pipelined":
             for _ in range(3):
@@ -371,6 +374,11 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
             res["attn_gbs"] = rf["gbs"]
             res["attn_frac_of_hbm"] = rf["gbs"] / peaks_hbm
             res["attn_us_per_layer"] = rf["us_per_layer"]
+            link_gbs = B.ps_link_probe(256 << 20, 0, 5)
+            model = {"a_d": rf["step_us"] / sum(w.ctx_lens[r] for r in batch), "b_d": 0.0, "t_c": 0.0,
+                     "t_block": sh.block_bytes / (link_gbs * 1e3) * (1.0 + 1.0 / sh.num_layers), "t_budget": 1e12}
+            res["adaptive_model"] = dict(model, note="a_d: measured decode step us per KV token; t_block: block bytes / "
+                                         "measured H2D rate, plus one layer chunk of pipeline fill")
         for r in w.victims:
             assert lib.swap_out(r) == 0, lib.last_error()
         assert lib.sync() == 0
@@ -380,12 +388,23 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
                 assert lib.swap_in_begin(r) == 0
             torch.cuda.synchronize()
             e0.record()
+            chosen = []
+
+            def step_budget(reqs_now):
+                if budget != "adaptive":
+                    return budget
+                rc, blocks, nbytes, case = lib.copy_budget(reqs_now, **model)
+                assert rc == 0, lib.last_error()
+                chosen.append(nbytes)
+                return nbytes
+
             while any(lib.missing_blocks(r) for r in w.victims):
-                rc, _, _ = lib.step(None, None, [], budget)
+                rc, _, _ = lib.step(None, None, [], step_budget(all_reqs))
                 assert rc == 0, lib.last_error()
                 assert lib.sync() == 0
             e1.record(); e1.synchronize()
             alone_ms = e0.elapsed_time(e1)
+            chosen.clear()
             for r in w.victims:
                 assert lib.swap_out(r) == 0
             assert lib.sync() == 0
@@ -398,7 +417,7 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
             torch.cuda.synchronize()
             e0.record()
             while True:
-                rc, mask, st = lib.step(q, out, all_reqs, budget)
+                rc, mask, st = lib.step(q, out, all_reqs, step_budget(all_reqs))
                 assert rc == 0, lib.last_error()
                 stream.synchronize()
                 masks.append(mask)
@@ -421,11 +440,14 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
             without_ms = e0.elapsed_time(e1)
             n_steps = len(masks)
             hidden = 1.0 - max(0.0, with_ms - without_ms) / alone_ms if alone_ms > 0 else None
-            key = f"{mode}_{'unlimited' if budget < 0 else str(budget // wl.MiB) + 'MiB'}"
+            key = f"{mode}_" + ("adaptive" if budget == "adaptive" else "unlimited" if budget < 0
+                                else str(budget // wl.MiB) + "MiB")
             res[key] = {"steps": n_steps, "step_us_with_reload": with_ms / n_steps * 1e3,
                         "step_us_no_reload": without_ms / n_steps * 1e3,
                         "reload_alone_ms": alone_ms, "reload_alone_gbs": reload_bytes / alone_ms / 1e6,
                         "reload_under_decode_gbs": reload_bytes / with_ms / 1e6, "hidden_frac": hidden}
+            if budget == "adaptive":
+                res[key]["chosen_budget_mib_per_step"] = [round(c / wl.MiB, 1) for c in chosen]
             for r in w.victims:
                 assert lib.swap_out(r) == 0
             assert lib.sync() == 0

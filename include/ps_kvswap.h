@@ -299,6 +299,38 @@ int32_t ps_decode_attn_static(const void* kpool, const void* vpool, const void* 
 int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs,
                 int32_t batch, int64_t copy_budget_bytes, int32_t* decoded_mask, ps_step_stats* stats);
 
+/* ---- adaptive copy budget (Section 4.3 "Adaptive Copy-Budget Control") -------------------- */
+
+/* Latency model of one decode step and of the host link, in microseconds (Section 4.1: a decode request
+ * costs a_d * l_kv + b_d, a batch the sum over its requests plus the constant t_c; Section 4.3: t_block
+ * is the profiled copy time of one block, all layers). */
+typedef struct ps_budget_model {
+    double a_d_us_per_token;  /* a_d */
+    double b_d_us;            /* b_d */
+    double t_c_us;            /* t_c */
+    double t_block_us;        /* t_block */
+    double t_budget_us;       /* the scheduler's latency budget for this step */
+} ps_budget_model;
+
+/* Chooses B_copy, the number of blocks to reload in the coming step, by the paper's decision procedure:
+ *   T_fwd_min   = estimated step time with every queued reload complete (all of `reqs` decode),
+ *   T_trans_max = (missing blocks over the reload queue) * t_block;
+ *   case 1  T_fwd_min > t_budget        : B_copy = floor(t_budget / t_block)
+ *   case 2  T_fwd_min <= t_budget and
+ *     2i    T_fwd_min > T_trans_max     : B_copy = all missing blocks
+ *     2ii   otherwise                   : binary search for the largest B with
+ *                                         B * t_block <= estimated step time after copying B blocks,
+ * where "after copying B blocks" means: the requests of `reqs` that are resident now, plus those the
+ * reload queue completes when it consumes B blocks in order.  (This library's path has no recomputation,
+ * so that estimate grows with B; the search is valid because a block takes longer to copy than to
+ * attend to: t_block > a_d * block_size is required in case 2ii, else PS_ERR_INVALID.)
+ *   reqs          : host array, the decode batch of the coming step (as for ps_step)
+ *   budget_blocks : B_copy;  budget_bytes : B_copy * bytes of a block over all layers, for ps_step
+ *   which_case    : 1, 21 or 22 (may be NULL)
+ * Decisions are taken in double precision.  Errors: PS_ERR_INVALID (non-positive t_block, negative terms). */
+int32_t ps_copy_budget(ps_ctx* ctx, const int64_t* reqs, int32_t batch, const ps_budget_model* model,
+                       int64_t* budget_blocks, int64_t* budget_bytes, int32_t* which_case);
+
 /* ---- completion ------------------------------------------------------------------------- */
 
 /* Non-blocking: reaps finished offloads (in issue order), releases host images of finished

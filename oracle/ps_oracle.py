@@ -17,6 +17,8 @@ What it follows (ProServe, Section 4.3 "Efficient Block Management", and Appendi
   the residual budget ("Put it Together", Alg. 1 lines 17 and 22-25).  -> `step_plan`, `step`.
   The beta admission test of that paragraph depends on the scheduler's computable-token count and
   is not modelled: a partial copy is always allowed and a request decodes only once complete.
+* The number of blocks to reload per step, B_copy, follows the three-case procedure of "Adaptive
+  Copy-Budget Control" with the decode latency model of Section 4.1.  -> `copy_budget`.
 * The computation the reload overlaps with is the decode forward; its KV-consuming part is
   attention over the paged cache.  The paper gives no formula; the textbook definition
   softmax(q K^T / sqrt(d)) V is used, in float64, over KV gathered through the block table.
@@ -302,6 +304,61 @@ class PsOracle:
                     o, _ = self.decode_attn(l, q_bits[l][live], [reqs[i] for i in live])
                     out[l, live] = o
         return plan, mask, out
+
+    # ------------------------------------------------------------------ adaptive copy budget
+    def step_latency_after(self, reqs: Sequence[int], n_blocks: int, a_d: float, b_d: float, t_c: float) -> float:
+        """Estimated time of the decode step (Section 4.1: sum over decode requests of a_d * l_kv + b_d, plus
+        t_c) if the reload queue consumed `n_blocks` blocks in order first: the requests of `reqs` that are
+        resident now decode, and so do the queued ones whose last missing block is among those blocks."""
+        done = set()
+        left = n_blocks
+        for q in self.in_fifo:
+            miss = self.missing_blocks(q)
+            if miss == 0:
+                continue
+            if miss > left:
+                break
+            left -= miss
+            done.add(q)
+        t = t_c
+        seen = set()
+        for q in reqs:
+            r = self.reqs.get(q)
+            if r is None or q in seen:
+                continue
+            seen.add(q)
+            if r.state == ST_RESIDENT or (r.state == ST_SWAPPING_IN and q in done):
+                t += a_d * r.n_tokens + b_d
+        return t
+
+    def copy_budget(self, reqs: Sequence[int], a_d: float, b_d: float, t_c: float, t_block: float,
+                    t_budget: float) -> Tuple[int, int]:
+        """B_copy by the decision procedure of Section 4.3, "Adaptive Copy-Budget Control".
+
+        T_fwd_min: estimated forward time with all host-resident blocks of the queue copied;
+        T_trans_max = sum of b_miss * t_block.  (1) T_fwd_min > t_budget: floor(t_budget / t_block).
+        (2) otherwise, (i) T_fwd_min > T_trans_max: all missing blocks; (ii) else binary search for the largest
+        B_copy whose transfer time does not exceed the estimated batch latency.  Reading for this decode-only
+        path (no recomputation): the batch latency after copying B blocks is `step_latency_after`, which
+        grows with B, slower than the transfer time as long as t_block > a_d * s_blk.
+        Returns (B_copy, case) with case 1, 21 or 22.
+        """
+        b_missing = sum(self.missing_blocks(q) for q in self.in_fifo)
+        t_fwd_min = self.step_latency_after(reqs, b_missing, a_d, b_d, t_c)
+        t_trans_max = b_missing * t_block
+        if t_fwd_min > t_budget:
+            return int(math.floor(t_budget / t_block)), 1
+        if t_fwd_min > t_trans_max:
+            return b_missing, 21
+        assert t_block > a_d * self.S
+        lo, hi = 0, b_missing
+        while lo < hi:
+            mid = lo + (hi - lo + 1) // 2
+            if mid * t_block <= self.step_latency_after(reqs, mid, a_d, b_d, t_c):
+                lo = mid
+            else:
+                hi = mid - 1
+        return lo, 22
 
     # ------------------------------------------------------------------ attention
     def gather_kv(self, layer: int, req: int) -> Tuple[np.ndarray, np.ndarray]:

@@ -30,7 +30,7 @@ EXPORTS = [
     "ps_num_free_blocks", "ps_swap_out", "ps_host_image", "ps_swap_in_begin", "ps_swap_in_cancel",
     "ps_swap_in_layer", "ps_missing_blocks", "ps_decode_attn", "ps_step", "ps_poll", "ps_sync",
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
-    "ps_decode_attn_static",
+    "ps_decode_attn_static", "ps_copy_budget",
 ]
 
 
@@ -68,6 +68,11 @@ class PsProfile(C.Structure):
 
     def as_dict(self):
         return {k: getattr(self, k) for k, _ in self._fields_}
+
+
+class PsBudgetModel(C.Structure):
+    _fields_ = [("a_d_us_per_token", C.c_double), ("b_d_us", C.c_double), ("t_c_us", C.c_double),
+                ("t_block_us", C.c_double), ("t_budget_us", C.c_double)]
 
 
 class PsTraceSpan(C.Structure):
@@ -122,6 +127,7 @@ def load() -> C.CDLL:
         "ps_copy_blocks": (i32, [vp, i32, p32, i32, vp, i32]),
         "ps_trace": (i32, [vp, i32]),
         "ps_trace_read": (i32, [vp, C.POINTER(PsTraceSpan), i32, p32]),
+        "ps_copy_budget": (i32, [vp, p64, i32, C.POINTER(PsBudgetModel), p64, p64, p32]),
         "ps_decode_attn_static": (i32, [vp, vp, vp, vp, vp, vp, i32, p32, i32, i32, i32, i32, i32, i32, i32, vp, vp,
                                         C.c_char_p, i32]),
     }
@@ -296,6 +302,14 @@ class KVSwap:
                               C.c_void_p(out_all.data_ptr()) if out_all is not None else None, arr, len(reqs),
                               copy_budget_bytes, mask, C.byref(st))
         return rc, list(mask[: len(reqs)]), st.as_dict()
+
+    def copy_budget(self, reqs: Sequence[int], *, a_d: float, b_d: float, t_c: float, t_block: float, t_budget: float):
+        """Adaptive copy budget for the coming step: (status, blocks, bytes, case 1 / 21 / 22); times in us."""
+        m = PsBudgetModel(a_d, b_d, t_c, t_block, t_budget)
+        blocks, nbytes, case = C.c_int64(), C.c_int64(), C.c_int32()
+        rc = self.lib.ps_copy_budget(self.h, _i64_array(reqs), len(reqs), C.byref(m), C.byref(blocks), C.byref(nbytes),
+                                     C.byref(case))
+        return rc, blocks.value, nbytes.value, case.value
 
     # ---- completion
     def poll(self) -> int:
