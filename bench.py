@@ -455,6 +455,42 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
     return res
 
 
+def proactive_offload_leg(torch, B, lib, w, n_off=16):
+    """Time from eviction to reclaimable blocks, on demand and after proactive incremental offloading
+    (Section 4.3: a copy for every n_off newly filled blocks, done in the background before eviction)."""
+    sh = w.shape
+
+    def evict_and_wait():
+        t0 = time.perf_counter()
+        for r in w.victims:
+            assert lib.swap_out(r) == 0, lib.last_error()
+        assert lib.sync() == 0, lib.last_error()
+        return (time.perf_counter() - t0) * 1e3
+
+    def reload_all():
+        for r in w.victims:
+            assert lib.swap_in_begin(r) == 0, lib.last_error()
+        rc, _, _ = lib.step(None, None, [], -1)
+        assert rc == 0 and lib.sync() == 0, lib.last_error()
+
+    on_demand_ms = evict_and_wait()
+    reload_all()
+    copied = 0
+    t0 = time.perf_counter()
+    for r in w.victims:
+        rc, n = lib.offload_progress(r, n_off)
+        assert rc == 0, lib.last_error()
+        copied += n
+    assert lib.sync() == 0
+    background_ms = (time.perf_counter() - t0) * 1e3
+    tail_ms = evict_and_wait()
+    reload_all()
+    total = sum(sh.blocks_for(w.ctx_lens[r]) for r in w.victims)
+    return {"n_off": n_off, "victim_blocks": total, "blocks_copied_ahead": copied,
+            "evict_to_reclaim_ms_on_demand": on_demand_ms, "evict_to_reclaim_ms_after_proactive": tail_ms,
+            "background_copy_ms": background_ms}
+
+
 def kernel_rates(torch, B, lib, sh, nb, n_blocks=2048, iters=20):
     """Gather / scatter kernels alone (no host link): payload read once + written once per launch.
 
@@ -626,6 +662,8 @@ def run_gpu(args):
             "decode_step_us_no_swap": rf_res["step_us"],
             "link": link,
         }
+    if rank == 0:
+        result["proactive_offload"] = proactive_offload_leg(torch, B, lib, w)
     lib.destroy()
     del lib
     if rank == 0:

@@ -185,12 +185,37 @@ int32_t ps_num_free_blocks(ps_ctx* ctx, int32_t* out);
  * enqueued on the compute stream.  Returns at once; the request is SWAPPING_OUT and still owns
  * its blocks.  When a later ps_poll / ps_step / ps_sync finds the transfer complete (offloads
  * complete in issue order) the blocks are pushed back to the pool and the state becomes HOST.
+ * Blocks already covered by ps_offload_progress are not copied again.
  * Errors: PS_ERR_STATE, PS_ERR_HOST_NOMEM, PS_ERR_INVALID, PS_ERR_CUDA. */
 int32_t ps_swap_out(ps_ctx* ctx, int64_t req);
 
+/* Proactive incremental offloading (Section 4.3 "Asynchronous Offloading": a copy is triggered for every
+ * n_off newly generated blocks of a request, with a smaller n_off for requests that are more likely to be
+ * preempted).  If the RESIDENT request has at least n_off blocks that are completely filled
+ * (n_tokens / block_size) and not yet offloaded, the largest whole number of groups of n_off such blocks
+ * is copied to the host as a new image segment, asynchronously and ordered after the work already
+ * enqueued on the compute stream; the request stays RESIDENT and keeps decoding and growing.  Filled
+ * blocks must not be rewritten afterwards (decode only appends).  *issued_blocks (may be NULL) = blocks
+ * issued by this call, possibly 0.  A later ps_swap_out then only offloads the remaining tail (the paper
+ * drops that tail and recomputes it on resume; this path has no recomputation, so it is copied), which
+ * shortens the time until the device blocks can be reclaimed.  Which n_off to use is the caller's policy.
+ * Errors: PS_ERR_STATE, PS_ERR_INVALID, PS_ERR_HOST_NOMEM, PS_ERR_CUDA. */
+int32_t ps_offload_progress(ps_ctx* ctx, int64_t req, int32_t n_off, int32_t* issued_blocks);
+
+/* b_host of Section 4.3 for one request: blocks whose offload has been issued, and blocks whose copy has
+ * been seen complete (as of the last ps_poll / ps_step / ps_sync).  Either pointer may be NULL. */
+int32_t ps_host_blocks(ps_ctx* ctx, int64_t req, int32_t* issued, int32_t* on_host);
+
 /* Host address and size of a HOST / SWAPPING_IN request's image (valid until the reload completes
- * or the request is freed).  For checks; the bytes are final only once the state is HOST. */
+ * or the request is freed).  For checks; the bytes are final only once the state is HOST.
+ * PS_ERR_STATE when the image consists of several segments (proactive offloading). */
 int32_t ps_host_image(ps_ctx* ctx, int64_t req, void** ptr, int64_t* bytes);
+
+/* Segment `index` of a request's host image: logical blocks [*blk_lo, *blk_hi) in the layout
+ * [num_layers][blk_hi - blk_lo][2 (K,V)][slab].  *n_segments receives the number of segments; index -1
+ * asks for the count only.  Any out pointer may be NULL. */
+int32_t ps_host_segment(ps_ctx* ctx, int64_t req, int32_t index, void** ptr, int64_t* bytes, int32_t* blk_lo,
+                        int32_t* blk_hi, int32_t* n_segments);
 
 /* ---- swap-in (Section 4.3 "Pipelined Reloading"; App. B: per-layer-chunk events) ---------- */
 

@@ -10,6 +10,9 @@ What it follows (ProServe, Section 4.3 "Efficient Block Management", and Appendi
 * Eviction spills a request's KV blocks to host memory instead of dropping them; the device
   blocks can be reclaimed only after the transfer has completed ("Asynchronous Offloading").
   -> `swap_out` copies the blocks byte for byte into a host image; `reap` gives the blocks back.
+* Offloading can also run ahead of eviction: a copy for every n_off newly filled blocks of a request
+  ("Asynchronous Offloading").  -> `offload_progress`; `swap_out` then copies only the rest.  (The paper
+  drops the not-yet-copied tail at eviction and recomputes it; without recomputation it is copied.)
 * A readmitted request gets its KV restored layer by layer ("Pipelined Reloading"; Appendix B:
   one completion event per layer chunk).  -> `swap_in_begin`, `swap_in_layer`.
 * A per-step host-to-device copy budget B_copy (in blocks) is consumed in queue order at request
@@ -62,7 +65,7 @@ def bf16_bits_to_f64(bits: np.ndarray) -> np.ndarray:
 
 
 class _Req:
-    __slots__ = ("n_tokens", "table", "state", "image", "image_bytes", "layer_done", "old_table")
+    __slots__ = ("n_tokens", "table", "state", "image", "image_bytes", "layer_done", "old_table", "segs")
 
     def __init__(self):
         self.n_tokens = 0
@@ -72,6 +75,9 @@ class _Req:
         self.image_bytes = 0
         self.layer_done: List[int] = []
         self.old_table: List[int] = []
+        # host image: segments (blk_lo, blk_hi, array [L][hi - lo][2][S][Hkv][D] or None without pools);
+        # `image` is the array of the only segment when there is exactly one
+        self.segs: List[Tuple[int, int, Optional[np.ndarray]]] = []
 
 
 class PsOracle:
@@ -136,8 +142,7 @@ class PsOracle:
             return ERR_BUSY
         if r.state == ST_RESIDENT:
             self.free.extend(r.table)            # pushed in table order: last entry ends on top
-        else:
-            self._release_image(r)
+        self._release_image(r)
         del self.reqs[req]
         return OK
 
@@ -156,6 +161,48 @@ class PsOracle:
         self.host_used -= r.image_bytes
         r.image_bytes = 0
         r.image = None
+        r.segs = []
+
+    def _host_issued(self, r: _Req) -> int:
+        return r.segs[-1][1] if r.segs else 0
+
+    def _offload_segment(self, r: _Req, lo: int, hi: int) -> int:
+        """Byte-for-byte copy of logical blocks [lo, hi), every layer, into a new image segment."""
+        nbytes = self._image_bytes(hi - lo)
+        if self.host_pool_bytes is not None and self.host_used + nbytes > self.host_pool_bytes:
+            return ERR_HOST_NOMEM
+        r.image_bytes += nbytes
+        self.host_used += nbytes
+        img = None
+        if self.K is not None:
+            img = np.empty((self.L, hi - lo, 2, self.S, self.Hkv, self.D), dtype=np.uint16)
+            for l in range(self.L):
+                for j in range(lo, hi):
+                    img[l, j - lo, 0] = self.K[l, r.table[j]]
+                    img[l, j - lo, 1] = self.V[l, r.table[j]]
+        r.segs.append((lo, hi, img))
+        r.image = img if len(r.segs) == 1 else None
+        return OK
+
+    def offload_progress(self, req: int, n_off: int):
+        """Proactive incremental offloading ("Asynchronous Offloading"): a copy for every n_off newly filled
+        blocks.  Copies the largest whole number of groups of n_off completely filled, not yet offloaded
+        blocks; the request stays resident.  Returns (status, blocks copied)."""
+        r = self.reqs.get(req)
+        if n_off <= 0 or r is None:
+            return ERR_INVALID, 0
+        if r.state != ST_RESIDENT:
+            return ERR_STATE, 0
+        lo = self._host_issued(r)
+        groups = (r.n_tokens // self.S - lo) // n_off
+        if groups <= 0:
+            return OK, 0
+        rc = self._offload_segment(r, lo, lo + groups * n_off)
+        return rc, (groups * n_off if rc == OK else 0)
+
+    def host_blocks(self, req: int) -> int:
+        """b_host of Section 4.3: blocks of the request that have a copy on host."""
+        return self._host_issued(self.reqs[req])
 
     def swap_out(self, req: int) -> int:
         """Spill the request's blocks to a host image; blocks stay owned until `reap`."""
@@ -165,17 +212,11 @@ class PsOracle:
         if r.state != ST_RESIDENT:
             return ERR_STATE
         n = len(r.table)
-        if self.host_pool_bytes is not None and self.host_used + self._image_bytes(n) > self.host_pool_bytes:
-            return ERR_HOST_NOMEM
-        r.image_bytes = self._image_bytes(n)
-        self.host_used += r.image_bytes
-        if self.K is not None:
-            img = np.empty((self.L, n, 2, self.S, self.Hkv, self.D), dtype=np.uint16)
-            for l in range(self.L):
-                for j, b in enumerate(r.table):
-                    img[l, j, 0] = self.K[l, b]
-                    img[l, j, 1] = self.V[l, b]
-            r.image = img
+        lo = self._host_issued(r)
+        if lo < n or not r.segs:                 # what proactive offloading has not covered goes out now
+            rc = self._offload_segment(r, lo, n)
+            if rc != OK:
+                return rc
         r.state = ST_SWAPPING_OUT
         self.out_fifo.append(req)
         return OK
@@ -207,6 +248,11 @@ class PsOracle:
         r.layer_done = [0] * self.L
         r.state = ST_SWAPPING_IN
         self.in_fifo.append(req)
+        if n == 0:                               # nothing to restore: resident at once
+            r.state = ST_RESIDENT
+            self._release_image(r)
+            r.old_table = []
+            self.in_fifo.remove(req)
         return OK
 
     def swap_in_cancel(self, req: int) -> int:
@@ -237,8 +283,9 @@ class PsOracle:
         if self.K is not None:
             for j in range(blk_lo, blk_hi):
                 b = r.table[j]
-                self.K[layer, b] = r.image[layer, j, 0]
-                self.V[layer, b] = r.image[layer, j, 1]
+                lo, hi, img = next(sg for sg in r.segs if sg[0] <= j < sg[1])
+                self.K[layer, b] = img[layer, j - lo, 0]
+                self.V[layer, b] = img[layer, j - lo, 1]
         r.layer_done[layer] = blk_hi
         if all(d == n for d in r.layer_done):
             r.state = ST_RESIDENT

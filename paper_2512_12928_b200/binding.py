@@ -30,7 +30,7 @@ EXPORTS = [
     "ps_num_free_blocks", "ps_swap_out", "ps_host_image", "ps_swap_in_begin", "ps_swap_in_cancel",
     "ps_swap_in_layer", "ps_missing_blocks", "ps_decode_attn", "ps_step", "ps_poll", "ps_sync",
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
-    "ps_decode_attn_static", "ps_copy_budget",
+    "ps_decode_attn_static", "ps_copy_budget", "ps_offload_progress", "ps_host_blocks", "ps_host_segment",
 ]
 
 
@@ -127,6 +127,9 @@ def load() -> C.CDLL:
         "ps_copy_blocks": (i32, [vp, i32, p32, i32, vp, i32]),
         "ps_trace": (i32, [vp, i32]),
         "ps_trace_read": (i32, [vp, C.POINTER(PsTraceSpan), i32, p32]),
+        "ps_offload_progress": (i32, [vp, i64, i32, p32]),
+        "ps_host_blocks": (i32, [vp, i64, p32, p32]),
+        "ps_host_segment": (i32, [vp, i64, i32, C.POINTER(vp), p64, p32, p32, p32]),
         "ps_copy_budget": (i32, [vp, p64, i32, C.POINTER(PsBudgetModel), p64, p64, p32]),
         "ps_decode_attn_static": (i32, [vp, vp, vp, vp, vp, vp, i32, p32, i32, i32, i32, i32, i32, i32, i32, vp, vp,
                                         C.c_char_p, i32]),
@@ -271,6 +274,29 @@ class KVSwap:
         ptr, nbytes = C.c_void_p(), C.c_int64()
         self._ck(self.lib.ps_host_image(self.h, req, C.byref(ptr), C.byref(nbytes)), "ps_host_image")
         return ptr.value or 0, nbytes.value
+
+    def offload_progress(self, req: int, n_off: int):
+        """Proactive offload of whole groups of n_off filled blocks: (status, blocks issued)."""
+        n = C.c_int32()
+        rc = self.lib.ps_offload_progress(self.h, req, n_off, C.byref(n))
+        return rc, n.value
+
+    def host_blocks(self, req: int) -> Tuple[int, int]:
+        a, b = C.c_int32(), C.c_int32()
+        self._ck(self.lib.ps_host_blocks(self.h, req, C.byref(a), C.byref(b)), "ps_host_blocks")
+        return a.value, b.value
+
+    def host_segments(self, req: int):
+        """List of (address, bytes, blk_lo, blk_hi) of the request's image segments."""
+        n = C.c_int32()
+        self._ck(self.lib.ps_host_segment(self.h, req, -1, None, None, None, None, C.byref(n)), "ps_host_segment")
+        out = []
+        for i in range(n.value):
+            ptr, nbytes, lo, hi = C.c_void_p(), C.c_int64(), C.c_int32(), C.c_int32()
+            self._ck(self.lib.ps_host_segment(self.h, req, i, C.byref(ptr), C.byref(nbytes), C.byref(lo), C.byref(hi),
+                                              None), "ps_host_segment")
+            out.append((ptr.value or 0, nbytes.value, lo.value, hi.value))
+        return out
 
     def swap_in_begin(self, req: int) -> int:
         return self.lib.ps_swap_in_begin(self.h, req)

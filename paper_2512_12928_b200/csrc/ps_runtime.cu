@@ -40,7 +40,16 @@ struct Req {
     int32_t n_tokens = 0;
     std::vector<int32_t> table;
     int32_t state = PS_REQ_RESIDENT;
-    int64_t img_off = -1, img_bytes = 0;
+    // Host image: one segment per offload issued for the request.  A segment covers logical blocks [lo, hi)
+    // in the layer-major layout [L][hi - lo][K,V][slab].  On-demand offloading makes one segment; proactive
+    // offloading (ps_offload_progress) adds segments as the request grows, ps_swap_out adds the last.
+    struct Seg {
+        int32_t lo, hi;
+        int64_t off, bytes;
+        uint64_t ticket;  // s_d2h ticket after the segment's last copy
+    };
+    std::vector<Seg> segs;
+    int32_t host_issued = 0;          // blocks covered by segs
     std::vector<int32_t> layer_done;  // blocks issued per layer while SWAPPING_IN
     uint64_t out_ticket = 0;          // s_d2h ticket after the last segment
     bool gated = false;               // RESIDENT but reload copies not yet seen complete
@@ -444,12 +453,19 @@ int32_t issue_reload_layer(ps_ctx* ctx, int32_t layer, const std::vector<PlanEnt
         ids.clear();
         while (i < plan.size() && used < cap) {
             Req& r = ctx->reqs[plan[i].req];
-            const int64_t n_blk = (int64_t)r.table.size();
             const int64_t take = std::min<int64_t>(plan[i].hi - lo, cap - used);
-            if (take > 0) {
-                const char* src = ctx->host_pool + r.img_off + ((int64_t)layer * n_blk + lo) * Bl;
-                ProfScope prof(ctx, kProfH2D, ctx->s_h2d, take * Bl, layer);
-                CK(cudaMemcpyAsync(sp + used * Bl, src, (size_t)(take * Bl), cudaMemcpyHostToDevice, ctx->s_h2d));
+            // one contiguous host range per (segment, layer): a run of blocks is cut at segment borders
+            for (int64_t j = lo, done = 0; done < take;) {
+                const Req::Seg* sg = nullptr;
+                for (const Req::Seg& c : r.segs)
+                    if (j >= c.lo && j < c.hi) sg = &c;
+                if (sg == nullptr) return ctx->fail(PS_ERR_STATE, "reload: block outside the host image");
+                const int64_t piece = std::min<int64_t>(take - done, sg->hi - j);
+                const char* src = ctx->host_pool + sg->off + ((int64_t)layer * (sg->hi - sg->lo) + (j - sg->lo)) * Bl;
+                ProfScope prof(ctx, kProfH2D, ctx->s_h2d, piece * Bl, layer);
+                CK(cudaMemcpyAsync(sp + (used + done) * Bl, src, (size_t)(piece * Bl), cudaMemcpyHostToDevice, ctx->s_h2d));
+                j += piece;
+                done += piece;
             }
             for (int64_t j = lo; j < lo + take; ++j) ids.push_back(r.table[(size_t)j]);
             used += take;
@@ -492,13 +508,15 @@ int32_t note_layer_issued(ps_ctx* ctx, int64_t id, Req& r, int32_t layer, int32_
         }
     int32_t rc = tracker_mark(ctx, ctx->t_scatter, &r.in_ticket);
     if (rc != PS_OK) return rc;
-    ctx->img_release.push_back({r.in_ticket, {r.img_off, r.img_bytes}});
-    r.img_off = -1;
-    r.img_bytes = 0;
-    if (ctx->bk) {
-        ctx->hpool.release(ctx->img_release.back().second.first, ctx->img_release.back().second.second);
-        ctx->img_release.pop_back();
-    } else {
+    for (const Req::Seg& sg : r.segs) {
+        if (ctx->bk)
+            ctx->hpool.release(sg.off, sg.bytes);
+        else
+            ctx->img_release.push_back({r.in_ticket, {sg.off, sg.bytes}});
+    }
+    r.segs.clear();
+    r.host_issued = 0;
+    if (!ctx->bk) {
         r.gated = true;
         ctx->gated_reqs.push_back(id);
     }
@@ -1105,10 +1123,15 @@ int32_t ps_kv_free(ps_ctx* ctx, int64_t req) {
             if (rc != PS_OK) return rc;
             if (r.gated) return ctx->fail(PS_ERR_BUSY, "ps_kv_free: reload copies still in flight");
         }
+        if (!r.segs.empty()) {  // proactive copies: their transfers must have ended before the image goes
+            int32_t rc = do_poll(ctx, nullptr);
+            if (rc != PS_OK) return rc;
+            if (r.segs.back().ticket > ctx->t_d2h.done)
+                return ctx->fail(PS_ERR_BUSY, "ps_kv_free: proactive offload still in flight");
+        }
         push_table(ctx, r.table);
-    } else {
-        ctx->hpool.release(r.img_off, r.img_bytes);
     }
+    for (const Req::Seg& sg : r.segs) ctx->hpool.release(sg.off, sg.bytes);
     ctx->reqs.erase(it);
     ctx->table_epoch++;
     return PS_OK;
@@ -1136,13 +1159,11 @@ int32_t ps_num_free_blocks(ps_ctx* ctx, int32_t* out) {
     return PS_OK;
 }
 
-int32_t ps_swap_out(ps_ctx* ctx, int64_t req) {
-    if (!ctx) return PS_ERR_INVALID;
-    auto it = ctx->reqs.find(req);
-    if (it == ctx->reqs.end()) return ctx->fail(PS_ERR_INVALID, "ps_swap_out: unknown request");
-    Req& r = it->second;
-    if (r.state != PS_REQ_RESIDENT) return ctx->fail(PS_ERR_STATE, "ps_swap_out: request is not resident");
-    const int64_t n_blk = (int64_t)r.table.size();
+// Starts the offload of logical blocks [lo, hi) of a request as a new image segment: gather through the
+// table into staging slots, slot by slot to the host.  Ordered after everything already enqueued on the
+// compute stream (and after the scatters of a reload that is still landing).
+static int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi) {
+    const int64_t n_blk = hi - lo;
     const int64_t bytes = n_blk * ctx->block_bytes;
     int64_t off = ctx->hpool.alloc(bytes);
     if (off < 0) {  // images of reloads that have landed since the last poll may still be held
@@ -1150,11 +1171,9 @@ int32_t ps_swap_out(ps_ctx* ctx, int64_t req) {
         if (rc != PS_OK) return rc;
         off = ctx->hpool.alloc(bytes);
     }
-    if (off < 0) return ctx->fail(PS_ERR_HOST_NOMEM, "ps_swap_out: host pool cannot hold the image");
+    if (off < 0) return ctx->fail(PS_ERR_HOST_NOMEM, "host pool cannot hold the image");
 
     if (!ctx->bk && n_blk > 0) {
-        // gather must see everything the compute stream has been asked to write, and, for a request
-        // whose reload is still landing, every scatter
         cudaError_t e = cudaEventRecord(ctx->e_mark2, ctx->compute);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_gather, ctx->e_mark2, 0);
         if (e == cudaSuccess && r.gated) {
@@ -1168,9 +1187,8 @@ int32_t ps_swap_out(ps_ctx* ctx, int64_t req) {
             ctx->hpool.release(off, bytes);
             return rc;
         }
-        memcpy(ctx->a_gather.h + toff, r.table.data(), (size_t)n_blk * 4);
+        memcpy(ctx->a_gather.h + toff, r.table.data() + lo, (size_t)n_blk * 4);
         auto bail = [&](cudaError_t ce, const char* what) {
-            // nothing can be undone once work is enqueued: the request stays SWAPPING_OUT-less and resident
             ctx->hpool.release(off, bytes);
             return ctx->fail_cuda(ce, what);
         };
@@ -1208,13 +1226,61 @@ int32_t ps_swap_out(ps_ctx* ctx, int64_t req) {
             ctx->out_used[slot] = true;
         }
     }
-    r.img_off = off;
-    r.img_bytes = bytes;
-    r.state = PS_REQ_SWAPPING_OUT;
-    int32_t rc = tracker_mark(ctx, ctx->t_d2h, &r.out_ticket);
+    Req::Seg sg{lo, hi, off, bytes, 0};
+    int32_t rc = tracker_mark(ctx, ctx->t_d2h, &sg.ticket);
     if (rc != PS_OK) return rc;
+    r.segs.push_back(sg);
+    r.host_issued = hi;
+    return PS_OK;
+}
+
+int32_t ps_swap_out(ps_ctx* ctx, int64_t req) {
+    if (!ctx) return PS_ERR_INVALID;
+    auto it = ctx->reqs.find(req);
+    if (it == ctx->reqs.end()) return ctx->fail(PS_ERR_INVALID, "ps_swap_out: unknown request");
+    Req& r = it->second;
+    if (r.state != PS_REQ_RESIDENT) return ctx->fail(PS_ERR_STATE, "ps_swap_out: request is not resident");
+    const int32_t n_blk = (int32_t)r.table.size();
+    // what proactive offloading has not covered yet (everything, without it) goes out now
+    if (r.host_issued < n_blk || r.segs.empty()) {
+        int32_t rc = offload_segment(ctx, r, r.host_issued, n_blk);
+        if (rc != PS_OK) return rc;
+    }
+    r.out_ticket = r.segs.back().ticket;  // copies complete in issue order
+    r.state = PS_REQ_SWAPPING_OUT;
     ctx->out_fifo.push_back(req);
     ctx->table_epoch++;
+    return PS_OK;
+}
+
+int32_t ps_offload_progress(ps_ctx* ctx, int64_t req, int32_t n_off, int32_t* issued_blocks) {
+    if (!ctx) return PS_ERR_INVALID;
+    if (issued_blocks) *issued_blocks = 0;
+    if (n_off <= 0) return ctx->fail(PS_ERR_INVALID, "ps_offload_progress: n_off must be positive");
+    auto it = ctx->reqs.find(req);
+    if (it == ctx->reqs.end()) return ctx->fail(PS_ERR_INVALID, "ps_offload_progress: unknown request");
+    Req& r = it->second;
+    if (r.state != PS_REQ_RESIDENT) return ctx->fail(PS_ERR_STATE, "ps_offload_progress: request is not resident");
+    const int32_t full = r.n_tokens / ctx->cfg.block_size;  // blocks that will not change any more
+    const int32_t groups = (full - r.host_issued) / n_off;
+    if (groups <= 0) return PS_OK;
+    const int32_t lo = r.host_issued, hi = lo + groups * n_off;
+    int32_t rc = offload_segment(ctx, r, lo, hi);
+    if (rc != PS_OK) return rc;
+    if (issued_blocks) *issued_blocks = hi - lo;
+    return PS_OK;
+}
+
+int32_t ps_host_blocks(ps_ctx* ctx, int64_t req, int32_t* issued, int32_t* on_host) {
+    if (!ctx) return PS_ERR_INVALID;
+    auto it = ctx->reqs.find(req);
+    if (it == ctx->reqs.end()) return ctx->fail(PS_ERR_INVALID, "ps_host_blocks: unknown request");
+    const Req& r = it->second;
+    int32_t done = 0;
+    for (const Req::Seg& sg : r.segs)
+        if (sg.ticket <= ctx->t_d2h.done) done = sg.hi;
+    if (issued) *issued = r.host_issued;
+    if (on_host) *on_host = done;
     return PS_OK;
 }
 
@@ -1223,9 +1289,30 @@ int32_t ps_host_image(ps_ctx* ctx, int64_t req, void** ptr, int64_t* bytes) {
     auto it = ctx->reqs.find(req);
     if (it == ctx->reqs.end()) return ctx->fail(PS_ERR_INVALID, "ps_host_image: unknown request");
     const Req& r = it->second;
-    if (r.img_off < 0) return ctx->fail(PS_ERR_STATE, "ps_host_image: request has no host image");
-    if (ptr) *ptr = ctx->host_pool ? (void*)(ctx->host_pool + r.img_off) : nullptr;
-    if (bytes) *bytes = r.img_bytes;
+    if (r.segs.empty()) return ctx->fail(PS_ERR_STATE, "ps_host_image: request has no host image");
+    if (r.segs.size() != 1)
+        return ctx->fail(PS_ERR_STATE, "ps_host_image: the image has several segments, use ps_host_segment");
+    if (ptr) *ptr = ctx->host_pool ? (void*)(ctx->host_pool + r.segs[0].off) : nullptr;
+    if (bytes) *bytes = r.segs[0].bytes;
+    return PS_OK;
+}
+
+int32_t ps_host_segment(ps_ctx* ctx, int64_t req, int32_t index, void** ptr, int64_t* bytes, int32_t* blk_lo,
+                        int32_t* blk_hi, int32_t* n_segments) {
+    if (!ctx) return PS_ERR_INVALID;
+    auto it = ctx->reqs.find(req);
+    if (it == ctx->reqs.end()) return ctx->fail(PS_ERR_INVALID, "ps_host_segment: unknown request");
+    const Req& r = it->second;
+    if (n_segments) *n_segments = (int32_t)r.segs.size();
+    if (index < 0 || index >= (int32_t)r.segs.size()) {
+        if (n_segments && index == -1) return PS_OK;  // count only
+        return ctx->fail(PS_ERR_INVALID, "ps_host_segment: no such segment");
+    }
+    const Req::Seg& sg = r.segs[(size_t)index];
+    if (ptr) *ptr = ctx->host_pool ? (void*)(ctx->host_pool + sg.off) : nullptr;
+    if (bytes) *bytes = sg.bytes;
+    if (blk_lo) *blk_lo = sg.lo;
+    if (blk_hi) *blk_hi = sg.hi;
     return PS_OK;
 }
 
