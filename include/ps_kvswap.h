@@ -356,6 +356,31 @@ typedef struct ps_budget_model {
 int32_t ps_copy_budget(ps_ctx* ctx, const int64_t* reqs, int32_t batch, const ps_budget_model* model,
                        int64_t* budget_blocks, int64_t* budget_bytes, int32_t* which_case);
 
+/* ---- eviction policy and partial-copy admission (Section 4.3) ----------------------------- */
+
+/* "Eviction Policy": when device memory is saturated, evict requests near the tail of the sorted queue,
+ * except those whose waiting time is close to the starvation threshold.
+ *   queue      : host array of n request ids in the scheduler's order, head (next to run) first
+ *   waited_us  : host array of n waiting times
+ *   tau_us     : the starvation threshold; near_frac in (0, 1]: "close to" means waited >= near_frac * tau
+ *   blocks_needed : device blocks to free
+ * Walks the queue from its tail and takes RESIDENT requests that hold blocks and are not close to
+ * starvation until their blocks add up to blocks_needed; writes them to victims (capacity cap) in
+ * eviction order.  *blocks_freed may end below blocks_needed when the queue does not hold enough.
+ * Chooses only; the caller evicts with ps_swap_out.  Errors: PS_ERR_INVALID. */
+int32_t ps_select_victims(ps_ctx* ctx, const int64_t* queue, int32_t n, const double* waited_us, double tau_us,
+                          double near_frac, int32_t blocks_needed, int64_t* victims, int32_t cap, int32_t* n_victims,
+                          int32_t* blocks_freed);
+
+/* "Put it Together": whether request r may be copied in this round when the residual budget b_rem does
+ * not cover its b_miss missing blocks.  A full copy (b_rem >= b_miss) is always allowed; a partial copy
+ * only if the tokens still computable for r after it, l_comp, reach the round's limit l_comp_max, or if
+ * l_comp / ((b_miss - b_rem) * s_blk) > beta (beta > 1).  *allowed = 1 or 0.  Pure arithmetic, for
+ * schedulers built on this library: ps_step itself always allows partial copies (its decode-only batch
+ * has no computable-token notion).  Errors: PS_ERR_INVALID (negative counts, s_blk <= 0, beta <= 1). */
+int32_t ps_copy_condition(int32_t l_comp, int32_t l_comp_max, int32_t b_miss, int32_t b_rem, int32_t s_blk,
+                          double beta, int32_t* allowed);
+
 /* ---- completion ------------------------------------------------------------------------- */
 
 /* Non-blocking: reaps finished offloads (in issue order), releases host images of finished

@@ -407,6 +407,26 @@ class PsOracle:
                 hi = mid - 1
         return lo, 22
 
+    # ------------------------------------------------------------------ eviction policy, partial-copy rule
+    def select_victims(self, queue: Sequence[int], waited: Sequence[float], tau: float, near_frac: float,
+                       blocks_needed: int) -> Tuple[List[int], int]:
+        """"Eviction Policy": requests near the tail of the sorted queue are evicted first, except those whose
+        waiting time is close to the starvation threshold (reading: waited >= near_frac * tau).  Returns the
+        victims in eviction order and the blocks they free (stops once blocks_needed is reached)."""
+        victims: List[int] = []
+        freed = 0
+        for pos in range(len(queue) - 1, -1, -1):
+            if freed >= blocks_needed:
+                break
+            r = self.reqs.get(queue[pos])
+            if r is None or r.state != ST_RESIDENT or not r.table or queue[pos] in victims:
+                continue
+            if waited[pos] >= near_frac * tau:
+                continue
+            victims.append(queue[pos])
+            freed += len(r.table)
+        return victims, freed
+
     # ------------------------------------------------------------------ attention
     def gather_kv(self, layer: int, req: int) -> Tuple[np.ndarray, np.ndarray]:
         """Contiguous K, V of a request for one layer: float64 [ctx][Hkv][D]."""
@@ -471,6 +491,17 @@ class PsOracle:
 # -------------------------------------------------------------------------------------------------
 # Brute-force restatements for tiny inputs (pure Python loops and floats)
 # -------------------------------------------------------------------------------------------------
+
+def copy_condition(l_comp: int, l_comp_max: int, b_miss: int, b_rem: int, s_blk: int, beta: float) -> bool:
+    """"Put it Together": all missing blocks are copied if the remaining budget covers them; otherwise partial
+    copying is enabled only when l_comp reaches the maximum computable-token limit of the round, or the ratio
+    l_comp / ((b_miss - B_rem) * s_blk) exceeds beta (beta > 1); else the request is skipped this round."""
+    if b_rem >= b_miss:
+        return True
+    if l_comp >= l_comp_max:
+        return True
+    return l_comp / ((b_miss - b_rem) * s_blk) > beta
+
 
 def _bf16_to_float(b: int) -> float:
     """One bf16 pattern to a Python float via its sign / exponent / mantissa fields."""

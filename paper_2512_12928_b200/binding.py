@@ -31,6 +31,7 @@ EXPORTS = [
     "ps_swap_in_layer", "ps_missing_blocks", "ps_decode_attn", "ps_step", "ps_poll", "ps_sync",
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
     "ps_decode_attn_static", "ps_copy_budget", "ps_offload_progress", "ps_host_blocks", "ps_host_segment",
+    "ps_select_victims", "ps_copy_condition",
 ]
 
 
@@ -130,6 +131,8 @@ def load() -> C.CDLL:
         "ps_offload_progress": (i32, [vp, i64, i32, p32]),
         "ps_host_blocks": (i32, [vp, i64, p32, p32]),
         "ps_host_segment": (i32, [vp, i64, i32, C.POINTER(vp), p64, p32, p32, p32]),
+        "ps_select_victims": (i32, [vp, p64, i32, C.POINTER(C.c_double), C.c_double, C.c_double, i32, p64, i32, p32, p32]),
+        "ps_copy_condition": (i32, [i32, i32, i32, i32, i32, C.c_double, p32]),
         "ps_copy_budget": (i32, [vp, p64, i32, C.POINTER(PsBudgetModel), p64, p64, p32]),
         "ps_decode_attn_static": (i32, [vp, vp, vp, vp, vp, vp, i32, p32, i32, i32, i32, i32, i32, i32, i32, vp, vp,
                                         C.c_char_p, i32]),
@@ -175,6 +178,13 @@ def ps_decode_attn_static(kpool, vpool, q, out, block_tables, ctx_lens: Sequence
                                       arr, batch, num_kv_heads, num_q_heads, head_dim, block_size, num_gpu_blocks,
                                       kv_split_tokens, ptr(status_word), C.c_void_p(stream or None), err, 512)
     return rc, err.value.decode()
+
+
+def ps_copy_condition(l_comp: int, l_comp_max: int, b_miss: int, b_rem: int, s_blk: int, beta: float):
+    """Partial-copy admission rule of Section 4.3: (status, allowed)."""
+    out = C.c_int32()
+    rc = load().ps_copy_condition(l_comp, l_comp_max, b_miss, b_rem, s_blk, beta, C.byref(out))
+    return rc, bool(out.value)
 
 
 def _i64_array(vals: Sequence[int]):
@@ -336,6 +346,17 @@ class KVSwap:
         rc = self.lib.ps_copy_budget(self.h, _i64_array(reqs), len(reqs), C.byref(m), C.byref(blocks), C.byref(nbytes),
                                      C.byref(case))
         return rc, blocks.value, nbytes.value, case.value
+
+    def select_victims(self, queue: Sequence[int], waited_us: Sequence[float], tau_us: float, near_frac: float,
+                       blocks_needed: int):
+        """Eviction policy: (status, victims in eviction order, blocks they free)."""
+        n = len(queue)
+        w = (C.c_double * max(n, 1))(*[float(v) for v in waited_us])
+        out = (C.c_int64 * max(n, 1))()
+        cnt, freed = C.c_int32(), C.c_int32()
+        rc = self.lib.ps_select_victims(self.h, _i64_array(queue), n, w, tau_us, near_frac, blocks_needed, out, n,
+                                        C.byref(cnt), C.byref(freed))
+        return rc, list(out[: cnt.value]), freed.value
 
     # ---- completion
     def poll(self) -> int:

@@ -1604,6 +1604,44 @@ int32_t ps_copy_budget(ps_ctx* ctx, const int64_t* reqs, int32_t batch, const ps
     return PS_OK;
 }
 
+int32_t ps_select_victims(ps_ctx* ctx, const int64_t* queue, int32_t n, const double* waited_us, double tau_us,
+                          double near_frac, int32_t blocks_needed, int64_t* victims, int32_t cap, int32_t* n_victims,
+                          int32_t* blocks_freed) {
+    if (!ctx) return PS_ERR_INVALID;
+    if (n < 0 || (n > 0 && (!queue || !waited_us)) || cap < 0 || (cap > 0 && !victims) || !n_victims ||
+        !(near_frac > 0.0 && near_frac <= 1.0) || tau_us < 0.0 || blocks_needed < 0)
+        return ctx->fail(PS_ERR_INVALID, "ps_select_victims: bad argument");
+    int32_t count = 0, freed = 0;
+    for (int32_t i = n - 1; i >= 0 && freed < blocks_needed && count < cap; --i) {
+        auto it = ctx->reqs.find(queue[i]);
+        if (it == ctx->reqs.end()) continue;
+        const Req& r = it->second;
+        if (r.state != PS_REQ_RESIDENT || r.table.empty()) continue;
+        if (waited_us[i] >= near_frac * tau_us) continue;  // close to starving: about to be promoted to the head
+        bool dup = false;
+        for (int32_t k = 0; k < count; ++k) dup |= victims[k] == queue[i];
+        if (dup) continue;
+        victims[count++] = queue[i];
+        freed += (int32_t)r.table.size();
+    }
+    *n_victims = count;
+    if (blocks_freed) *blocks_freed = freed;
+    return PS_OK;
+}
+
+int32_t ps_copy_condition(int32_t l_comp, int32_t l_comp_max, int32_t b_miss, int32_t b_rem, int32_t s_blk,
+                          double beta, int32_t* allowed) {
+    if (!allowed || l_comp < 0 || l_comp_max < 0 || b_miss < 0 || b_rem < 0 || s_blk <= 0 || !(beta > 1.0))
+        return PS_ERR_INVALID;
+    if (b_rem >= b_miss)
+        *allowed = 1;
+    else if (l_comp >= l_comp_max)
+        *allowed = 1;
+    else
+        *allowed = (double)l_comp / ((double)(b_miss - b_rem) * (double)s_blk) > beta ? 1 : 0;
+    return PS_OK;
+}
+
 int32_t ps_poll(ps_ctx* ctx, int32_t* n_reaped) {
     if (!ctx) return PS_ERR_INVALID;
     return do_poll(ctx, n_reaped);
