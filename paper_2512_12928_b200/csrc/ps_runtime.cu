@@ -134,7 +134,7 @@ struct BatchMeta {  // cached device metadata of the last prepared decode batch
     int32_t n_items = 0, n_ungated_items = 0, n_parts = 0;
     int32_t n_gated_rows = 0;
     bool any_multi = false, lane_multi[2] = {false, false};
-    bool two_lanes = false;
+    bool two_lanes = false, contended = false;
     int64_t kv_bytes_per_layer = 0;
 };
 
@@ -569,13 +569,14 @@ int32_t choose_split(const ps_ctx* ctx, int64_t total_tokens) {
 // the layer's reload event.  With want_lanes they get a work list of their own (lane 1), launched on
 // the reload-lane stream behind the event, so that the launches of the other rows never wait.
 int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::vector<char>& active,
-                      const std::vector<char>& gated, bool want_lanes) {
+                      const std::vector<char>& gated, bool want_lanes, bool contended) {
     BatchMeta& m = ctx->meta;
     // two work lists (lanes) only for the tensor-core kernel and only when some row is gated
     bool two_lanes = false;
     if (want_lanes && ctx->attn_kernel == PS_ATTN_MMA)
         for (int32_t b = 0; b < B; ++b) two_lanes |= active[b] && gated[b];
     if (m.valid && m.epoch == ctx->table_epoch && (int32_t)m.reqs.size() == B && m.two_lanes == two_lanes &&
+        m.contended == contended &&
         std::equal(m.reqs.begin(), m.reqs.end(), reqs) && m.gated == gated && m.active == active)
         return PS_OK;
 
@@ -619,12 +620,16 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
                 if (gated[b]) ++n_gated_rows;
             }
         } else {
-            // Tensor-core kernel: the lane's 16-token tiles form one sequence.  Its head is cut into
-            // equal static shares, one per CTA; its tail (kDynFrac of the tiles, when there are enough)
-            // into small chunks that the CTAs take dynamically.  An item is the part of a row that
-            // falls into one share or chunk.
+            // Tensor-core kernel: the lane's 16-token tiles form one sequence, cut into equal static shares,
+            // one per CTA: every CTA streams the same number of bytes whatever the context-length mix, and
+            // only the rows cut by share borders need combining.  When reload traffic runs beside the step
+            // (scatter kernels and the reload lane take SM time unevenly) the last 5 % of the tiles become
+            // chunks that the CTAs take dynamically; without contention such a tail only costs (more parts
+            // to combine, a last round of chunks that does not fill the machine): 172 against 189 us per
+            // 1 GiB launch.  An item is the part of a row that falls into one share or chunk.
             constexpr int kTile = ps::kMmaTileTokens;
             constexpr int64_t kMinTilesPerCta = 8;
+            constexpr int64_t kDynMinChunk = 16;
             constexpr int64_t kDynChunksPerCta = 6;
             int64_t total_tiles = 0;
             int32_t lane_rows = 0;
@@ -638,9 +643,9 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
                 n_cta = std::min<int64_t>(std::max<int64_t>((total_tiles + kMinTilesPerCta - 1) / kMinTilesPerCta, 1),
                                           ctx->num_sms);
             int64_t dyn_tiles = 0, chunk = 0;
-            if (n_cta > 0 && total_tiles >= 32 * n_cta) {
-                dyn_tiles = total_tiles * 15 / 100;
-                chunk = std::max<int64_t>(kMinTilesPerCta, (dyn_tiles + kDynChunksPerCta * n_cta - 1) / (kDynChunksPerCta * n_cta));
+            if (contended && n_cta > 0 && total_tiles >= 32 * n_cta) {
+                dyn_tiles = total_tiles * 5 / 100;
+                chunk = std::max<int64_t>(kDynMinChunk, (dyn_tiles + kDynChunksPerCta * n_cta - 1) / (kDynChunksPerCta * n_cta));
             }
             const int64_t static_tiles = total_tiles - dyn_tiles;
             const int64_t per = n_cta > 0 ? std::max<int64_t>((static_tiles + n_cta - 1) / n_cta, 1) : 1;
@@ -751,6 +756,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     m.gated = gated;
     m.active = active;
     m.two_lanes = two_lanes;
+    m.contended = contended;
     m.epoch = ctx->table_epoch;
     m.valid = true;
     m.dev.block_tables = (const int32_t*)d;
@@ -1410,7 +1416,7 @@ int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, flo
     }
     std::vector<char> active((size_t)batch, 1), gated((size_t)batch, 0);
     for (int32_t b = 0; b < batch; ++b) gated[(size_t)b] = ctx->reqs[reqs[b]].gated ? 1 : 0;
-    int32_t rc = prepare_batch(ctx, reqs, batch, active, gated, /*want_lanes=*/false);
+    int32_t rc = prepare_batch(ctx, reqs, batch, active, gated, /*want_lanes=*/false, /*contended=*/false);
     if (rc != PS_OK) return rc;
     int32_t launched = 0;
     return launch_layer_attn(ctx, layer, q, out, lse, ctx->meta.n_gated_rows ? ctx->ev_in[(size_t)layer] : nullptr,
@@ -1461,7 +1467,8 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
     }
     const bool attn = want_attn && st.decoded > 0;
     if (attn) {
-        rc = prepare_batch(ctx, reqs, batch, active, gated, (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) == 0);
+        rc = prepare_batch(ctx, reqs, batch, active, gated, (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) == 0,
+                           /*contended=*/!plan.empty() && (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) == 0);
         if (rc != PS_OK) return rc;
         st.gated = ctx->meta.n_gated_rows;
     }
