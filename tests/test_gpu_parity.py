@@ -330,3 +330,46 @@ def test_sync_reload_flag_gives_identical_results():
     assert prof["attn_launches"] >= w.shape.num_layers and prof["attn_ms"] > 0
     assert prof["gather_bytes"] == prof["d2h_bytes"] == prof["h2d_bytes"] == prof["scatter_bytes"] > 0
     assert p.lib.launch_count() > 0
+
+
+def test_sync_times_out_while_the_compute_stream_is_busy_and_recovers():
+    """Bounded host wait: PS_ERR_TIMEOUT leaves everything in flight; a later wait succeeds."""
+    w, p = tiny_pair()
+    torch.cuda._sleep(400_000_000)                      # a kernel that ends by itself after ~0.2 s
+    assert p.lib.sync(timeout_ms=1) == B.PS_ERR_TIMEOUT
+    assert "timed out" in p.lib.last_error()
+    assert p.lib.sync(timeout_ms=-1) == B.PS_OK
+    r = w.victims[0]
+    assert p.both("swap_out", r) == B.PS_OK             # the context is fully usable afterwards
+    p.sync()
+    assert np.array_equal(p.host_image_bits(r), p.orc.reqs[r].image.reshape(-1))
+
+
+def test_kernel_skips_a_block_id_outside_the_pool_and_reports_it():
+    """A table entry outside [0, num_blocks) is never dereferenced: the kernel records status 2 and goes on;
+    rows with valid tables are unaffected."""
+    Hkv, Hq, D, S, nb = 2, 4, 64, 16, 32
+    rng = np.random.default_rng(31)
+    K = wl.randn_bf16_bits(rng, (1, nb, S, Hkv, D))
+    V = wl.randn_bf16_bits(rng, (1, nb, S, Hkv, D))
+    p = Pair(wl.KVShape(1, Hkv, Hq, D, S, nb), None, K, V, max_batch=2)
+    assert p.both("kv_alloc", 0, 3 * S) == B.PS_OK and p.both("kv_alloc", 1, 2 * S) == B.PS_OK
+    tables = torch.tensor([p.lib.block_table(0)[0], p.lib.block_table(1)[0] + [0]], dtype=torch.int32, device="cuda")
+    bad = tables.clone()
+    bad[1, 1] = nb + 5                                   # out of range, in the second request only
+    q = wl.randn_bf16_bits(rng, (2, Hq, D))
+    qd = bits_to_dev(q)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    out = torch.zeros_like(qd)
+    kw = dict(num_kv_heads=Hkv, num_q_heads=Hq, head_dim=D, block_size=S, num_gpu_blocks=nb, status_word=status)
+    rc, text = B.ps_decode_attn_static(p.Kd[0], p.Vd[0], qd, out, bad, [3 * S, 2 * S], **kw)
+    assert rc == B.PS_OK, text
+    torch.cuda.synchronize()
+    assert int(status.item()) == 2
+    want, _ = p.orc.decode_attn(0, q, [0, 1])
+    check_attn(out[0:1], want[0:1])                      # the request with a valid table is exact
+    status.zero_()
+    rc, text = B.ps_decode_attn_static(p.Kd[0], p.Vd[0], qd, out, tables, [3 * S, 2 * S], **kw)
+    torch.cuda.synchronize()
+    assert rc == B.PS_OK and int(status.item()) == 0
+    check_attn(out, want)
