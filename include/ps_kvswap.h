@@ -10,7 +10,7 @@
  *     event per layer chunk, the compute stream waiting on a chunk's event only before it
  *     runs that chunk,
  *   - a per-step host-to-device copy budget B_copy consumed in queue order at request
- *     granularity, partially for the request that does not fit (Alg. 1 lines 17, 22-25),
+ *     granularity, partially for the request that does not fit (Alg. 1: GetCopyBudget, ConsumeCopyBudget),
  *   - the decode forward the reload overlaps with, here its KV-consuming part: paged
  *     grouped-query attention over the block table.
  * Which request to evict and how large the budget should be are scheduler decisions and stay

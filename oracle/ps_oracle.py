@@ -17,7 +17,7 @@ What it follows (ProServe, Section 4.3 "Efficient Block Management", and Appendi
   one completion event per layer chunk).  -> `swap_in_begin`, `swap_in_layer`.
 * A per-step host-to-device copy budget B_copy (in blocks) is consumed in queue order at request
   granularity: all missing blocks b_miss of a request if they fit, otherwise a partial copy with
-  the residual budget ("Put it Together", Alg. 1 lines 17 and 22-25).  -> `step_plan`, `step`.
+  the residual budget ("Put it Together"; Alg. 1: GetCopyBudget, ConsumeCopyBudget).  -> `step_plan`, `step`.
   The beta admission test of that paragraph depends on the scheduler's computable-token count and
   is not modelled: a partial copy is always allowed and a request decodes only once complete.
 * The number of blocks to reload per step, B_copy, follows the three-case procedure of "Adaptive

@@ -531,7 +531,7 @@ int32_t missing_of(const Req& r) {
     return (int32_t)r.table.size() - mn;
 }
 
-// Copy-budget consumption (Alg. 1 lines 22-25 reduced to the byte budget): FIFO, whole request if it
+// Copy-budget consumption (Alg. 1, ConsumeCopyBudget, reduced to the byte budget): FIFO, whole request if it
 // fits, otherwise the residual.
 std::vector<PlanEntry> make_plan(ps_ctx* ctx, int64_t copy_budget_bytes) {
     std::vector<PlanEntry> plan;
