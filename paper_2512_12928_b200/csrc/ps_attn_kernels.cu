@@ -506,10 +506,16 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
-    // Programmatic dependent launch: the next layer's launch (same kernel, the other set of scratch buffers,
-    // independent inputs) may start filling SMs as the CTAs of this one retire, which hides its launch latency
-    // and prologue under this launch's tail.  A no-op for ordinary launches.
+    // Programmatic dependent launch: the next layer's launch (same kernel, independent inputs) may start filling
+    // SMs as the CTAs of this one retire, which hides its launch latency and prologue under this launch's tail.
+    // What consecutive launches do share is the split-KV scratch (partials, arrival counters, chunk counters):
+    // a thread executes griddepcontrol.wait (dep_wait below) before it first touches any of it, i.e. it waits
+    // until the launch this one depends on has completed and its memory operations are visible; as every
+    // launch also executes it before it ends, launches complete in order, so no earlier launch is still
+    // running either.  The first such access comes at the end of a CTA's first row part, long after the
+    // predecessor's tail.  All of it is a no-op for ordinary launches.
     if (threadIdx.x == 0) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    auto dep_wait = []() { asm volatile("griddepcontrol.wait;" ::: "memory"); };
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kMmaStages; ++s) {
@@ -544,6 +550,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             if (!dynamic && it >= item1) dynamic = true;
             if (dynamic) {
                 int c = 0;
+                dep_wait();
                 if (lane == 0) c = atomicAdd(counter, 1);
                 c = __shfl_sync(0xffffffffu, c, 0);
                 it = dyn_begin + c;
@@ -620,6 +627,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             }
         }
         // the last CTA to finish fetching re-arms the chunk counter for the lane's next launch
+        dep_wait();
         if (lane == 0) {
             __threadfence();
             if (atomicAdd(counter + 1, 1) == (int)gridDim.x - 1) {
@@ -756,6 +764,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                         if (lse != nullptr && t == 0)
                             lse[(int64_t)item_b * Hq + hq] = L > 0.f ? (m_run + log2f(L)) * kLn2 : -CUDART_INF_F;
                     } else {
+                        dep_wait();
                         float* pr = partials + ((int64_t)item_part * Hq + hq) * kMmaPartStride;
 #pragma unroll
                         for (int i = 0; i < 16; ++i)
@@ -767,6 +776,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                     }
                 }
                 if (item_nparts > 1) {
+                    dep_wait();
                     // Split-KV fix-up: the warp that delivers the last part of a (row, KV head) combines the
                     // parts.  Combining costs a few round trips to L2 during which this warp would hold up the
                     // CTA's ring, so the row is only noted here and combined after the CTA's last tile.
@@ -793,7 +803,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
     }
     // A launch does not complete before the launch it was made programmatically dependent on has completed:
     // work enqueued after this launch may rely on both.  (Returns at once for ordinary launches.)
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    dep_wait();
 }
 
 template <int G>

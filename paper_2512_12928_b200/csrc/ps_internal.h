@@ -93,9 +93,10 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
                                int32_t lane, float* partials, int32_t* sched, int32_t* row_done, int32_t* d_status,
                                bool after_own_launch, cudaStream_t stream);
 // after_own_launch (tensor-core kernel only): the previous kernel on `stream` is a launch of the same kernel
-// that filled every SM, used the OTHER set of partials / sched / row_done, and shares no data with this one;
-// the launch is then made programmatically dependent on it, so its CTAs start as that launch's CTAs retire.
-// With one CTA per SM and full grids at most two consecutive launches overlap, hence two sets of scratch.
+// whose inputs and outputs are independent of this one's; the launch is then made programmatically
+// dependent on it, so its CTAs start as that launch's CTAs retire.  The kernel waits for its predecessor's
+// completion before it first touches partials / sched / row_done, so consecutive launches may even share
+// them (the runtime alternates two sets all the same).
 
 // Token granularity at which the tensor-core kernel splits a context.
 constexpr int kMmaTileTokens = 16;
