@@ -16,8 +16,9 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB_DIR = os.path.join(PKG, "lib")
 LIB_PATH = os.path.join(LIB_DIR, "libps_kvswap.so")
-SOURCES = ["ps_runtime.cu", "ps_copy_kernels.cu", "ps_attn_kernels.cu", "ps_static_scratch.cu"]
-HEADERS = [os.path.join(CSRC, "ps_internal.h"), os.path.join(ROOT, "include", "ps_kvswap.h")]
+SOURCES = ["ps_runtime.cu", "ps_swap.cu", "ps_step.cu", "ps_policy.cu", "ps_measure.cu", "ps_copy_kernels.cu",
+           "ps_attn_kernels.cu", "ps_static_scratch.cu"]
+HEADERS = [os.path.join(CSRC, "ps_internal.h"), os.path.join(CSRC, "ps_ctx.h"), os.path.join(ROOT, "include", "ps_kvswap.h")]
 
 
 def _nvcc() -> str:

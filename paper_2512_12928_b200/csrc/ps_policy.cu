@@ -1,0 +1,116 @@
+// Decisions of Section 4.3 as host arithmetic: adaptive copy budget, eviction policy, partial-copy rule.
+#include "ps_ctx.h"
+
+extern "C" {
+
+int32_t ps_copy_budget(ps_ctx* ctx, const int64_t* reqs, int32_t batch, const ps_budget_model* model,
+                       int64_t* budget_blocks, int64_t* budget_bytes, int32_t* which_case) {
+    if (!ctx) return PS_ERR_INVALID;
+    if (!model || !budget_blocks || batch < 0 || (batch > 0 && !reqs))
+        return ctx->fail(PS_ERR_INVALID, "ps_copy_budget: null argument");
+    const double a_d = model->a_d_us_per_token, b_d = model->b_d_us, t_c = model->t_c_us;
+    const double t_block = model->t_block_us, t_budget = model->t_budget_us;
+    if (!(t_block > 0.0) || a_d < 0.0 || b_d < 0.0 || t_c < 0.0 || t_budget < 0.0)
+        return ctx->fail(PS_ERR_INVALID, "ps_copy_budget: t_block must be positive, the other terms non-negative");
+    // the step's requests: resident ones decode whatever is copied; queued reloads decode once complete
+    std::unordered_map<int64_t, char> in_batch;
+    double t_resident = t_c, t_all = t_c;
+    for (int32_t b = 0; b < batch; ++b) {
+        auto it = ctx->reqs.find(reqs[b]);
+        if (it == ctx->reqs.end()) continue;
+        const Req& r = it->second;
+        if (r.state != PS_REQ_RESIDENT && r.state != PS_REQ_SWAPPING_IN) continue;
+        if (in_batch.count(reqs[b])) continue;
+        in_batch[reqs[b]] = 1;
+        const double t = a_d * (double)r.n_tokens + b_d;
+        t_all += t;
+        if (r.state == PS_REQ_RESIDENT) t_resident += t;
+    }
+    // the reload queue in order: missing blocks and what the request adds to the step once complete
+    std::vector<int64_t> cum_miss;
+    std::vector<double> cum_time;
+    int64_t missing = 0;
+    double t_added = 0.0;
+    for (int64_t id : ctx->in_fifo) {
+        const Req& r = ctx->reqs[id];
+        const int32_t miss = missing_of(r);
+        if (miss == 0) continue;
+        missing += miss;
+        if (in_batch.count(id)) t_added += a_d * (double)r.n_tokens + b_d;
+        cum_miss.push_back(missing);
+        cum_time.push_back(t_added);
+    }
+    const double t_fwd_min = t_all;
+    const double t_trans_max = (double)missing * t_block;
+    int64_t B = 0;
+    int32_t wc = 0;
+    if (t_fwd_min > t_budget) {
+        wc = 1;
+        B = (int64_t)std::floor(t_budget / t_block);
+    } else if (t_fwd_min > t_trans_max) {
+        wc = 21;
+        B = missing;
+    } else {
+        wc = 22;
+        if (!(t_block > a_d * (double)ctx->cfg.block_size))
+            return ctx->fail(PS_ERR_INVALID, "ps_copy_budget: the search needs t_block > a_d * block_size");
+        auto step_time_after = [&](int64_t blocks) {  // requests whose last missing block is among the first `blocks`
+            double t = t_resident;
+            for (size_t i = 0; i < cum_miss.size() && cum_miss[i] <= blocks; ++i) t = t_resident + cum_time[i];
+            return t;
+        };
+        int64_t lo = 0, hi = missing;  // lo is feasible (0 blocks take no time)
+        while (lo < hi) {
+            const int64_t mid = lo + (hi - lo + 1) / 2;
+            if ((double)mid * t_block <= step_time_after(mid))
+                lo = mid;
+            else
+                hi = mid - 1;
+        }
+        B = lo;
+    }
+    *budget_blocks = B;
+    if (budget_bytes) *budget_bytes = B * ctx->block_bytes;
+    if (which_case) *which_case = wc;
+    return PS_OK;
+}
+
+int32_t ps_select_victims(ps_ctx* ctx, const int64_t* queue, int32_t n, const double* waited_us, double tau_us,
+                          double near_frac, int32_t blocks_needed, int64_t* victims, int32_t cap, int32_t* n_victims,
+                          int32_t* blocks_freed) {
+    if (!ctx) return PS_ERR_INVALID;
+    if (n < 0 || (n > 0 && (!queue || !waited_us)) || cap < 0 || (cap > 0 && !victims) || !n_victims ||
+        !(near_frac > 0.0 && near_frac <= 1.0) || tau_us < 0.0 || blocks_needed < 0)
+        return ctx->fail(PS_ERR_INVALID, "ps_select_victims: bad argument");
+    int32_t count = 0, freed = 0;
+    for (int32_t i = n - 1; i >= 0 && freed < blocks_needed && count < cap; --i) {
+        auto it = ctx->reqs.find(queue[i]);
+        if (it == ctx->reqs.end()) continue;
+        const Req& r = it->second;
+        if (r.state != PS_REQ_RESIDENT || r.table.empty()) continue;
+        if (waited_us[i] >= near_frac * tau_us) continue;  // close to starving: about to be promoted to the head
+        bool dup = false;
+        for (int32_t k = 0; k < count; ++k) dup |= victims[k] == queue[i];
+        if (dup) continue;
+        victims[count++] = queue[i];
+        freed += (int32_t)r.table.size();
+    }
+    *n_victims = count;
+    if (blocks_freed) *blocks_freed = freed;
+    return PS_OK;
+}
+
+int32_t ps_copy_condition(int32_t l_comp, int32_t l_comp_max, int32_t b_miss, int32_t b_rem, int32_t s_blk,
+                          double beta, int32_t* allowed) {
+    if (!allowed || l_comp < 0 || l_comp_max < 0 || b_miss < 0 || b_rem < 0 || s_blk <= 0 || !(beta > 1.0))
+        return PS_ERR_INVALID;
+    if (b_rem >= b_miss)
+        *allowed = 1;
+    else if (l_comp >= l_comp_max)
+        *allowed = 1;
+    else
+        *allowed = (double)l_comp / ((double)(b_miss - b_rem) * (double)s_blk) > beta ? 1 : 0;
+    return PS_OK;
+}
+
+}  // extern "C"

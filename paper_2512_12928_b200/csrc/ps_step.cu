@@ -1,0 +1,463 @@
+// One engine step under the copy budget: budget consumption over the reload queue, the decode batch's device
+// metadata and work split, per-layer attention launches gated on the reload events (Section 4.3 "Put it
+// Together"; Appendix B).
+#include "ps_ctx.h"
+
+namespace psrt {
+
+// Copy-budget consumption (Alg. 1, ConsumeCopyBudget, reduced to the byte budget): FIFO, whole request if it
+// fits, otherwise the residual.
+std::vector<PlanEntry> make_plan(ps_ctx* ctx, int64_t copy_budget_bytes) {
+    std::vector<PlanEntry> plan;
+    const bool unlimited = copy_budget_bytes < 0;
+    int64_t left = unlimited ? 0 : copy_budget_bytes / ctx->block_bytes;
+    for (int64_t id : ctx->in_fifo) {
+        Req& r = ctx->reqs[id];
+        const int32_t miss = missing_of(r);
+        if (miss == 0) continue;
+        const int32_t lo = (int32_t)r.table.size() - miss;
+        const int64_t take = unlimited ? miss : std::min<int64_t>(miss, left);
+        if (take == 0) break;
+        plan.push_back({id, lo, lo + (int32_t)take});
+        if (!unlimited) {
+            left -= take;
+            if (left == 0) break;
+        }
+    }
+    return plan;
+}
+
+// ---- attention batch ------------------------------------------------------------------------------------
+
+int32_t choose_split(const ps_ctx* ctx, int64_t total_tokens) {
+    if (ctx->cfg.kv_split_tokens > 0) return ctx->cfg.kv_split_tokens;
+    const int64_t target_items = std::max<int64_t>(1, 4096 / ctx->cfg.num_kv_heads);
+    int64_t split = (total_tokens + target_items - 1) / target_items;
+    split = round_up(std::max<int64_t>(split, 1), 64);
+    return (int32_t)std::min<int64_t>(std::max<int64_t>(split, 256), 1 << 20);
+}
+
+// Builds (or reuses) the device metadata for a decode batch.  Row b of the metadata is position b of
+// the caller's request array (q / out rows are addressed by that position); rows with active[b] == 0
+// get no work item.  gated[b] != 0 marks rows whose reload is still landing: their attention waits on
+// the layer's reload event.  With want_lanes they get a work list of their own (lane 1), launched on
+// the reload-lane stream behind the event, so that the launches of the other rows never wait.
+int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::vector<char>& active,
+                      const std::vector<char>& gated, bool want_lanes, bool contended) {
+    BatchMeta& m = ctx->meta;
+    // two work lists (lanes) only for the tensor-core kernel and only when some row is gated
+    bool two_lanes = false;
+    if (want_lanes && ctx->attn_kernel == PS_ATTN_MMA)
+        for (int32_t b = 0; b < B; ++b) two_lanes |= active[b] && gated[b];
+    if (m.valid && m.epoch == ctx->table_epoch && (int32_t)m.reqs.size() == B && m.two_lanes == two_lanes &&
+        m.contended == contended &&
+        std::equal(m.reqs.begin(), m.reqs.end(), reqs) && m.gated == gated && m.active == active)
+        return PS_OK;
+
+    int32_t stride = 1;
+    int64_t total_tokens = 0;
+    for (int32_t b = 0; b < B; ++b) {
+        if (!active[b]) continue;
+        const Req& r = ctx->reqs[reqs[b]];
+        stride = std::max<int32_t>(stride, (int32_t)r.table.size());
+        total_tokens += r.n_tokens;
+    }
+    std::vector<int32_t> row_first(B, 0), row_parts(B, 0), ctx_len(B, 0);
+    std::vector<ps::AttnItem> items;
+    std::vector<int32_t> cta_begin[2];
+    int32_t parts = 0, n_ungated = 0, n_gated_rows = 0;
+    bool any_multi = false, lane_multi[2] = {false, false};
+    const bool mma = ctx->attn_kernel == PS_ATTN_MMA;
+    const int32_t split = mma ? 0 : choose_split(ctx, total_tokens);
+    for (int pass = 0; pass < (two_lanes ? 2 : 1); ++pass) {  // lane 0: rows that need no wait (or all rows); lane 1: gated rows
+        if (!mma) {
+            // SIMT kernel: one CTA per (item, KV head); items are fixed-size token ranges of a row
+            for (int32_t b = 0; b < B; ++b) {
+                if (!active[b] || (two_lanes && (gated[b] ? 1 : 0) != pass)) continue;
+                const Req& r = ctx->reqs[reqs[b]];
+                const int32_t n = std::max(1, (r.n_tokens + split - 1) / split);
+                row_first[b] = parts;
+                row_parts[b] = n;
+                ctx_len[b] = r.n_tokens;
+                any_multi |= n > 1;
+                lane_multi[pass] |= n > 1;
+                for (int32_t k = 0; k < n; ++k) {
+                    ps::AttnItem it{};
+                    it.b = b;
+                    it.t_begin = k * split;
+                    it.t_end = std::min(r.n_tokens, (k + 1) * split);
+                    it.part = parts + k;
+                    it.n_parts = n;
+                    items.push_back(it);
+                }
+                parts += n;
+                if (gated[b]) ++n_gated_rows;
+            }
+        } else {
+            // Tensor-core kernel: the lane's 16-token tiles form one sequence, cut into equal static shares,
+            // one per CTA: every CTA streams the same number of bytes whatever the context-length mix, and
+            // only the rows cut by share borders need combining.  When reload traffic runs beside the step
+            // (scatter kernels and the reload lane take SM time unevenly) the last 5 % of the tiles become
+            // chunks that the CTAs take dynamically; without contention such a tail only costs (more parts
+            // to combine, a last round of chunks that does not fill the machine): 172 against 189 us per
+            // 1 GiB launch.  An item is the part of a row that falls into one share or chunk.
+            constexpr int kTile = ps::kMmaTileTokens;
+            constexpr int64_t kMinTilesPerCta = 8;
+            constexpr int64_t kDynMinChunk = 16;
+            constexpr int64_t kDynChunksPerCta = 6;
+            int64_t total_tiles = 0;
+            int32_t lane_rows = 0;
+            for (int32_t b = 0; b < B; ++b)
+                if (active[b] && !(two_lanes && (gated[b] ? 1 : 0) != pass)) {
+                    total_tiles += (ctx->reqs[reqs[b]].n_tokens + kTile - 1) / kTile;
+                    ++lane_rows;
+                }
+            int64_t n_cta = 0;
+            if (lane_rows > 0)
+                n_cta = std::min<int64_t>(std::max<int64_t>((total_tiles + kMinTilesPerCta - 1) / kMinTilesPerCta, 1),
+                                          ctx->num_sms);
+            int64_t dyn_tiles = 0, chunk = 0;
+            if (contended && n_cta > 0 && total_tiles >= 32 * n_cta) {
+                dyn_tiles = total_tiles * 5 / 100;
+                chunk = std::max<int64_t>(kDynMinChunk, (dyn_tiles + kDynChunksPerCta * n_cta - 1) / (kDynChunksPerCta * n_cta));
+            }
+            const int64_t static_tiles = total_tiles - dyn_tiles;
+            const int64_t per = n_cta > 0 ? std::max<int64_t>((static_tiles + n_cta - 1) / n_cta, 1) : 1;
+            // walk the rows; `pos` is the position in the lane's tile sequence
+            int64_t pos = 0, filled = 0;       // filled: tiles in the current share or chunk
+            bool in_dyn = false;
+            if (n_cta > 0) cta_begin[pass].push_back((int32_t)items.size());
+            auto close_static = [&]() {        // pad the share list and mark where the dynamic chunks start
+                while ((int64_t)cta_begin[pass].size() < n_cta + 1) cta_begin[pass].push_back((int32_t)items.size());
+                in_dyn = true;
+                filled = 0;
+            };
+            for (int32_t b = 0; b < B; ++b) {
+                if (!active[b] || (two_lanes && (gated[b] ? 1 : 0) != pass)) continue;
+                const Req& r = ctx->reqs[reqs[b]];
+                const int64_t tiles_b = (r.n_tokens + kTile - 1) / kTile;
+                const size_t first_item = items.size();
+                ctx_len[b] = r.n_tokens;
+                row_first[b] = parts;
+                if (tiles_b == 0) {  // empty context: one item without tiles writes the zero row
+                    ps::AttnItem it{};
+                    it.b = b;
+                    items.push_back(it);
+                }
+                for (int64_t lo = 0; lo < tiles_b;) {
+                    if (!in_dyn && pos >= static_tiles) close_static();
+                    int64_t room;
+                    if (!in_dyn) {
+                        if (filled == per && (int64_t)cta_begin[pass].size() < n_cta) {
+                            cta_begin[pass].push_back((int32_t)items.size());
+                            filled = 0;
+                        }
+                        room = std::min(per - filled, static_tiles - pos);
+                    } else {
+                        if (filled == chunk) filled = 0;
+                        room = chunk - filled;
+                    }
+                    const int64_t take = std::min(tiles_b - lo, std::max<int64_t>(room, 1));
+                    ps::AttnItem it{};
+                    it.b = b;
+                    it.t_begin = (int32_t)(lo * kTile);
+                    it.t_end = (int32_t)std::min<int64_t>(r.n_tokens, (lo + take) * kTile);
+                    items.push_back(it);
+                    lo += take;
+                    pos += take;
+                    // a dynamic chunk never spans two rows: every item of the tail is its own chunk
+                    filled = in_dyn ? chunk : filled + take;
+                    if (in_dyn && take < chunk && lo < tiles_b) filled = chunk;
+                }
+                const int32_t n = (int32_t)(items.size() - first_item);
+                for (size_t k = first_item; k < items.size(); ++k) {
+                    items[k].part = parts + (int32_t)(k - first_item);
+                    items[k].n_parts = n;
+                }
+                row_parts[b] = n;
+                parts += n;
+                any_multi |= n > 1;
+                lane_multi[pass] |= n > 1;
+                if (gated[b]) ++n_gated_rows;
+            }
+            if (n_cta > 0 && !in_dyn) close_static();
+        }
+        if (pass == 0) n_ungated = (int32_t)items.size();
+    }
+    if (parts > ctx->max_parts) return ctx->fail(PS_ERR_INVALID, "split-KV scratch too small for this batch");
+
+    const size_t sz_tables = (size_t)round_up((int64_t)B * stride * 4, 256);
+    const size_t sz_vec = (size_t)round_up((int64_t)B * 4, 256);
+    const size_t sz_items = (size_t)round_up((int64_t)std::max<size_t>(items.size(), 1) * sizeof(ps::AttnItem), 256);
+    const size_t sz_cta = (size_t)round_up((int64_t)(cta_begin[0].size() + cta_begin[1].size() + 2) * 4, 256);
+    const size_t total = sz_tables + 4 * sz_vec + sz_items + sz_cta;
+    if (total > ctx->a_meta.chunk) return ctx->fail(PS_ERR_INVALID, "decode batch metadata exceeds its buffer");
+    // a fresh chunk: the chunk of the cached batch stays intact until this point
+    int32_t rc = arena_next_chunk(ctx, ctx->a_meta, /*record_fence=*/false);
+    if (rc != PS_OK) return rc;
+    size_t off = 0;
+    rc = arena_alloc(ctx, ctx->a_meta, total, &off);
+    if (rc != PS_OK) return rc;
+    char* h = ctx->a_meta.h + off;
+    char* d = ctx->a_meta.d + off;
+    int32_t* ht = (int32_t*)h;
+    memset(ht, 0, sz_tables);
+    for (int32_t b = 0; b < B; ++b) {
+        if (!active[b]) continue;
+        const Req& r = ctx->reqs[reqs[b]];
+        if (!r.table.empty()) memcpy(ht + (size_t)b * stride, r.table.data(), r.table.size() * 4);
+    }
+    memcpy(h + sz_tables, ctx_len.data(), (size_t)B * 4);
+    memcpy(h + sz_tables + sz_vec, row_first.data(), (size_t)B * 4);
+    memcpy(h + sz_tables + 2 * sz_vec, row_parts.data(), (size_t)B * 4);
+    {
+        int32_t* lane = (int32_t*)(h + sz_tables + 3 * sz_vec);
+        for (int32_t b = 0; b < B; ++b) lane[b] = two_lanes && gated[b] ? 1 : 0;
+    }
+    if (!items.empty()) memcpy(h + sz_tables + 4 * sz_vec, items.data(), items.size() * sizeof(ps::AttnItem));
+    {
+        int32_t* cb = (int32_t*)(h + sz_tables + 4 * sz_vec + sz_items);
+        if (!cta_begin[0].empty()) memcpy(cb, cta_begin[0].data(), cta_begin[0].size() * 4);
+        if (!cta_begin[1].empty()) memcpy(cb + cta_begin[0].size(), cta_begin[1].data(), cta_begin[1].size() * 4);
+    }
+    CK(ps::launch_upload(d, ctx->a_meta.hd + off, total, ctx->compute));
+    ctx->launches++;
+    // the pinned side of this chunk may be rewritten once this upload has run
+    CK(cudaEventRecord(ctx->a_meta.fence[ctx->a_meta.cur], ctx->compute));
+    ctx->a_meta.fenced[ctx->a_meta.cur] = 1;
+
+    m.reqs.assign(reqs, reqs + B);
+    m.gated = gated;
+    m.active = active;
+    m.two_lanes = two_lanes;
+    m.contended = contended;
+    m.epoch = ctx->table_epoch;
+    m.valid = true;
+    m.dev.block_tables = (const int32_t*)d;
+    m.dev.ctx_len = (const int32_t*)(d + sz_tables);
+    m.dev.row_first_part = (const int32_t*)(d + sz_tables + sz_vec);
+    m.dev.row_parts = (const int32_t*)(d + sz_tables + 2 * sz_vec);
+    m.dev.row_lane = (const int32_t*)(d + sz_tables + 3 * sz_vec);
+    m.dev.items = (const ps::AttnItem*)(d + sz_tables + 4 * sz_vec);
+    {
+        const int32_t* cb = (const int32_t*)(d + sz_tables + 4 * sz_vec + sz_items);
+        m.dev.cta_begin[0] = cb;
+        m.dev.cta_begin[1] = cb + cta_begin[0].size();
+        m.dev.n_cta[0] = cta_begin[0].empty() ? 0 : (int32_t)cta_begin[0].size() - 1;
+        m.dev.n_cta[1] = cta_begin[1].empty() ? 0 : (int32_t)cta_begin[1].size() - 1;
+        m.dev.lane_items[0] = 0;
+        m.dev.lane_items[1] = n_ungated;
+        m.dev.lane_items[2] = (int32_t)items.size();
+    }
+    m.dev.table_stride = stride;
+    m.dev.batch = B;
+    m.n_items = (int32_t)items.size();
+    m.n_ungated_items = n_ungated;
+    m.n_parts = parts;
+    m.n_gated_rows = n_gated_rows;
+    m.any_multi = any_multi;
+    m.lane_multi[0] = lane_multi[0];
+    m.lane_multi[1] = lane_multi[1];
+    m.kv_bytes_per_layer = total_tokens * 2 * ctx->cfg.num_kv_heads * ctx->cfg.head_dim * 2;
+    return PS_OK;
+}
+
+// Launches one layer of attention for the prepared batch.  wait_event: the layer's reload event when rows
+// of the batch are still being reloaded (Appendix B: the computation synchronises on a layer chunk's event
+// only before it executes that chunk); nullptr = no wait.  With two work lists the rows that need no wait
+// run on the compute stream and the gated rows on the reload lane behind the event; with one list the
+// whole launch waits.  follows_own: the previous kernel on the compute stream is this function's launch
+// for the previous layer of the same step (independent data); full-grid tensor-core launches then overlap
+// head to tail.
+int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, float* lse, cudaEvent_t wait_event,
+                          bool follows_own, int32_t* n_launched) {
+    BatchMeta& m = ctx->meta;
+    if (m.n_items == 0) return PS_OK;
+    ps::AttnShape sh{ctx->cfg.num_kv_heads, ctx->cfg.num_q_heads, ctx->cfg.head_dim, ctx->cfg.block_size,
+                     ctx->cfg.num_gpu_blocks};
+    const bool mma = ctx->attn_kernel == PS_ATTN_MMA;
+    const ps::AttnTensorMaps* maps = ctx->tmaps.empty() ? nullptr : &ctx->tmaps[(size_t)layer];
+    const bool lanes = m.two_lanes && m.n_items > m.n_ungated_items;
+    if (wait_event && !lanes) CK(cudaStreamWaitEvent(ctx->compute, wait_event, 0));
+    if (m.n_ungated_items > 0) {
+        const bool overlap = follows_own && mma && !ctx->profile && m.dev.n_cta[0] == ctx->num_sms;
+        const int set = ctx->scratch_set;
+        ctx->scratch_set ^= 1;
+        const int64_t bytes = m.kv_bytes_per_layer * m.n_ungated_items / m.n_items;
+        {
+            ProfScope prof(ctx, kProfAttn, ctx->compute, bytes, wait_event && !lanes ? 1000 + layer : layer);
+            CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], maps, q, out, lse, m.dev,
+                                      0, ctx->partials[set], ctx->d_sched[set], ctx->d_row_done[set], ctx->d_status,
+                                      overlap, ctx->compute));
+            ctx->launches++;
+            ++*n_launched;
+        }
+        // the tensor-core kernel combines split rows itself; the CUDA-core kernel needs the merge pass
+        if (!mma && m.any_multi) {
+            ProfScope prof(ctx, kProfMerge, ctx->compute, 0, layer);
+            CK(ps::launch_attn_merge(sh, out, lse, m.dev, ctx->partials[set], -1, ctx->compute));
+            ctx->launches++;
+            ++*n_launched;
+        }
+    }
+    if (lanes) {
+        if (wait_event) CK(cudaStreamWaitEvent(ctx->s_lane, wait_event, 0));
+        const int64_t bytes = m.kv_bytes_per_layer * (m.n_items - m.n_ungated_items) / m.n_items;
+        ProfScope prof(ctx, kProfAttn, ctx->s_lane, bytes, 1000 + layer);
+        CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], maps, q, out, lse, m.dev, 1,
+                                  ctx->partials[2], ctx->d_sched[2], ctx->d_row_done[2], ctx->d_status, false, ctx->s_lane));
+        ctx->launches++;
+        ++*n_launched;
+    }
+    return PS_OK;
+}
+
+}  // namespace psrt
+
+extern "C" {
+
+int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, float* lse, const int64_t* reqs,
+                       int32_t batch) {
+    if (!ctx) return PS_ERR_INVALID;
+    if (ctx->bk) return ctx->fail(PS_ERR_INVALID, "ps_decode_attn: context holds no device (bookkeeping only)");
+    if (layer < 0 || layer >= ctx->cfg.num_layers || batch < 0 || batch > ctx->cfg.max_batch ||
+        (batch > 0 && (!q || !out || !reqs)))
+        return ctx->fail(PS_ERR_INVALID, "ps_decode_attn: bad argument");
+    if (batch == 0) return PS_OK;
+    bool any_gated = false;
+    for (int32_t b = 0; b < batch; ++b) {
+        auto it = ctx->reqs.find(reqs[b]);
+        if (it == ctx->reqs.end()) return ctx->fail(PS_ERR_INVALID, "ps_decode_attn: unknown request");
+        if (it->second.state != PS_REQ_RESIDENT) return ctx->fail(PS_ERR_STATE, "ps_decode_attn: request is not resident");
+        any_gated |= it->second.gated;
+    }
+    if (any_gated) {
+        int32_t rc = do_poll(ctx, nullptr);  // the copies may have landed since
+        if (rc != PS_OK) return rc;
+    }
+    std::vector<char> active((size_t)batch, 1), gated((size_t)batch, 0);
+    for (int32_t b = 0; b < batch; ++b) gated[(size_t)b] = ctx->reqs[reqs[b]].gated ? 1 : 0;
+    int32_t rc = prepare_batch(ctx, reqs, batch, active, gated, /*want_lanes=*/false, /*contended=*/false);
+    if (rc != PS_OK) return rc;
+    int32_t launched = 0;
+    return launch_layer_attn(ctx, layer, q, out, lse, ctx->meta.n_gated_rows ? ctx->ev_in[(size_t)layer] : nullptr,
+                             /*follows_own=*/false, &launched);
+}
+
+int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs, int32_t batch,
+                int64_t copy_budget_bytes, int32_t* decoded_mask, ps_step_stats* stats) {
+    if (!ctx) return PS_ERR_INVALID;
+    if (batch < 0 || (batch > 0 && !reqs)) return ctx->fail(PS_ERR_INVALID, "ps_step: bad batch");
+    const bool want_attn = q_all_layers != nullptr || out_all_layers != nullptr;
+    if (want_attn && (ctx->bk || !q_all_layers || !out_all_layers || batch > ctx->cfg.max_batch))
+        return ctx->fail(PS_ERR_INVALID, "ps_step: attention needs q and out on a device context, batch <= max_batch");
+    ps_step_stats st{};
+    int32_t reaped = 0;
+    int32_t rc = do_poll(ctx, &reaped);
+    if (rc != PS_OK) return rc;
+    st.swapouts_reaped = reaped;
+
+    // 1. the copy budget is consumed over the reload queue
+    const std::vector<PlanEntry> plan = make_plan(ctx, copy_budget_bytes);
+    std::vector<char> completes(plan.size(), 0);
+    for (size_t i = 0; i < plan.size(); ++i) {
+        st.blocks_copied += plan[i].hi - plan[i].lo;
+        completes[i] = plan[i].hi == (int32_t)ctx->reqs[plan[i].req].table.size();
+    }
+    st.h2d_bytes = st.blocks_copied * ctx->block_bytes;
+    const int L = ctx->cfg.num_layers;
+    const int64_t launches_before = ctx->launches;
+
+    // 2. the decode set: resident now, or made complete by this step's reload (those wait on events)
+    std::vector<char> active((size_t)batch, 0), gated((size_t)batch, 0);
+    for (int32_t b = 0; b < batch; ++b) {
+        auto it = ctx->reqs.find(reqs[b]);
+        if (it == ctx->reqs.end()) {
+            if (decoded_mask) decoded_mask[b] = 0;
+            continue;
+        }
+        if (it->second.state == PS_REQ_RESIDENT) {
+            active[(size_t)b] = 1;
+            gated[(size_t)b] = it->second.gated ? 1 : 0;
+        } else if (it->second.state == PS_REQ_SWAPPING_IN) {
+            for (size_t i = 0; i < plan.size(); ++i)
+                if (plan[i].req == reqs[b] && completes[i]) active[(size_t)b] = gated[(size_t)b] = 1;
+        }
+        if (decoded_mask) decoded_mask[b] = active[(size_t)b];
+        st.decoded += active[(size_t)b];
+    }
+    const bool attn = want_attn && st.decoded > 0;
+    if (attn) {
+        rc = prepare_batch(ctx, reqs, batch, active, gated, (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) == 0,
+                           /*contended=*/!plan.empty() && (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) == 0);
+        if (rc != PS_OK) return rc;
+        st.gated = ctx->meta.n_gated_rows;
+    }
+
+    // 3. per layer: reload chunk on the copy streams, then that layer's attention on the compute stream
+    if (!plan.empty()) {
+        rc = order_scatter_after_compute(ctx);
+        if (rc != PS_OK) return rc;
+    }
+    const bool sync_reload = (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) != 0 || !attn;
+    if (sync_reload)
+        for (int l = 0; l < L; ++l) {
+            rc = issue_reload_layer(ctx, l, plan);
+            if (rc != PS_OK) return rc;
+        }
+    if (attn) {
+        const int64_t layer_bytes = (int64_t)batch * ctx->cfg.num_q_heads * ctx->cfg.head_dim * 2;
+        const bool any_gated = ctx->meta.n_gated_rows > 0;
+        const bool lanes = ctx->meta.two_lanes;
+        if (lanes) {  // the reload lane starts where the compute stream stands now (metadata uploaded)
+            CK(cudaEventRecord(ctx->e_fork, ctx->compute));
+            CK(cudaStreamWaitEvent(ctx->s_lane, ctx->e_fork, 0));
+        }
+        for (int l = 0; l < L; ++l) {
+            if (!sync_reload) {
+                rc = issue_reload_layer(ctx, l, plan);
+                if (rc != PS_OK) return rc;
+            }
+            cudaEvent_t wait = nullptr;
+            if (any_gated) {
+                if (!sync_reload)
+                    wait = ctx->ev_in[(size_t)l];
+                else if (l == 0)
+                    wait = ctx->ev_in[(size_t)L - 1];  // the whole reload, once, before the first layer
+            }
+            int32_t launched = 0;
+            rc = launch_layer_attn(ctx, l, (const char*)q_all_layers + l * layer_bytes,
+                                   (char*)out_all_layers + l * layer_bytes, nullptr, wait, /*follows_own=*/l > 0, &launched);
+            if (rc != PS_OK) return rc;
+        }
+        if (lanes) {  // the step is complete on the compute stream only when the reload lane is
+            CK(cudaEventRecord(ctx->e_join, ctx->s_lane));
+            CK(cudaStreamWaitEvent(ctx->compute, ctx->e_join, 0));
+        }
+    }
+
+    // 4. request states follow what was issued
+    for (size_t i = 0; i < plan.size(); ++i) {
+        Req& r = ctx->reqs[plan[i].req];
+        for (int l = 0; l < L; ++l) {
+            rc = note_layer_issued(ctx, plan[i].req, r, l, plan[i].hi);
+            if (rc != PS_OK) return rc;
+            if (r.state == PS_REQ_RESIDENT) break;
+        }
+        if (completes[i]) st.reloads_completed++;
+    }
+    if (attn && ctx->meta.n_gated_rows > 0) {
+        // the compute stream is now ordered after every layer's reload event: later launches over
+        // these requests need no wait
+        for (int32_t b = 0; b < batch; ++b)
+            if (active[(size_t)b] && gated[(size_t)b]) {
+                auto it = ctx->reqs.find(reqs[b]);
+                if (it != ctx->reqs.end()) it->second.gated = false;
+            }
+    }
+    st.kernel_launches = (int32_t)(ctx->launches - launches_before);
+    if (stats) *stats = st;
+    return PS_OK;
+}
+
+}  // extern "C"
