@@ -51,20 +51,30 @@ def read_peaks():
     return FALLBACK_HBM_GBS, "fallback"
 
 
+def kernel_code_sha256(path):
+    """Hash of a CUDA source with comments and white space removed (a comment edit is not a kernel change)."""
+    import hashlib
+    import re
+    text = open(path).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    text = re.sub(r"//[^\n]*", "", text)
+    text = re.sub(r"\s+", "", text)
+    return hashlib.sha256(text.encode()).hexdigest()
+
+
 def read_traffic_ratio():
     """DRAM bytes per algorithmic byte of the attention kernel from the committed ncu summary, or None when
-    the kernel source has changed since that capture (the counters then describe another kernel)."""
+    the kernel's code has changed since that capture (the counters then describe another kernel)."""
     import glob
-    import hashlib
     import re
     src = os.path.join(ROOT, "paper_2512_12928_b200", "csrc", "ps_attn_kernels.cu")
     try:
-        sha = hashlib.sha256(open(src, "rb").read()).hexdigest()
+        sha = kernel_code_sha256(src)
     except OSError:
         return None
     for path in sorted(glob.glob(os.path.join(ROOT, "profiles", "decode_attn_mma_*.md"))):
         text = open(path).read()
-        m_sha = re.search(r"^kernel_source_sha256:\s*([0-9a-f]{64})", text, re.M)
+        m_sha = re.search(r"^kernel_code_sha256:\s*([0-9a-f]{64})", text, re.M)
         m_ratio = re.search(r"^dram_bytes_per_algorithmic_byte:\s*([0-9.]+)", text, re.M)
         if m_sha and m_ratio and m_sha.group(1) == sha:
             return float(m_ratio.group(1))

@@ -6,7 +6,8 @@
 // bf16 inputs, fp32 accumulation, softmax in base 2 with log2(e)/sqrt(D) folded into q.  The
 // work is split over the KV axis into items of a bounded token count; an item that is the only
 // one of its row writes the final output, otherwise it writes an unnormalised partial (running
-// max, running sum, D accumulators per head) that the merge kernel combines.
+// max, running sum, D accumulators per head); partials are combined by the merge kernel (CUDA-core
+// path) or inside the tensor-core kernel.
 //
 // The kernel is HBM-bound (G flop per KV byte), so the SIMT kernel below spends its effort on
 // 16-byte coalesced loads with many of them in flight; softmax statistics are reduced with warp
@@ -256,20 +257,25 @@ cudaError_t launch_simt(const AttnShape& sh, const void* kpool, const void* vpoo
 // ------------------------------------------------------------------------------------------------
 // Tensor-core kernel (head_dim 128, 8 KV heads, block size a multiple of 16).
 //
-// Work: the lane's contexts are cut into 16-token tiles forming one sequence.  Its first ~85 % is
-// divided evenly over the CTAs (one per SM): every CTA streams the same number of bytes whatever
-// the context-length mix.  The rest is cut into small chunks handed out through an atomic counter
-// to whichever CTA finishes first, so that an SM slowed down by a neighbour (scatter kernels, the
-// reload lane) does not stretch the launch.  An item is a (row, token range); each item produces
-// one result (final if it covers the whole row, else a partial for the merge kernel).
+// Work: the batch's contexts are cut into 16-token tiles forming one sequence, which the host divides
+// into equal static shares, one per CTA (one CTA per SM): every CTA streams the same number of bytes
+// whatever the context-length mix.  Optionally the sequence's tail is cut into chunks handed out through
+// an atomic counter to whichever CTA finishes first (the host asks for that when reload traffic makes
+// SMs unevenly fast).  An item is a (row, token range); each item produces one result: final if it
+// covers the whole row, else a partial.  The warp that delivers the last partial of a (row, KV head),
+// found through an arrival counter, combines the row's partials after its CTA's last tile.
 //
 // Data path: a tile is 16 token rows of K and 16 of V; a token row holds all 8 KV heads (2 KiB,
-// contiguous in the pool).  The producer warp issues one bulk async copy (TMA) per row -- lane r
-// the K row r, lane 16 + r the V row r -- into a 3-stage shared-memory ring signalled through
-// mbarriers; next to each stage it publishes which item and tile the stage holds, and the
-// consumers follow that stream.  Rows sit at a 2064-byte pitch so that ldmatrix over 8 tokens of one
-// head touches 8 different bank groups.  Rows past the end of a context are never copied (the ring
-// is zeroed once, so a stale row is always finite).
+// contiguous in the pool).  Stages of a 3-deep shared-memory ring are signalled through mbarriers; next to
+// each stage the producer warp publishes which item and tile it holds, and the consumers follow that
+// stream.  Tensor-map mode: per stage two box copies (cp.async.bulk.tensor) of 32 KiB through maps that
+// view a pool as (64 elements, token row, 128-byte chunk of the row) with the 128-byte swizzle, so a tile
+// lands as [chunk][token][128 B] with 16-byte units XORed by the token index and ldmatrix over 8 tokens
+// of one head touches 8 different bank groups; token rows past a context's end arrive too and are
+// cleared (V) or masked (scores) by the consumers.  Row mode: one 2 KiB bulk copy per token row at a
+// 2064-byte pitch (same bank property by padding); rows past the end are never copied, and the ring is
+// zeroed once so that a stale row is always finite.  Row mode is limited by the rate at which the copy
+// unit retires 2 KiB copies (about 6.5 TB/s over the chip), box copies by HBM.
 //
 // Math: warp w owns KV head w.  Scores: mma.m16n8k16 with the G query heads of the group as the M
 // rows (padded to 16; the padding rows of every product are dropped) and 8 tokens as N; softmax
