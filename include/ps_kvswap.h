@@ -90,7 +90,7 @@ enum ps_attn_kernel {
 typedef struct ps_config {
     int32_t num_layers;          /* L */
     int32_t num_kv_heads;        /* Hkv */
-    int32_t num_q_heads;         /* Hq, a multiple of Hkv; group G = Hq/Hkv in {1,2,4,8} */
+    int32_t num_q_heads;         /* Hq, a multiple of Hkv; group G = Hq/Hkv from 1 to 8 */
     int32_t head_dim;            /* D in {64, 128} */
     int32_t block_size;          /* s_blk, tokens per block */
     int32_t num_gpu_blocks;      /* M, blocks in every per-layer pool */
@@ -283,8 +283,8 @@ int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, flo
  * Limits (PS_ERR_INVALID with a message naming the limit when exceeded): batch <=
  * PS_STATIC_MAX_BATCH; at most 4096 work items (sum over requests of ceil(ctx / split)); their
  * partial results, num_q_heads * (head_dim + 4) floats per item, must fit in the scratch less
- * 192 KiB.  Shapes as for ps_decode_attn: head_dim 64 or 128, num_q_heads / num_kv_heads in
- * {1, 2, 4, 8}.  Results equal those of ps_decode_attn with the CUDA-core kernel.
+ * 192 KiB.  Shapes as for ps_decode_attn: head_dim 64 or 128, num_q_heads / num_kv_heads from
+ * 1 to 8.  Results equal those of ps_decode_attn with the CUDA-core kernel.
  *
  * The first call on a device looks up the scratch's device address (cudaGetSymbolAddress, with that
  * device current) and caches it; make that first call before any stream capture begins.  All calls

@@ -856,7 +856,7 @@ size_t attn_partial_bytes(const AttnShape& sh, int32_t max_parts) {
 
 bool attn_mma_supported(const AttnShape& sh) {
     const int G = sh.num_q_heads / sh.num_kv_heads;
-    return sh.head_dim == kMmaD && sh.num_kv_heads == kMmaHkv && (G == 1 || G == 2 || G == 4 || G == 8) &&
+    return sh.head_dim == kMmaD && sh.num_kv_heads == kMmaHkv && G >= 1 && G <= 8 &&
            sh.block_size % kMmaTileTokens == 0;
 }
 
@@ -869,7 +869,7 @@ cudaError_t attn_init() {
     e = cudaFuncSetAttribute(decode_attn_mma_kernel<GG, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
                              mma_smem_bytes(true));                                                               \
     if (e != cudaSuccess) return e;
-    PS_MMA_ATTR(1) PS_MMA_ATTR(2) PS_MMA_ATTR(4) PS_MMA_ATTR(8)
+    PS_MMA_ATTR(1) PS_MMA_ATTR(2) PS_MMA_ATTR(3) PS_MMA_ATTR(4) PS_MMA_ATTR(5) PS_MMA_ATTR(6) PS_MMA_ATTR(7) PS_MMA_ATTR(8)
 #undef PS_MMA_ATTR
     return cudaSuccess;
 }
@@ -925,7 +925,15 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
                                        after_own_launch, stream);
             case 2: return launch_mma<2>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
+            case 3: return launch_mma<3>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+                                       after_own_launch, stream);
             case 4: return launch_mma<4>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+                                       after_own_launch, stream);
+            case 5: return launch_mma<5>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+                                       after_own_launch, stream);
+            case 6: return launch_mma<6>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+                                       after_own_launch, stream);
+            case 7: return launch_mma<7>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
             case 8: return launch_mma<8>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
@@ -937,8 +945,10 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
     if (sh.head_dim == DD && G == GG)                                                                              \
         return launch_simt<DD, GG>(sh, kpool, vpool, q, out, lse, batch, item_begin, n_items, partials, d_status, \
                                    stream);
-    PS_SIMT_CASE(128, 1) PS_SIMT_CASE(128, 2) PS_SIMT_CASE(128, 4) PS_SIMT_CASE(128, 8)
-    PS_SIMT_CASE(64, 1) PS_SIMT_CASE(64, 2) PS_SIMT_CASE(64, 4) PS_SIMT_CASE(64, 8)
+    PS_SIMT_CASE(128, 1) PS_SIMT_CASE(128, 2) PS_SIMT_CASE(128, 3) PS_SIMT_CASE(128, 4)
+    PS_SIMT_CASE(128, 5) PS_SIMT_CASE(128, 6) PS_SIMT_CASE(128, 7) PS_SIMT_CASE(128, 8)
+    PS_SIMT_CASE(64, 1) PS_SIMT_CASE(64, 2) PS_SIMT_CASE(64, 3) PS_SIMT_CASE(64, 4)
+    PS_SIMT_CASE(64, 5) PS_SIMT_CASE(64, 6) PS_SIMT_CASE(64, 7) PS_SIMT_CASE(64, 8)
 #undef PS_SIMT_CASE
     return cudaErrorNotSupported;
 }

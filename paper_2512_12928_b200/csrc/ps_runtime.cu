@@ -275,9 +275,9 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     }
     ctx->G = cfg->num_q_heads / cfg->num_kv_heads;
     if (!ctx->bk) {
-        const bool g_ok = ctx->G == 1 || ctx->G == 2 || ctx->G == 4 || ctx->G == 8;
+        const bool g_ok = ctx->G >= 1 && ctx->G <= 8;
         if (!g_ok || (cfg->head_dim != 64 && cfg->head_dim != 128)) {
-            ctx->err = "unsupported attention shape: head_dim must be 64 or 128, Hq/Hkv in {1,2,4,8}";
+            ctx->err = "unsupported attention shape: head_dim must be 64 or 128, Hq/Hkv from 1 to 8";
             return create_fail(ctx, PS_ERR_INVALID);
         }
         if (!k_pools || !v_pools) {

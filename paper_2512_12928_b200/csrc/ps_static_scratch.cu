@@ -140,9 +140,9 @@ extern "C" int32_t ps_decode_attn_static(const void* kpool, const void* vpool, c
     if (num_q_heads % num_kv_heads != 0)
         return fail(err_buf, err_cap, PS_ERR_INVALID, "ps_decode_attn_static: num_q_heads must be a multiple of num_kv_heads");
     const int G = num_q_heads / num_kv_heads;
-    if ((head_dim != 64 && head_dim != 128) || !(G == 1 || G == 2 || G == 4 || G == 8))
+    if ((head_dim != 64 && head_dim != 128) || G < 1 || G > 8)
         return fail(err_buf, err_cap, PS_ERR_INVALID,
-                    "ps_decode_attn_static: unsupported shape (head_dim 64 or 128, Hq/Hkv in {1,2,4,8})");
+                    "ps_decode_attn_static: unsupported shape (head_dim 64 or 128, Hq/Hkv from 1 to 8)");
     char msg[400];
     if (batch > kMaxBatch) {
         snprintf(msg, sizeof msg, "ps_decode_attn_static: batch %d exceeds the fixed maximum of %d", batch, kMaxBatch);

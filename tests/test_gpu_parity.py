@@ -122,6 +122,12 @@ SHAPES = [
     (8, 64, 128, 16, B.PS_ATTN_MMA, 0),
     (8, 64, 128, 32, B.PS_ATTN_MMA, 0),
     (8, 32, 128, 48, B.PS_ATTN_MMA, 0),
+    # group sizes that are not powers of two (28 query heads over 4 KV heads is Qwen2-7B's shape)
+    (4, 28, 128, 16, B.PS_ATTN_SIMT, 0),
+    (2, 10, 64, 16, B.PS_ATTN_SIMT, 40),
+    (8, 24, 128, 16, B.PS_ATTN_MMA, 0),
+    (8, 56, 128, 32, B.PS_ATTN_MMA, 0),
+    (8, 40, 128, 16, B.PS_ATTN_MMA_ROWS, 0),
     # the same kernel fed by one bulk copy per token row instead of tensor-map boxes
     (8, 32, 128, 16, B.PS_ATTN_MMA_ROWS, 0),
     (8, 64, 128, 32, B.PS_ATTN_MMA_ROWS, 0),
