@@ -381,6 +381,30 @@ int32_t ps_select_victims(ps_ctx* ctx, const int64_t* queue, int32_t n, const do
 int32_t ps_copy_condition(int32_t l_comp, int32_t l_comp_max, int32_t b_miss, int32_t b_rem, int32_t s_blk,
                           double beta, int32_t* allowed);
 
+/* Queue ordering of the local scheduler (Section 4.2, SlideBatching, with the co-located load judgment of
+ * Eq. "phi(Q)" and the starvation rule), as arithmetic for callers that want to drive the block management
+ * in the paper's closed loop: the ordered queue feeds ps_select_victims (tail) and the reload order (head),
+ * *t_budget_us feeds ps_copy_budget.
+ *   exec_us[i]   : estimated execution time of request i in the coming batch (Section 4.1)
+ *   remain_us[i] : time left to its deadline;  weight[i] : its token-level gain;  density = weight / exec
+ *   waited_us    : waiting times, or NULL (no starvation rule)
+ *   t_budget = max(min_i remain, eta);  phi = t_budget / (t_budget - t_c) * sum_i exec  (needs t_budget > t_c)
+ *   request i is URGENT if remain[i] < gamma * phi, else NORMAL
+ *   order: starving requests (waited > tau) first, in input order; then URGENT by density, largest first;
+ *          then NORMAL by remaining time, smallest first; ties keep the input order.
+ *   order   : out, n indices into the input arrays, head of the queue first
+ *   urgent  : out, n flags per input index (1 urgent, 0 normal, 2 starving), or NULL
+ * Errors: PS_ERR_INVALID (n < 0, null arrays, non-positive exec, t_budget <= t_c). */
+typedef struct ps_sched_params {
+    double eta_us;    /* lower bound of the latency budget */
+    double gamma;     /* aggressiveness coefficient */
+    double t_c_us;    /* constant per-batch overhead */
+    double tau_us;    /* starvation threshold (used only with waited_us) */
+} ps_sched_params;
+int32_t ps_order_queue(int32_t n, const double* exec_us, const double* remain_us, const double* weight,
+                       const double* waited_us, const ps_sched_params* params, int32_t* order, int32_t* urgent,
+                       double* t_budget_us);
+
 /* ---- completion ------------------------------------------------------------------------- */
 
 /* Non-blocking: reaps finished offloads (in issue order), releases host images of finished

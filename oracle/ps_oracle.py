@@ -492,6 +492,32 @@ class PsOracle:
 # Brute-force restatements for tiny inputs (pure Python loops and floats)
 # -------------------------------------------------------------------------------------------------
 
+def order_queue(exec_t: Sequence[float], remain: Sequence[float], weight: Sequence[float], eta: float, gamma: float,
+                t_c: float, waited: Optional[Sequence[float]] = None, tau: float = 0.0):
+    """The request ordering of the SlideBatching algorithm (Section 4.2) with the co-located load judgment.
+
+    The latency budget is the smallest remaining deadline, bounded below by eta.  A request is URGENT if its
+    remaining time is below gamma * phi(Q), phi(Q) = t_budget / (t_budget - t_c) * sum of exec.  URGENT requests
+    come first in descending density (weight / exec), the others in ascending remaining time; a request whose
+    waiting time exceeds the starvation threshold tau is promoted to the head.  Returns (order as indices,
+    class per index: 2 starving / 1 urgent / 0 normal, t_budget)."""
+    n = len(exec_t)
+    t_budget = max(min(remain), eta) if n else eta
+    if n == 0:
+        return [], [], t_budget
+    phi = t_budget / (t_budget - t_c) * sum(exec_t)
+    cls = []
+    for i in range(n):
+        if waited is not None and waited[i] > tau:
+            cls.append(2)
+        else:
+            cls.append(1 if remain[i] < gamma * phi else 0)
+    starving = [i for i in range(n) if cls[i] == 2]
+    urgent = sorted((i for i in range(n) if cls[i] == 1), key=lambda i: -(weight[i] / exec_t[i]))   # stable
+    normal = sorted((i for i in range(n) if cls[i] == 0), key=lambda i: remain[i])
+    return starving + urgent + normal, cls, t_budget
+
+
 def copy_condition(l_comp: int, l_comp_max: int, b_miss: int, b_rem: int, s_blk: int, beta: float) -> bool:
     """"Put it Together": all missing blocks are copied if the remaining budget covers them; otherwise partial
     copying is enabled only when l_comp reaches the maximum computable-token limit of the round, or the ratio

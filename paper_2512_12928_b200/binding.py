@@ -31,7 +31,7 @@ EXPORTS = [
     "ps_swap_in_layer", "ps_missing_blocks", "ps_decode_attn", "ps_step", "ps_poll", "ps_sync",
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
     "ps_decode_attn_static", "ps_copy_budget", "ps_offload_progress", "ps_host_blocks", "ps_host_segment",
-    "ps_select_victims", "ps_copy_condition",
+    "ps_select_victims", "ps_copy_condition", "ps_order_queue",
 ]
 
 
@@ -74,6 +74,10 @@ class PsProfile(C.Structure):
 class PsBudgetModel(C.Structure):
     _fields_ = [("a_d_us_per_token", C.c_double), ("b_d_us", C.c_double), ("t_c_us", C.c_double),
                 ("t_block_us", C.c_double), ("t_budget_us", C.c_double)]
+
+
+class PsSchedParams(C.Structure):
+    _fields_ = [("eta_us", C.c_double), ("gamma", C.c_double), ("t_c_us", C.c_double), ("tau_us", C.c_double)]
 
 
 class PsTraceSpan(C.Structure):
@@ -133,6 +137,8 @@ def load() -> C.CDLL:
         "ps_host_segment": (i32, [vp, i64, i32, C.POINTER(vp), p64, p32, p32, p32]),
         "ps_select_victims": (i32, [vp, p64, i32, C.POINTER(C.c_double), C.c_double, C.c_double, i32, p64, i32, p32, p32]),
         "ps_copy_condition": (i32, [i32, i32, i32, i32, i32, C.c_double, p32]),
+        "ps_order_queue": (i32, [i32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double),
+                                 C.POINTER(C.c_double), C.POINTER(PsSchedParams), p32, p32, C.POINTER(C.c_double)]),
         "ps_copy_budget": (i32, [vp, p64, i32, C.POINTER(PsBudgetModel), p64, p64, p32]),
         "ps_decode_attn_static": (i32, [vp, vp, vp, vp, vp, vp, i32, p32, i32, i32, i32, i32, i32, i32, i32, vp, vp,
                                         C.c_char_p, i32]),
@@ -178,6 +184,17 @@ def ps_decode_attn_static(kpool, vpool, q, out, block_tables, ctx_lens: Sequence
                                       arr, batch, num_kv_heads, num_q_heads, head_dim, block_size, num_gpu_blocks,
                                       kv_split_tokens, ptr(status_word), C.c_void_p(stream or None), err, 512)
     return rc, err.value.decode()
+
+
+def ps_order_queue(exec_us, remain_us, weight, *, eta: float, gamma: float, t_c: float, waited_us=None, tau: float = 0.0):
+    """SlideBatching's queue order: (status, order as indices head first, classes per index, t_budget)."""
+    n = len(exec_us)
+    arr = lambda v: (C.c_double * max(n, 1))(*[float(x) for x in v])
+    params = PsSchedParams(eta, gamma, t_c, tau)
+    order, cls, tb = (C.c_int32 * max(n, 1))(), (C.c_int32 * max(n, 1))(), C.c_double()
+    rc = load().ps_order_queue(n, arr(exec_us), arr(remain_us), arr(weight), arr(waited_us) if waited_us is not None else None,
+                               C.byref(params), order, cls, C.byref(tb))
+    return rc, list(order[:n]), list(cls[:n]), tb.value
 
 
 def ps_copy_condition(l_comp: int, l_comp_max: int, b_miss: int, b_rem: int, s_blk: int, beta: float):

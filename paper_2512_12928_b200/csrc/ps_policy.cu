@@ -100,6 +100,40 @@ int32_t ps_select_victims(ps_ctx* ctx, const int64_t* queue, int32_t n, const do
     return PS_OK;
 }
 
+int32_t ps_order_queue(int32_t n, const double* exec_us, const double* remain_us, const double* weight,
+                       const double* waited_us, const ps_sched_params* params, int32_t* order, int32_t* urgent,
+                       double* t_budget_us) {
+    if (n < 0 || !params || (n > 0 && (!exec_us || !remain_us || !weight || !order))) return PS_ERR_INVALID;
+    double t_min = INFINITY, sum_exec = 0.0;
+    for (int32_t i = 0; i < n; ++i) {
+        if (!(exec_us[i] > 0.0)) return PS_ERR_INVALID;
+        t_min = std::min(t_min, remain_us[i]);
+        sum_exec += exec_us[i];
+    }
+    const double t_budget = n > 0 ? std::max(t_min, params->eta_us) : params->eta_us;
+    if (t_budget_us) *t_budget_us = t_budget;
+    if (n == 0) return PS_OK;
+    if (!(t_budget > params->t_c_us)) return PS_ERR_INVALID;
+    const double phi = t_budget / (t_budget - params->t_c_us) * sum_exec;
+    std::vector<int32_t> cls((size_t)n);  // 2 starving, 1 urgent, 0 normal
+    for (int32_t i = 0; i < n; ++i) {
+        if (waited_us && waited_us[i] > params->tau_us)
+            cls[(size_t)i] = 2;
+        else
+            cls[(size_t)i] = remain_us[i] < params->gamma * phi ? 1 : 0;
+        order[i] = i;
+    }
+    std::stable_sort(order, order + n, [&](int32_t a, int32_t b) {
+        if (cls[(size_t)a] != cls[(size_t)b]) return cls[(size_t)a] > cls[(size_t)b];
+        if (cls[(size_t)a] == 1) return weight[a] / exec_us[a] > weight[b] / exec_us[b];
+        if (cls[(size_t)a] == 0) return remain_us[a] < remain_us[b];
+        return false;
+    });
+    if (urgent)
+        for (int32_t i = 0; i < n; ++i) urgent[i] = cls[(size_t)i];
+    return PS_OK;
+}
+
 int32_t ps_copy_condition(int32_t l_comp, int32_t l_comp_max, int32_t b_miss, int32_t b_rem, int32_t s_blk,
                           double beta, int32_t* allowed) {
     if (!allowed || l_comp < 0 || l_comp_max < 0 || b_miss < 0 || b_rem < 0 || s_blk <= 0 || !(beta > 1.0))
