@@ -82,9 +82,9 @@ enum ps_flags {
 enum ps_attn_kernel {
     PS_ATTN_AUTO = 0,
     PS_ATTN_SIMT = 1,   /* CUDA-core kernel, warp-shuffle softmax; any supported shape */
-    PS_ATTN_MMA = 2,    /* tensor-core kernel (head_dim 128, 8 KV heads): tiles staged by tensor-map box copies
-                           when the driver accepts the maps, else as PS_ATTN_MMA_ROWS */
-    PS_ATTN_MMA_ROWS = 3 /* the same kernel with one bulk copy per token row */
+    PS_ATTN_MMA = 2,    /* tensor-core kernel (head_dim 128; 1, 2, 4 or 8 KV heads): tiles staged by tensor-map
+                           box copies when the driver accepts the maps, else (8 KV heads) as PS_ATTN_MMA_ROWS */
+    PS_ATTN_MMA_ROWS = 3 /* the same kernel with one bulk copy per token row (8 KV heads only) */
 };
 
 typedef struct ps_config {

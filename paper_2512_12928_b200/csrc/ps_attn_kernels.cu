@@ -296,7 +296,8 @@ constexpr int kMmaSlabBytes = kMmaTileTokens * kMmaPitch; // one K (or V) tile i
 constexpr int kMmaStageBytes = 2 * kMmaSlabBytes;
 constexpr int kMmaRingBytes = kMmaStages * kMmaStageBytes;
 constexpr int kMmaMaxPending = 14;                        // rows a warp may note for combining after its last tile
-constexpr int kMmaCtrlBytes = 128 + 8 * 16 * 4;           // barriers, stage descriptors, abort word; pending-row lists
+constexpr int kMmaCtrlBytes = 128 + 8 * 16 * 4 + 128;     // barriers, stage descriptors, abort word; pending-row lists;
+                                                          // exchange barriers
 constexpr int kMmaConsumerWarps = kMmaHkv;
 constexpr int kMmaThreads = (kMmaConsumerWarps + 1) * 32;
 constexpr int kMmaPartStride = kMmaD + 4;                 // floats per (part, query head): 16-byte aligned rows
@@ -310,8 +311,15 @@ constexpr int kTmaStageBytes = 2 * kTmaTileBytes;              // 65536
 constexpr int kTmaRingBytes = kMmaStages * kTmaStageBytes;
 constexpr int kTmaAlign = 1024;                                // the swizzle pattern repeats every 1 KiB
 
-constexpr int mma_smem_bytes(bool tma) {
-    return tma ? kTmaRingBytes + kTmaAlign + kMmaCtrlBytes : kMmaRingBytes + kMmaCtrlBytes;
+// Fewer than 8 KV heads (tensor-map mode only): a stage still holds 64 KiB, now 8 / HKV sub-tiles of 16 tokens
+// each (one K and one V box per sub-tile, possibly from different blocks), and the 8 consumer warps are
+// (head, sub-tile) pairs: warp w works on head w % HKV, sub-tile w / HKV.  The warps of one head each keep their
+// own softmax state over every (8 / HKV)-th 16-token slice of the row and combine the states at the end of an
+// item through a small exchange area (34 floats per lane of every warp with a sub-tile index above 0).
+constexpr int mma_subs(int hkv) { return kMmaHkv / hkv; }
+constexpr int mma_xchg_bytes(int hkv) { return (kMmaHkv - hkv) * 32 * 34 * 4; }
+constexpr int mma_smem_bytes(bool tma, int hkv) {
+    return tma ? kTmaRingBytes + kTmaAlign + kMmaCtrlBytes + mma_xchg_bytes(hkv) : kMmaRingBytes + kMmaCtrlBytes;
 }
 
 struct StageDesc {  // published by the producer next to every ring stage
@@ -408,11 +416,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
 // Combines the parts of batch row b for the G query heads of KV head h (one warp; every part has been
 // delivered and fenced).  Parts are combined in part order, whoever calls.  The loads of all G heads
 // are issued together, two parts at a time.  Re-arms the row's arrival counter.
-template <int G>
+template <int G, int HKV>
 __device__ __forceinline__ void merge_row(int b, int h, int lane, const AttnBatch& batch,
                                           const float* __restrict__ partials, __nv_bfloat16* __restrict__ out,
                                           float* __restrict__ lse, int32_t* __restrict__ row_done) {
-    constexpr int Hq = kMmaHkv * G;
+    constexpr int Hq = HKV * G;
     __threadfence();
     const int n = batch.row_parts[b];
     const float* base = partials + ((int64_t)batch.row_first_part[b] * Hq + h * G) * kMmaPartStride;
@@ -483,10 +491,10 @@ __device__ __forceinline__ void merge_row(int b, int h, int lane, const AttnBatc
         if (lse != nullptr && lane == 0)
             lse[(int64_t)b * Hq + hq] = Ls[gg] > 0.f ? (M[gg] + log2f(Ls[gg])) * kLn2 : -CUDART_INF_F;
     }
-    if (lane == 0) row_done[b * kMmaHkv + h] = 0;  // every part has arrived: re-arm for the next launch
+    if (lane == 0) row_done[b * HKV + h] = 0;  // every part has arrived: re-arm for the next launch
 }
 
-template <int G, bool kTma>
+template <int G, int HKV, bool kTma>
 __global__ void __launch_bounds__(kMmaThreads, 1)
 decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloat16* __restrict__ vpool,
                        const __grid_constant__ CUtensorMap kmap, const __grid_constant__ CUtensorMap vmap,
@@ -495,10 +503,14 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                        int32_t num_blocks, float* __restrict__ partials, int32_t* __restrict__ sched,
                        int32_t* __restrict__ row_done, float scale_log2e, int32_t* status) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    constexpr int Hq = kMmaHkv * G;
+    static_assert(HKV == kMmaHkv || kTma, "fewer than 8 KV heads need the tensor-map mode");
+    constexpr int Hq = HKV * G;
+    constexpr int kSubs = kMmaHkv / HKV;                         // 16-token sub-tiles per stage
+    constexpr int kSubBytes = kMmaTileTokens * HKV * kMmaD * 2;   // one K (or V) sub-tile in tensor-map mode
+    constexpr int kStageTokens = kMmaTileTokens * kSubs;
     constexpr int kStageBytes = kTma ? kTmaStageBytes : kMmaStageBytes;
     constexpr int kRingBytes = kTma ? kTmaRingBytes : kMmaRingBytes;
-    constexpr int kVOff = kTma ? kTmaTileBytes : kMmaSlabBytes;   // V tile inside a stage
+    constexpr int kVOff = kTma ? kTmaTileBytes : kMmaSlabBytes;   // V tiles inside a stage
     // the swizzled layout needs the ring on a 1 KiB boundary of the shared address space
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t ring = kTma ? (raw + kTmaAlign - 1) & ~(uint32_t)(kTmaAlign - 1) : raw;
@@ -509,6 +521,9 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
     // 48 bytes of barriers, then the stage descriptors and the abort word
     volatile StageDesc* sdesc = reinterpret_cast<volatile StageDesc*>(ctrl + 64);
     volatile int32_t* abort_word = reinterpret_cast<volatile int32_t*>(ctrl + 64 + 16 * kMmaStages);
+    const uint32_t bar_xfull = bar_full + 640;              // [HKV] exchange: states of a head's other warps are in
+    const uint32_t bar_xempty = bar_xfull + 8 * kMmaHkv;    // [HKV] exchange: the combining warp has read them
+    float* xchg = reinterpret_cast<float*>(ctrl + kMmaCtrlBytes);
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
@@ -528,6 +543,11 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             mbar_init(bar_full + 8 * s, 1);
             mbar_init(bar_empty + 8 * s, kMmaConsumerWarps);
         }
+        if (kSubs > 1)
+            for (int hh = 0; hh < HKV; ++hh) {
+                mbar_init(bar_xfull + 8 * hh, kSubs - 1);
+                mbar_init(bar_xempty + 8 * hh, 1);
+            }
         *abort_word = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -564,7 +584,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             }
             const AttnItem item = batch.items[it];
             const int32_t* table = batch.block_tables + (int64_t)item.b * batch.table_stride;
-            const int ntiles = max(1, (item.t_end - item.t_begin + kMmaTileTokens - 1) / kMmaTileTokens);
+            const int ntiles = max(1, (item.t_end - item.t_begin + kStageTokens - 1) / kStageTokens);
             // Block ids are read 32 at a time, one per lane, a window ahead of their use: the table read
             // never sits between a freed stage and the copies that refill it.
             const int last_blk = (max(item.t_end, 1) - 1) / block_size;
@@ -573,10 +593,10 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             int ids_next = win + 32 + lane <= last_blk ? __ldg(table + win + 32 + lane) : 0;
             for (int ti = 0; ti < ntiles; ++ti, ++n) {
                 const int s = n % kMmaStages;
-                const int t0 = item.t_begin + ti * kMmaTileTokens;
-                const int rows = max(0, min(kMmaTileTokens, item.t_end - t0));
+                const int t0 = item.t_begin + ti * kStageTokens;
+                const int rows = max(0, min(kStageTokens, item.t_end - t0));
                 const int blk = block_shift >= 0 ? (t0 >> block_shift) : (t0 / block_size);
-                if (blk >= win + 32) {  // tiles advance by at most one block: the next window is the one ahead
+                if (blk >= win + 32) {  // a stage starts at most 8 blocks after the last: the next window is the one ahead
                     win += 32;
                     ids = ids_next;
                     ids_next = win + 32 + lane <= last_blk ? __ldg(table + win + 32 + lane) : 0;
@@ -584,34 +604,41 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                 if (n >= kMmaStages) ok = mbar_wait(bar_empty + 8 * s, ((n / kMmaStages) - 1) & 1, abort_word, status);
                 if (!ok) break;
                 const uint32_t full = bar_full + 8 * s;
-                int id = __shfl_sync(0xffffffffu, ids, (blk - win) & 31);
-                int slot = 0;
+                // this lane's sub-tile (tensor-map mode: lanes 2 s and 2 s + 1 copy K and V of sub-tile s; row mode:
+                // every lane looks at the stage's only sub-tile) and its block: ids of the current or next window
+                const int my_sub = kTma ? (lane >> 1) : 0;
+                const int my_t = t0 + kMmaTileTokens * my_sub;
+                const bool my_valid = my_sub < kSubs && kMmaTileTokens * my_sub < rows;
+                const int my_blk = my_valid ? (block_shift >= 0 ? (my_t >> block_shift) : (my_t / block_size)) : blk;
+                const int id_a = __shfl_sync(0xffffffffu, ids, (my_blk - win) & 31);
+                const int id_b = __shfl_sync(0xffffffffu, ids_next, (my_blk - win) & 31);
+                const int id = my_blk - win < 32 ? id_a : id_b;
+                const int slot = my_t - my_blk * block_size;
+                const bool bad = my_valid && (unsigned)id >= (unsigned)num_blocks;
                 bool copy = rows > 0;
-                if (copy) {
-                    slot = t0 - blk * block_size;
-                    if ((unsigned)id >= (unsigned)num_blocks) {  // nothing is copied and the tile is skipped
-                        *(volatile int32_t*)status = 2;
-                        copy = false;
-                    }
+                if (__any_sync(0xffffffffu, bad)) {  // nothing is copied and the tile is skipped
+                    *(volatile int32_t*)status = 2;
+                    copy = false;
                 }
+                const int n_subs = (rows + kMmaTileTokens - 1) / kMmaTileTokens;
                 if (lane == 0) {
                     sdesc[s].item = it;
                     sdesc[s].t0 = t0;
                     sdesc[s].rows = copy ? rows : 0;
                     sdesc[s].flags = (ti == 0 ? kFlagFirst : 0) | (ti == ntiles - 1 ? kFlagLast : 0);
                     if (copy)
-                        mbar_expect_tx(full, kTma ? (uint32_t)kTmaStageBytes : (uint32_t)rows * 2u * kMmaRowBytes);
+                        mbar_expect_tx(full, kTma ? (uint32_t)(n_subs * 2 * kSubBytes) : (uint32_t)rows * 2u * kMmaRowBytes);
                     else
                         mbar_arrive(full);
                 }
                 __syncwarp();  // descriptor and expected byte count are posted before any copy can complete
                 if (copy) {
                     if (kTma) {
-                        // whole boxes of 16 token rows: the tile lies inside one block, so rows past the context's
+                        // whole boxes of 16 token rows: a sub-tile lies inside one block, so rows past the context's
                         // end are in bounds (the consumers clear them in V and mask them in the scores)
-                        if (lane < 2)
-                            tensor_g2s(ring + s * kStageBytes + lane * kVOff, lane == 0 ? &kmap : &vmap,
-                                       id * block_size + slot, full, kv_policy);
+                        if (my_valid)
+                            tensor_g2s(ring + s * kStageBytes + (lane & 1) * kVOff + my_sub * kSubBytes,
+                                       (lane & 1) ? &vmap : &kmap, id * block_size + slot, full, kv_policy);
                     } else {
                         const int r = lane & 15;
                         if (r < rows) {
@@ -642,8 +669,9 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             }
         }
     } else {
-        // ------------------------------------------------ consumers: warp = KV head
-        const int h = warp;
+        // ------------------------------------------------ consumers: warp = (KV head, 16-token sub-tile of the stage)
+        const int h = warp % HKV;
+        const int sub = warp / HKV;
         const int g = lane >> 2;  // mma row = query head inside the group (real if g < G)
         const int t = lane & 3;
         const int ld_row = lane & 7;
@@ -655,9 +683,9 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
         // Row-copy mode: token rows at a 2064-byte pitch, head h at byte 256 h.  Tensor-map mode: head h is the
         // 128-byte chunks 2h and 2h + 1, each [16 tokens][128 B]; the 16-byte unit u of a token row sits at
         // unit u ^ (token mod 8).  k_x[u] / v_x[u]: byte offset of the lane's unit for dims 32 u .. 32 u + 15.
-        const uint32_t k_lane_off = kTma ? (uint32_t)(2 * h * 2048 + k_tok * 128)
+        const uint32_t k_lane_off = kTma ? (uint32_t)(sub * kSubBytes + 2 * h * 2048 + k_tok * 128)
                                          : (uint32_t)(k_tok * kMmaPitch + h * 256 + k_half * 16);
-        const uint32_t v_lane_off = kTma ? (uint32_t)(kVOff + 2 * h * 2048 + v_tok * 128)
+        const uint32_t v_lane_off = kTma ? (uint32_t)(kVOff + sub * kSubBytes + 2 * h * 2048 + v_tok * 128)
                                          : (uint32_t)(kVOff + v_tok * kMmaPitch + h * 256 + v_half * 16);
         uint32_t k_x[4], v_x[4];
 #pragma unroll
@@ -671,6 +699,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
         int item_b = 0, item_part = 0, item_nparts = 1;
         volatile int32_t* pending = reinterpret_cast<volatile int32_t*>(ctrl + 128) + warp * 16;
         int n_pend = 0;
+        int xphase = 0;  // item ends seen so far: phase of the exchange barriers
         bool ok = true;
 #pragma unroll
         for (int j = 0; j < 8; ++j) qa[j][0] = qa[j][1] = 0u;
@@ -683,7 +712,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             if (!ok) break;
             const int flags = sdesc[s].flags;
             if (flags & kFlagEnd) break;
-            const int rows = sdesc[s].rows;
+            const int rows = max(0, min(kMmaTileTokens, sdesc[s].rows - kMmaTileTokens * sub));  // of this warp's sub-tile
             if (flags & kFlagFirst) {
                 const AttnItem* ip = batch.items + sdesc[s].item;
                 item_b = ip->b;
@@ -707,8 +736,9 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                     // (a zero weight times a non-finite leftover would poison the row's output)
                     if (lane < 16)
                         for (int r = rows; r < kMmaTileTokens; ++r)
-                            *reinterpret_cast<uint4*>(smem + s * kStageBytes + kVOff + (2 * h + (lane >> 3)) * 2048 + r * 128 +
-                                                      (lane & 7) * 16) = make_uint4(0, 0, 0, 0);
+                            *reinterpret_cast<uint4*>(smem + s * kStageBytes + kVOff + sub * kSubBytes +
+                                                      (2 * h + (lane >> 3)) * 2048 + r * 128 + (lane & 7) * 16) =
+                                make_uint4(0, 0, 0, 0);
                     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // before the stage is refilled
                     __syncwarp();
                 }
@@ -755,7 +785,45 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_empty + 8 * s);
 
-            if (flags & kFlagLast) {
+            if ((flags & kFlagLast) && kSubs > 1) {
+                // the warps of a head combine their softmax states: the others hand theirs to the warp of sub-tile 0
+                // (same fragment layout in every warp, so lane i combines with lane i)
+                if (sub > 0) {
+                    if (xphase > 0) ok = mbar_wait(bar_xempty + 8 * h, (xphase - 1) & 1, abort_word, status);
+                    if (!ok) break;
+                    float* mine = xchg + ((size_t)((sub - 1) * HKV + h) * 32 + lane) * 34;
+                    mine[0] = m_run;
+                    mine[1] = l_run;
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        mine[2 + 2 * i] = o[i][0];
+                        mine[3 + 2 * i] = o[i][1];
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_xfull + 8 * h);
+                } else {
+                    ok = mbar_wait(bar_xfull + 8 * h, xphase & 1, abort_word, status);
+                    if (!ok) break;
+#pragma unroll 1
+                    for (int ss = 1; ss < kSubs; ++ss) {
+                        const float* other = xchg + ((size_t)((ss - 1) * HKV + h) * 32 + lane) * 34;
+                        const float m_o = other[0];
+                        const float m_new = fmaxf(m_run, m_o);
+                        const float a = exp2f(m_run - m_new), b = exp2f(m_o - m_new);
+                        m_run = m_new;
+                        l_run = l_run * a + other[1] * b;
+#pragma unroll
+                        for (int i = 0; i < 16; ++i) {
+                            o[i][0] = o[i][0] * a + other[2 + 2 * i] * b;
+                            o[i][1] = o[i][1] * a + other[3 + 2 * i] * b;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(bar_xempty + 8 * h);
+                }
+                ++xphase;
+            }
+            if ((flags & kFlagLast) && sub == 0) {
                 float L = l_run;
                 L += __shfl_xor_sync(0xffffffffu, L, 1);
                 L += __shfl_xor_sync(0xffffffffu, L, 2);
@@ -789,14 +857,14 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                     __threadfence();
                     __syncwarp();
                     int prev = 0;
-                    if (lane == 0) prev = atomicAdd(row_done + item_b * kMmaHkv + h, 1);
+                    if (lane == 0) prev = atomicAdd(row_done + item_b * HKV + h, 1);
                     prev = __shfl_sync(0xffffffffu, prev, 0);
                     if (prev == item_nparts - 1) {
                         if (n_pend < kMmaMaxPending) {
                             if (lane == 0) pending[n_pend] = item_b;
                             ++n_pend;
                         } else {
-                            merge_row<G>(item_b, h, lane, batch, partials, out, lse, row_done);
+                            merge_row<G, HKV>(item_b, h, lane, batch, partials, out, lse, row_done);
                         }
                     }
                 }
@@ -804,7 +872,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
         }
         if (ok) {
             __syncwarp();
-            for (int p = 0; p < n_pend; ++p) merge_row<G>(pending[p], h, lane, batch, partials, out, lse, row_done);
+            for (int p = 0; p < n_pend; ++p) merge_row<G, HKV>(pending[p], h, lane, batch, partials, out, lse, row_done);
         }
     }
     // A launch does not complete before the launch it was made programmatically dependent on has completed:
@@ -812,16 +880,17 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
     dep_wait();
 }
 
-template <int G>
+template <int G, int HKV>
 cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool, const AttnTensorMaps* maps, const void* q,
                        void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials, int32_t* sched,
                        int32_t* row_done, int32_t* d_status, bool after_own_launch, cudaStream_t stream) {
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)kMmaD);
     static_assert(sizeof(CUtensorMap) == sizeof(maps->k), "AttnTensorMaps must hold driver tensor maps");
+    if (HKV != kMmaHkv && maps == nullptr) return cudaErrorNotSupported;
     cudaLaunchConfig_t cfg{};
     cfg.gridDim = dim3((unsigned)batch.n_cta[lane]);
     cfg.blockDim = dim3(kMmaThreads);
-    cfg.dynamicSmemBytes = (size_t)mma_smem_bytes(maps != nullptr);
+    cfg.dynamicSmemBytes = (size_t)mma_smem_bytes(maps != nullptr, HKV);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -842,10 +911,28 @@ cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool
     __nv_bfloat16* op = (__nv_bfloat16*)out;
     const int32_t shift = shift_of(sh.block_size);
     if (maps != nullptr)
-        return cudaLaunchKernelEx(&cfg, decode_attn_mma_kernel<G, true>, kp, vp, km, vm, qp, op, lse, batch, lane,
+        return cudaLaunchKernelEx(&cfg, decode_attn_mma_kernel<G, HKV, true>, kp, vp, km, vm, qp, op, lse, batch, lane,
                                   sh.block_size, shift, sh.num_blocks, partials, sched, row_done, scale_log2e, d_status);
-    return cudaLaunchKernelEx(&cfg, decode_attn_mma_kernel<G, false>, kp, vp, km, vm, qp, op, lse, batch, lane,
-                              sh.block_size, shift, sh.num_blocks, partials, sched, row_done, scale_log2e, d_status);
+    if constexpr (HKV == kMmaHkv)
+        return cudaLaunchKernelEx(&cfg, decode_attn_mma_kernel<G, HKV, false>, kp, vp, km, vm, qp, op, lse, batch, lane,
+                                  sh.block_size, shift, sh.num_blocks, partials, sched, row_done, scale_log2e, d_status);
+    return cudaErrorNotSupported;
+}
+
+template <int G>
+cudaError_t launch_mma_hkv(const AttnShape& sh, const void* kpool, const void* vpool, const AttnTensorMaps* maps,
+                           const void* q, void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials,
+                           int32_t* sched, int32_t* row_done, int32_t* d_status, bool after_own_launch,
+                           cudaStream_t stream) {
+    switch (sh.num_kv_heads) {
+#define PS_HKV_CASE(HH)                                                                                              \
+    case HH:                                                                                                         \
+        return launch_mma<G, HH>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status, \
+                                 after_own_launch, stream);
+        PS_HKV_CASE(1) PS_HKV_CASE(2) PS_HKV_CASE(4) PS_HKV_CASE(8)
+#undef PS_HKV_CASE
+    }
+    return cudaErrorNotSupported;
 }
 
 }  // namespace
@@ -856,27 +943,31 @@ size_t attn_partial_bytes(const AttnShape& sh, int32_t max_parts) {
 
 bool attn_mma_supported(const AttnShape& sh) {
     const int G = sh.num_q_heads / sh.num_kv_heads;
-    return sh.head_dim == kMmaD && sh.num_kv_heads == kMmaHkv && G >= 1 && G <= 8 &&
+    const int hkv = sh.num_kv_heads;
+    return sh.head_dim == kMmaD && (hkv == 1 || hkv == 2 || hkv == 4 || hkv == 8) && G >= 1 && G <= 8 &&
            sh.block_size % kMmaTileTokens == 0;
 }
 
+int32_t attn_mma_tile_tokens(const AttnShape& sh) { return kMmaTileTokens * mma_subs(sh.num_kv_heads); }
+
 cudaError_t attn_init() {
     cudaError_t e;
-#define PS_MMA_ATTR(GG)                                                                                           \
-    e = cudaFuncSetAttribute(decode_attn_mma_kernel<GG, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,      \
-                             mma_smem_bytes(false));                                                              \
-    if (e != cudaSuccess) return e;                                                                               \
-    e = cudaFuncSetAttribute(decode_attn_mma_kernel<GG, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,       \
-                             mma_smem_bytes(true));                                                               \
+#define PS_MMA_ATTR_ONE(GG, HH, TT)                                                                                   \
+    e = cudaFuncSetAttribute(decode_attn_mma_kernel<GG, HH, TT>, cudaFuncAttributeMaxDynamicSharedMemorySize,         \
+                             mma_smem_bytes(TT, HH));                                                                 \
     if (e != cudaSuccess) return e;
+#define PS_MMA_ATTR(GG)                                                                                               \
+    PS_MMA_ATTR_ONE(GG, 8, false) PS_MMA_ATTR_ONE(GG, 8, true) PS_MMA_ATTR_ONE(GG, 4, true) PS_MMA_ATTR_ONE(GG, 2, true) \
+        PS_MMA_ATTR_ONE(GG, 1, true)
     PS_MMA_ATTR(1) PS_MMA_ATTR(2) PS_MMA_ATTR(3) PS_MMA_ATTR(4) PS_MMA_ATTR(5) PS_MMA_ATTR(6) PS_MMA_ATTR(7) PS_MMA_ATTR(8)
 #undef PS_MMA_ATTR
+#undef PS_MMA_ATTR_ONE
     return cudaSuccess;
 }
 
 // Tensor maps over one layer's pools, seen as rank-3 tensors (64 elements = 128 bytes, token row, 128-byte chunk
-// of the row): strides 2 KiB per token row and 128 bytes per chunk, box 64 x 16 token rows x 16 chunks, 128-byte
-// swizzle.  The driver entry point is looked up at run time (the library does not link against the driver).
+// of the row): strides one token row (256 bytes per KV head) and 128 bytes per chunk, box 64 x 16 token rows x all
+// chunks of a row, 128-byte swizzle.  The driver entry point is looked up at run time (the library does not link against the driver).
 cudaError_t attn_make_tensor_maps(const AttnShape& sh, const void* kpool, const void* vpool, AttnTensorMaps* out) {
     if (!attn_mma_supported(sh)) return cudaErrorNotSupported;
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
@@ -891,9 +982,10 @@ cudaError_t attn_make_tensor_maps(const AttnShape& sh, const void* kpool, const 
         if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
         encode = (EncodeFn)fn;
     }
-    const cuuint64_t dims[3] = {64, (cuuint64_t)sh.num_blocks * (cuuint64_t)sh.block_size, (cuuint64_t)(kMmaRowBytes / 128)};
-    const cuuint64_t strides[2] = {(cuuint64_t)kMmaRowBytes, 128};   // bytes: token row, then chunk of the row
-    const cuuint32_t box[3] = {64, (cuuint32_t)kMmaTileTokens, (cuuint32_t)(kMmaRowBytes / 128)};
+    const cuuint64_t row_bytes = (cuuint64_t)sh.num_kv_heads * kMmaD * 2;
+    const cuuint64_t dims[3] = {64, (cuuint64_t)sh.num_blocks * (cuuint64_t)sh.block_size, row_bytes / 128};
+    const cuuint64_t strides[2] = {row_bytes, 128};   // bytes: token row, then chunk of the row
+    const cuuint32_t box[3] = {64, (cuuint32_t)kMmaTileTokens, (cuuint32_t)(row_bytes / 128)};
     const cuuint32_t estr[3] = {1, 1, 1};
     const void* pools[2] = {kpool, vpool};
     unsigned char* dst[2] = {out->k, out->v};
@@ -921,21 +1013,21 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
         if (!attn_mma_supported(sh) || batch.n_cta[lane] <= 0 || sched == nullptr || row_done == nullptr)
             return cudaErrorNotSupported;
         switch (G) {
-            case 1: return launch_mma<1>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 1: return launch_mma_hkv<1>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
-            case 2: return launch_mma<2>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 2: return launch_mma_hkv<2>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
-            case 3: return launch_mma<3>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 3: return launch_mma_hkv<3>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
-            case 4: return launch_mma<4>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 4: return launch_mma_hkv<4>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
-            case 5: return launch_mma<5>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 5: return launch_mma_hkv<5>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
-            case 6: return launch_mma<6>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 6: return launch_mma_hkv<6>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
-            case 7: return launch_mma<7>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 7: return launch_mma_hkv<7>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
-            case 8: return launch_mma<8>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
+            case 8: return launch_mma_hkv<8>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
                                        after_own_launch, stream);
         }
         return cudaErrorNotSupported;

@@ -98,8 +98,10 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
 // completion before it first touches partials / sched / row_done, so consecutive launches may even share
 // them (the runtime alternates two sets all the same).
 
-// Token granularity at which the tensor-core kernel splits a context.
+// Token granularity of the tensor-core kernel's copies; a context is split at multiples of
+// attn_mma_tile_tokens(shape) = 16 * 8 / num_kv_heads tokens (one ring stage).
 constexpr int kMmaTileTokens = 16;
+int32_t attn_mma_tile_tokens(const AttnShape& sh);
 
 // Merges the partial results of every row with more than one part into out / lse.  lane: 0 or 1
 // restricts the merge to the rows of that lane, -1 takes all rows.

@@ -410,6 +410,14 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
                     break;
                 }
         }
+        if (ctx->attn_kernel == PS_ATTN_MMA && ctx->tmaps.empty() && cfg->num_kv_heads != 8) {
+            // the row-copy form of the kernel exists for 8 KV heads only
+            if (cfg->attn_kernel != PS_ATTN_AUTO) {
+                ctx->err = "the tensor-core attention kernel needs tensor maps for fewer than 8 KV heads";
+                return create_fail(ctx, PS_ERR_INVALID);
+            }
+            ctx->attn_kernel = PS_ATTN_SIMT;
+        }
         const int64_t max_batch = std::max(cfg->max_batch, 1);
         int64_t max_parts;
         if (cfg->kv_split_tokens > 0) {

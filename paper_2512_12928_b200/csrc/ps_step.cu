@@ -101,7 +101,9 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
             // chunks that the CTAs take dynamically; without contention such a tail only costs (more parts
             // to combine, a last round of chunks that does not fill the machine): 172 against 189 us per
             // 1 GiB launch.  An item is the part of a row that falls into one share or chunk.
-            constexpr int kTile = ps::kMmaTileTokens;
+            const ps::AttnShape shape{ctx->cfg.num_kv_heads, ctx->cfg.num_q_heads, ctx->cfg.head_dim, ctx->cfg.block_size,
+                                      ctx->cfg.num_gpu_blocks};
+            const int kTile = ps::attn_mma_tile_tokens(shape);
             constexpr int64_t kMinTilesPerCta = 8;
             constexpr int64_t kDynMinChunk = 16;
             constexpr int64_t kDynChunksPerCta = 6;

@@ -1,6 +1,6 @@
 """Small, self-contained cases of the three kernels for profilers and quick timing.
 
-    python -m paper_2512_12928_b200.profile_case attn    [--iters N] [--batch B] [--ctx T] [--q-heads H] [--simt | --rows]
+    python -m paper_2512_12928_b200.profile_case attn    [--iters N] [--batch B] [--ctx T] [--q-heads H] [--kv-heads H] [--simt | --rows]
     python -m paper_2512_12928_b200.profile_case gather  [--iters N] [--blocks K]
     python -m paper_2512_12928_b200.profile_case scatter [--iters N] [--blocks K]
 
@@ -29,12 +29,13 @@ def main():
     ap.add_argument("--batch", type=int, default=64)
     ap.add_argument("--ctx", type=int, default=2048)
     ap.add_argument("--q-heads", type=int, default=32)
+    ap.add_argument("--kv-heads", type=int, default=8)
     ap.add_argument("--blocks", type=int, default=2048)
     ap.add_argument("--simt", action="store_true")
     ap.add_argument("--rows", action="store_true", help="tensor-core kernel fed by per-row bulk copies")
     args = ap.parse_args()
 
-    L, Hkv, D, S = 2, 8, 128, 16
+    L, Hkv, D, S = 2, args.kv_heads, 128, 16
     nblk_req = (args.ctx + S - 1) // S
     nb = max(args.batch * nblk_req + 64, 2 * args.blocks + 64)
     sh = wl.KVShape(L, Hkv, args.q_heads, D, S, nb)
@@ -69,7 +70,7 @@ def main():
         ms = e0.elapsed_time(e1) / args.iters
         kv_bytes = args.batch * args.ctx * 2 * Hkv * D * 2
         res.update(us_per_launch=ms * 1e3, kv_bytes_per_launch=kv_bytes, gb_per_s=kv_bytes / ms / 1e6,
-                   batch=args.batch, ctx=args.ctx, q_heads=args.q_heads, kernel="simt" if args.simt else "mma_rows" if args.rows else "auto")
+                   batch=args.batch, ctx=args.ctx, q_heads=args.q_heads, kv_heads=Hkv, kernel="simt" if args.simt else "mma_rows" if args.rows else "auto")
     else:
         direction = 0 if args.case == "gather" else 1
         ids = np.random.default_rng(2).permutation(nb)[: args.blocks].astype(np.int32)

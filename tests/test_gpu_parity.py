@@ -128,6 +128,13 @@ SHAPES = [
     (8, 24, 128, 16, B.PS_ATTN_MMA, 0),
     (8, 56, 128, 32, B.PS_ATTN_MMA, 0),
     (8, 40, 128, 16, B.PS_ATTN_MMA_ROWS, 0),
+    # fewer than 8 KV heads: a stage holds 8 / Hkv sub-tiles, the warps of a head combine their states
+    (4, 16, 128, 16, B.PS_ATTN_MMA, 0),
+    (4, 28, 128, 32, B.PS_ATTN_MMA, 0),
+    (2, 16, 128, 16, B.PS_ATTN_MMA, 0),
+    (2, 2, 128, 48, B.PS_ATTN_MMA, 0),
+    (1, 8, 128, 16, B.PS_ATTN_MMA, 0),
+    (1, 5, 128, 32, B.PS_ATTN_MMA, 0),
     # the same kernel fed by one bulk copy per token row instead of tensor-map boxes
     (8, 32, 128, 16, B.PS_ATTN_MMA_ROWS, 0),
     (8, 64, 128, 32, B.PS_ATTN_MMA_ROWS, 0),
@@ -174,7 +181,8 @@ def test_decode_attn_shapes_ragged_contexts(Hkv, Hq, D, S, kernel, split):
     check_attn(out, want)
 
 
-@pytest.mark.parametrize("Hkv,Hq,D,S", [(4, 8, 64, 16), (8, 32, 128, 16), (8, 64, 128, 32)])
+@pytest.mark.parametrize("Hkv,Hq,D,S", [(4, 8, 64, 16), (8, 32, 128, 16), (8, 64, 128, 32), (4, 16, 128, 16),
+                                        (1, 4, 128, 16)])
 def test_decode_attn_index_coded_values_and_equal_keys(Hkv, Hq, D, S):
     """Outputs of magnitude ~1..100: a read from a wrong block, slot or head cannot hide under 2e-2."""
     L, nb = 1, 64

@@ -18,9 +18,10 @@ if torch.cuda.is_available():
     from gpu_util import Pair, bits_to_dev, check_attn
 
 
-@pytest.mark.parametrize("seed,Hq,S", [(1, 32, 16), (2, 64, 32), (3, 8, 16), (4, 16, 48)])
-def test_random_script_with_data(seed, Hq, S):
-    L, Hkv, D, nb = 2, 8, 128, 160
+@pytest.mark.parametrize("seed,Hkv,Hq,S", [(1, 8, 32, 16), (2, 8, 64, 32), (3, 8, 8, 16), (4, 8, 16, 48), (5, 4, 28, 16),
+                                           (6, 2, 8, 32), (7, 1, 8, 16)])
+def test_random_script_with_data(seed, Hkv, Hq, S):
+    L, D, nb = 2, 128, 160
     sh = wl.KVShape(L, Hkv, Hq, D, S, nb)
     rng = np.random.default_rng([2512, seed])
     K = wl.randn_bf16_bits(rng, (L, nb, S, Hkv, D))
