@@ -29,7 +29,11 @@ What it follows (ProServe, Section 4.3 "Efficient Block Management", and Appendi
 Parity pins (tests/test_oracle_*.py): brute-force loops on tiny inputs, torch's own fp64
 scaled-dot-product attention on contiguous KV, scipy's logsumexp, closed forms (one token, equal
 keys, two-token sigmoid mix), masking and permutation invariants, hand-worked budget schedules,
-round-trip and ownership invariants.  No function here is "parity unpinned".
+round-trip and ownership invariants.  The adaptive budget is pinned by hand-worked cases and an
+exhaustive scan (tests/test_adaptive_budget.py), proactive offloading by element loops and equality
+with on-demand offloading (tests/test_proactive_offload.py), the eviction policy, the partial-copy
+rule and the queue ordering by hand-worked cases and properties (tests/test_eviction_policy.py).
+No function here is "parity unpinned".
 
 Layouts (this build's reading; the paper is silent): per layer a K pool and a V pool,
 uint16[num_blocks][S][Hkv][D] holding bf16 bit patterns; host image of a request
