@@ -390,8 +390,10 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
     }
     const bool attn = want_attn && st.decoded > 0;
     if (attn) {
-        rc = prepare_batch(ctx, reqs, batch, active, gated, (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) == 0,
-                           /*contended=*/!plan.empty() && (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) == 0);
+        // a reload of 32 MiB or more per step slows SMs unevenly enough for a dynamic tail to pay off
+        const bool pipelined = (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) == 0;
+        rc = prepare_batch(ctx, reqs, batch, active, gated, pipelined,
+                           /*contended=*/pipelined && st.h2d_bytes >= (32LL << 20));
         if (rc != PS_OK) return rc;
         st.gated = ctx->meta.n_gated_rows;
     }
