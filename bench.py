@@ -41,6 +41,7 @@ from paper_2512_12928_b200 import workloads as wl
 METRIC = "swap-out/in GB/s vs host-link peak; decode+reload step us vs no-reload step"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1400.0
 
 
 def read_peaks():
@@ -49,6 +50,16 @@ def read_peaks():
         p = json.load(open(path))
         return float(p["hbm_gbs"]), "measured"
     return FALLBACK_HBM_GBS, "fallback"
+
+
+def read_bf16_peak():
+    """Dense bf16 TFLOP/s of a long-running GEMM: measured if the file is there, else the pool's earlier figure."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        if "bf16_tflops_sustained" in p:
+            return float(p["bf16_tflops_sustained"]), "measured"
+    return FALLBACK_BF16_TFLOPS, "fallback"
 
 
 def kernel_code_sha256(path):
@@ -462,7 +473,44 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
                 assert lib.swap_out(r) == 0
             assert lib.sync() == 0
         lib.destroy()
+    res["recompute_arm"] = recompute_arm(B, w, res)
     return res
+
+
+def recompute_arm(B, w, res):
+    """The evaluation's "Recompute" ablation arm (blocks discarded at eviction, the context prefilled again on
+    resume) against the measured reload, for the overlap workload's preempted requests.  The recompute side is
+    NOT measured: it is ps_resume_cost with estimator coefficients set to a lower bound, the prefill's matrix
+    and attention FLOPs at the dense bf16 rate of a long-running library GEMM on this GPU (a real prefill is
+    slower).  hidden and ffn are the public dimensions of the 8B model family whose KV shape the workload has."""
+    sh = w.shape
+    hidden, ffn = 4096, 14336
+    kv_dim = sh.num_kv_heads * sh.head_dim
+    layer_params = hidden * (hidden + 2 * kv_dim) + hidden * hidden + 3 * hidden * ffn
+    tflops, kind = read_bf16_peak()
+    flop_per_us = tflops * 1e6
+    pair_flops = 4 * sh.num_q_heads * sh.head_dim * sh.num_layers       # q.k and p.v, one (query, key) pair
+    model = B.PsLatencyModel(a_p_us=0.5 * pair_flops / flop_per_us, b_p_us=pair_flops / flop_per_us,
+                             c_p_us=2.0 * layer_params * sh.num_layers / flop_per_us, a_d_us=0.0, b_d_us=0.0,
+                             t_c_us=0.0)
+    t_block = res["adaptive_model"]["t_block"]
+    reload_us = recompute_us = 0.0
+    for r in w.victims:
+        rc, a, b = B.ps_resume_cost(model, w.ctx_lens[r], 2048, sh.block_size, t_block)
+        assert rc == 0
+        reload_us += a
+        recompute_us += b
+    row = res["pipelined_adaptive"]
+    exposed_ms = max(0.0, row["step_us_with_reload"] - row["step_us_no_reload"]) * row["steps"] / 1e3
+    return {
+        "tokens": sum(w.ctx_lens[r] for r in w.victims), "chunk_tokens": 2048,
+        "recompute_lower_bound_ms": recompute_us / 1e3, "bf16_tflops": tflops, "bf16_peak_kind": kind,
+        "coefficients_us": {"a_p": model.a_p_us, "b_p": model.b_p_us, "c_p": model.c_p_us},
+        "reload_estimate_ms": reload_us / 1e3, "reload_alone_measured_ms": row["reload_alone_ms"],
+        "reload_exposed_under_decode_measured_ms": exposed_ms,
+        "note": "recompute side is a cost model at 100 % of the GEMM rate, not a measurement; the reload sides are "
+                "the measured transfer alone and the measured step-time inflation under the adaptive budget",
+    }
 
 
 def proactive_offload_leg(torch, B, lib, w, n_off=16):

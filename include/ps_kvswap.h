@@ -405,6 +405,41 @@ int32_t ps_order_queue(int32_t n, const double* exec_us, const double* remain_us
                        const double* waited_us, const ps_sched_params* params, int32_t* order, int32_t* urgent,
                        double* t_budget_us);
 
+/* ---- batch latency estimator and the cost of resuming an evicted request ------------------- */
+
+/* Coefficients of the batch latency estimator (Section 4.1, "Batch Latency Estimator"), microseconds:
+ *   prefill request  T~_p = a_p * l_q^2 + b_p * l_q * l_kv + c_p * l_q
+ *   decode request   T~_d = a_d * l_kv + b_d
+ *   batch            T(B) = sum of T~ over its requests + t_c
+ * l_q = tokens processed in this forward pass, l_kv = KV-cache length before it. */
+typedef struct ps_latency_model {
+    double a_p_us, b_p_us, c_p_us;
+    double a_d_us, b_d_us;
+    double t_c_us;
+} ps_latency_model;
+
+/* Estimated execution time of one batch (the batch equation of Section 4.1).
+ *   l_q, l_kv_prefill : host int32[n_prefill];  l_kv_decode : host int32[n_decode]
+ * An empty batch costs t_c.  Errors: PS_ERR_INVALID (null arrays with a positive count, negative lengths
+ * or coefficients). */
+int32_t ps_estimate_batch(const ps_latency_model* model, int32_t n_prefill, const int32_t* l_q,
+                          const int32_t* l_kv_prefill, int32_t n_decode, const int32_t* l_kv_decode,
+                          double* batch_us);
+
+/* The two ways of bringing an evicted request of n_tokens back, compared by the estimator: the paper spills
+ * evicted blocks to host memory and reloads them (Section 4.3, "Eviction Policy"); its ablation arm
+ * "Recompute" discards them instead, so the context is prefilled again.  The paper prints no cost formula
+ * for that arm; here it is the estimator's own prefill time of the whole context, run in chunks of
+ * chunk_tokens (chunk k processes l_q = min(chunk, n - k*chunk) tokens on l_kv = k*chunk cached ones; every
+ * chunk is a batch of its own and pays t_c; chunk_tokens = 0 means one pass):
+ *   recompute_us = sum over chunks of (T~_p(l_q, l_kv) + t_c)
+ *   reload_us    = ceil(n_tokens / s_blk) * t_block_us        (Section 4.3: T_trans = b_miss * t_block)
+ * The reload figure is the full transfer time; how much of it hides under decode steps is what ps_step's
+ * statistics measure.  Pure arithmetic.  Errors: PS_ERR_INVALID (negative n_tokens or chunk, s_blk <= 0,
+ * negative coefficients or t_block). */
+int32_t ps_resume_cost(const ps_latency_model* model, int32_t n_tokens, int32_t chunk_tokens, int32_t s_blk,
+                       double t_block_us, double* reload_us, double* recompute_us);
+
 /* ---- completion ------------------------------------------------------------------------- */
 
 /* Non-blocking: reaps finished offloads (in issue order), releases host images of finished

@@ -32,7 +32,9 @@ keys, two-token sigmoid mix), masking and permutation invariants, hand-worked bu
 round-trip and ownership invariants.  The adaptive budget is pinned by hand-worked cases and an
 exhaustive scan (tests/test_adaptive_budget.py), proactive offloading by element loops and equality
 with on-demand offloading (tests/test_proactive_offload.py), the eviction policy, the partial-copy
-rule and the queue ordering by hand-worked cases and properties (tests/test_eviction_policy.py).
+rule and the queue ordering by hand-worked cases and properties (tests/test_eviction_policy.py), the
+batch latency estimator and the reload-versus-recompute cost by hand-worked values and the identity that
+chunking leaves a causal prefill's cost unchanged (tests/test_resume_cost.py).
 No function here is "parity unpinned".
 
 Layouts (this build's reading; the paper is silent): per layer a K pool and a V pool,
@@ -520,6 +522,36 @@ def order_queue(exec_t: Sequence[float], remain: Sequence[float], weight: Sequen
     urgent = sorted((i for i in range(n) if cls[i] == 1), key=lambda i: -(weight[i] / exec_t[i]))   # stable
     normal = sorted((i for i in range(n) if cls[i] == 0), key=lambda i: remain[i])
     return starving + urgent + normal, cls, t_budget
+
+
+def estimate_batch(model: Dict[str, float], prefill: Sequence[Tuple[int, int]], decode: Sequence[int]) -> float:
+    """Section 4.1, "Batch Latency Estimator": a prefill request costs a_p l_q^2 + b_p l_q l_kv + c_p l_q, a
+    decode request a_d l_kv + b_d, and a batch the sum over its requests plus the constant overhead t_c.
+    prefill holds (l_q, l_kv) pairs, decode holds l_kv values."""
+    total = 0.0
+    for l_q, l_kv in prefill:
+        total += model["a_p"] * l_q ** 2 + model["b_p"] * l_q * l_kv + model["c_p"] * l_q
+    for l_kv in decode:
+        total += model["a_d"] * l_kv + model["b_d"]
+    return total + model["t_c"]
+
+
+def resume_cost(model: Dict[str, float], n_tokens: int, chunk_tokens: int, s_blk: int, t_block: float):
+    """Cost of bringing an evicted request back, both ways (Section 4.3 "Eviction Policy" spills and restores;
+    the ablation arm "Recompute" of the evaluation discards blocks at eviction).  Reload: every block of the
+    context is missing, T_trans = b_miss * t_block.  Recompute (no formula is printed; the estimator's own
+    prefill model is used): the context is prefilled again in chunks, chunk k being a batch of one prefill
+    request with l_q tokens on the k * chunk tokens already rebuilt.  Returns (reload, recompute)."""
+    b_miss = -(-n_tokens // s_blk)
+    reload_t = b_miss * t_block
+    chunk = chunk_tokens if chunk_tokens > 0 else n_tokens
+    recompute_t = 0.0
+    done = 0
+    while done < n_tokens:
+        l_q = min(chunk, n_tokens - done)
+        recompute_t += estimate_batch(model, [(l_q, done)], [])
+        done += l_q
+    return reload_t, recompute_t
 
 
 def copy_condition(l_comp: int, l_comp_max: int, b_miss: int, b_rem: int, s_blk: int, beta: float) -> bool:

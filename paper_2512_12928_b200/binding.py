@@ -31,7 +31,7 @@ EXPORTS = [
     "ps_swap_in_layer", "ps_missing_blocks", "ps_decode_attn", "ps_step", "ps_poll", "ps_sync",
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
     "ps_decode_attn_static", "ps_copy_budget", "ps_offload_progress", "ps_host_blocks", "ps_host_segment",
-    "ps_select_victims", "ps_copy_condition", "ps_order_queue",
+    "ps_select_victims", "ps_copy_condition", "ps_order_queue", "ps_estimate_batch", "ps_resume_cost",
 ]
 
 
@@ -78,6 +78,11 @@ class PsBudgetModel(C.Structure):
 
 class PsSchedParams(C.Structure):
     _fields_ = [("eta_us", C.c_double), ("gamma", C.c_double), ("t_c_us", C.c_double), ("tau_us", C.c_double)]
+
+
+class PsLatencyModel(C.Structure):
+    _fields_ = [("a_p_us", C.c_double), ("b_p_us", C.c_double), ("c_p_us", C.c_double),
+                ("a_d_us", C.c_double), ("b_d_us", C.c_double), ("t_c_us", C.c_double)]
 
 
 class PsTraceSpan(C.Structure):
@@ -140,6 +145,9 @@ def load() -> C.CDLL:
         "ps_order_queue": (i32, [i32, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_double),
                                  C.POINTER(C.c_double), C.POINTER(PsSchedParams), p32, p32, C.POINTER(C.c_double)]),
         "ps_copy_budget": (i32, [vp, p64, i32, C.POINTER(PsBudgetModel), p64, p64, p32]),
+        "ps_estimate_batch": (i32, [C.POINTER(PsLatencyModel), i32, p32, p32, i32, p32, C.POINTER(C.c_double)]),
+        "ps_resume_cost": (i32, [C.POINTER(PsLatencyModel), i32, i32, i32, C.c_double, C.POINTER(C.c_double),
+                                 C.POINTER(C.c_double)]),
         "ps_decode_attn_static": (i32, [vp, vp, vp, vp, vp, vp, i32, p32, i32, i32, i32, i32, i32, i32, i32, vp, vp,
                                         C.c_char_p, i32]),
     }
@@ -202,6 +210,23 @@ def ps_copy_condition(l_comp: int, l_comp_max: int, b_miss: int, b_rem: int, s_b
     out = C.c_int32()
     rc = load().ps_copy_condition(l_comp, l_comp_max, b_miss, b_rem, s_blk, beta, C.byref(out))
     return rc, bool(out.value)
+
+
+def ps_estimate_batch(model: PsLatencyModel, prefill: Sequence[Tuple[int, int]], decode: Sequence[int]):
+    """Batch latency estimate of Section 4.1: prefill = (l_q, l_kv) pairs, decode = l_kv values.  (status, us)."""
+    i32s = lambda v: (C.c_int32 * max(len(v), 1))(*[int(x) for x in v])
+    out = C.c_double()
+    rc = load().ps_estimate_batch(C.byref(model), len(prefill), i32s([p[0] for p in prefill]),
+                                  i32s([p[1] for p in prefill]), len(decode), i32s(decode), C.byref(out))
+    return rc, out.value
+
+
+def ps_resume_cost(model: PsLatencyModel, n_tokens: int, chunk_tokens: int, s_blk: int, t_block_us: float):
+    """Reload versus recompute of an evicted request: (status, reload_us, recompute_us)."""
+    reload_us, recompute_us = C.c_double(), C.c_double()
+    rc = load().ps_resume_cost(C.byref(model), n_tokens, chunk_tokens, s_blk, t_block_us, C.byref(reload_us),
+                               C.byref(recompute_us))
+    return rc, reload_us.value, recompute_us.value
 
 
 def _i64_array(vals: Sequence[int]):

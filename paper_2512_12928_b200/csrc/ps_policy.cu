@@ -147,4 +147,48 @@ int32_t ps_copy_condition(int32_t l_comp, int32_t l_comp_max, int32_t b_miss, in
     return PS_OK;
 }
 
+static bool latency_model_ok(const ps_latency_model* m) {
+    return m && m->a_p_us >= 0.0 && m->b_p_us >= 0.0 && m->c_p_us >= 0.0 && m->a_d_us >= 0.0 && m->b_d_us >= 0.0 &&
+           m->t_c_us >= 0.0;
+}
+
+static double prefill_us(const ps_latency_model* m, double l_q, double l_kv) {
+    return m->a_p_us * l_q * l_q + m->b_p_us * l_q * l_kv + m->c_p_us * l_q;
+}
+
+int32_t ps_estimate_batch(const ps_latency_model* model, int32_t n_prefill, const int32_t* l_q,
+                          const int32_t* l_kv_prefill, int32_t n_decode, const int32_t* l_kv_decode,
+                          double* batch_us) {
+    if (!latency_model_ok(model) || !batch_us || n_prefill < 0 || n_decode < 0) return PS_ERR_INVALID;
+    if ((n_prefill > 0 && (!l_q || !l_kv_prefill)) || (n_decode > 0 && !l_kv_decode)) return PS_ERR_INVALID;
+    double t = 0.0;
+    for (int32_t i = 0; i < n_prefill; ++i) {
+        if (l_q[i] < 0 || l_kv_prefill[i] < 0) return PS_ERR_INVALID;
+        t += prefill_us(model, (double)l_q[i], (double)l_kv_prefill[i]);
+    }
+    for (int32_t i = 0; i < n_decode; ++i) {
+        if (l_kv_decode[i] < 0) return PS_ERR_INVALID;
+        t += model->a_d_us * (double)l_kv_decode[i] + model->b_d_us;
+    }
+    *batch_us = t + model->t_c_us;
+    return PS_OK;
+}
+
+int32_t ps_resume_cost(const ps_latency_model* model, int32_t n_tokens, int32_t chunk_tokens, int32_t s_blk,
+                       double t_block_us, double* reload_us, double* recompute_us) {
+    if (!latency_model_ok(model) || !reload_us || !recompute_us || n_tokens < 0 || chunk_tokens < 0 || s_blk <= 0 ||
+        !(t_block_us >= 0.0))
+        return PS_ERR_INVALID;
+    const int64_t b_miss = ((int64_t)n_tokens + s_blk - 1) / s_blk;
+    *reload_us = (double)b_miss * t_block_us;
+    const int64_t chunk = chunk_tokens > 0 ? chunk_tokens : n_tokens;
+    double t = 0.0;
+    for (int64_t done = 0; done < n_tokens; done += chunk) {
+        const int64_t l_q = n_tokens - done < chunk ? n_tokens - done : chunk;
+        t += prefill_us(model, (double)l_q, (double)done) + model->t_c_us;
+    }
+    *recompute_us = t;
+    return PS_OK;
+}
+
 }  // extern "C"
