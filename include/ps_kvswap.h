@@ -238,6 +238,16 @@ int32_t ps_swap_in_cancel(ps_ctx* ctx, int64_t req);
  * Errors: PS_ERR_STATE, PS_ERR_INVALID, PS_ERR_CUDA. */
 int32_t ps_swap_in_layer(ps_ctx* ctx, int64_t req, int32_t layer, int32_t blk_lo, int32_t blk_hi);
 
+/* Orders the compute stream after every reload issued so far into `layer` (layer = -1: into every layer):
+ * work the caller enqueues on the compute stream afterwards finds those blocks of that layer complete
+ * (Appendix B: the computation synchronises on a layer chunk's event before it executes that chunk).  For
+ * callers that drive the layer loop themselves and write into reloaded blocks, e.g. a decode forward that
+ * appends the new token's K and V to a request readmitted in this step before that layer's attention: without
+ * the fence the scatter of the block's reloaded bytes could land after the caller's write.  ps_decode_attn
+ * and ps_step order their own launches and need no fence.  A stream-side wait; the host does not block.
+ * Errors: PS_ERR_INVALID (layer out of range), PS_ERR_CUDA. */
+int32_t ps_reload_fence(ps_ctx* ctx, int32_t layer);
+
 /* b_miss of Section 4.3 for one request: blocks on host not yet issued to the device. */
 int32_t ps_missing_blocks(ps_ctx* ctx, int64_t req, int32_t* out);
 

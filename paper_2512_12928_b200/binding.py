@@ -32,6 +32,7 @@ EXPORTS = [
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
     "ps_decode_attn_static", "ps_copy_budget", "ps_offload_progress", "ps_host_blocks", "ps_host_segment",
     "ps_select_victims", "ps_copy_condition", "ps_order_queue", "ps_estimate_batch", "ps_resume_cost",
+    "ps_reload_fence",
 ]
 
 
@@ -127,6 +128,7 @@ def load() -> C.CDLL:
         "ps_swap_in_cancel": (i32, [vp, i64]),
         "ps_swap_in_layer": (i32, [vp, i64, i32, i32, i32]),
         "ps_missing_blocks": (i32, [vp, i64, p32]),
+        "ps_reload_fence": (i32, [vp, i32]),
         "ps_decode_attn": (i32, [vp, i32, vp, vp, vp, p64, i32]),
         "ps_step": (i32, [vp, vp, vp, p64, i32, i64, p32, C.POINTER(PsStepStats)]),
         "ps_poll": (i32, [vp, p32]),
@@ -358,6 +360,9 @@ class KVSwap:
 
     def swap_in_layer(self, req: int, layer: int, blk_lo: int, blk_hi: int) -> int:
         return self.lib.ps_swap_in_layer(self.h, req, layer, blk_lo, blk_hi)
+
+    def reload_fence(self, layer: int = -1) -> int:
+        return self.lib.ps_reload_fence(self.h, layer)
 
     def missing_blocks(self, req: int) -> int:
         out = C.c_int32()

@@ -336,6 +336,16 @@ int32_t ps_swap_in_layer(ps_ctx* ctx, int64_t req, int32_t layer, int32_t blk_lo
     return note_layer_issued(ctx, req, r, layer, blk_hi);
 }
 
+int32_t ps_reload_fence(ps_ctx* ctx, int32_t layer) {
+    if (!ctx) return PS_ERR_INVALID;
+    if (layer < -1 || layer >= ctx->cfg.num_layers) return ctx->fail(PS_ERR_INVALID, "ps_reload_fence: layer out of range");
+    if (ctx->bk) return PS_OK;
+    // the layer's event was last recorded behind its most recent scatter, and the scatter stream runs in order
+    const int lo = layer < 0 ? 0 : layer, hi = layer < 0 ? ctx->cfg.num_layers : layer + 1;
+    for (int l = lo; l < hi; ++l) CK(cudaStreamWaitEvent(ctx->compute, ctx->ev_in[(size_t)l], 0));
+    return PS_OK;
+}
+
 int32_t ps_missing_blocks(ps_ctx* ctx, int64_t req, int32_t* out) {
     if (!ctx || !out) return PS_ERR_INVALID;
     auto it = ctx->reqs.find(req);
