@@ -19,6 +19,7 @@ roofline, the gather / scatter kernels against HBM, the budget sweep of the over
 CPU checker timed on the host cores.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-overlap]
+  python bench.py --workload long_context | churn      (the other full-size workloads, a line of their own)
 """
 from __future__ import annotations
 
@@ -359,17 +360,22 @@ def single_launch_rate(torch, lib, sh, ctx_lens, reqs, q, out, rounds=3):
     return {"us_per_launch": us, "gbs": alg / us / 1e3}
 
 
-def overlap_sweep(torch, B, K, V, peaks_hbm):
-    """Overlap workload: decode batch 128 + 8 preempted requests reloading under 16/64/256 MiB budgets.
+def overlap_sweep(torch, B, K, V, peaks_hbm, w=None, label=None, pipelined_budgets=None, sync_budgets=None):
+    """Overlap workload: decode batch 128 + 8 preempted requests reloading under 16/64/256 MiB budgets (or
+    another workload with victims, e.g. the long-context one).
 
     Contexts carry no per-launch profiling events: under host-link load those events delay the compute
     stream's commands and would be charged to the reload."""
-    w = wl.overlap()
+    w = w or wl.overlap()
     sh = w.shape
     nb = sh.num_gpu_blocks
     host_bytes = sum(sh.blocks_for(w.ctx_lens[r]) for r in w.victims) * sh.block_bytes + (64 << 20)
-    res = {"workload": "overlap: decode batch 128, lognormal contexts (mean 2k, cap 8k), 8 preempted requests"}
+    res = {"workload": label or "overlap: decode batch 128, lognormal contexts (mean 2k, cap 8k), 8 preempted requests"}
     stream = torch.cuda.current_stream()
+    if pipelined_budgets is None:
+        pipelined_budgets = w.budgets + ["adaptive", -1]
+    if sync_budgets is None:
+        sync_budgets = [256 * wl.MiB, -1]
     for mode in ("pipelined", "sync_reload"):
         flags = B.PS_FLAG_SYNC_RELOAD if mode == "sync_reload" else 0
         lib = make_ctx(B, w, K, V, nb, max_batch=len(w.ctx_lens), host_pool_bytes=host_bytes, flags=flags)
@@ -385,7 +391,7 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
         reload_bytes = sum(sh.blocks_for(w.ctx_lens[r]) for r in w.victims) * sh.block_bytes
         # "adaptive": B_copy chosen every step by ps_copy_budget (Section 4.3) from the measured decode time per
         # token and the measured copy time per block (no latency budget: case 2 of the procedure)
-        budgets = w.budgets + ["adaptive", -1] if mode == "pipelined" else [256 * wl.MiB, -1]
+        budgets = pipelined_budgets if mode == "pipelined" else sync_budgets
         model = None
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         if mode == "pipelined":
@@ -400,9 +406,13 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
                      "t_block": sh.block_bytes / (link_gbs * 1e3) * (1.0 + 1.0 / sh.num_layers), "t_budget": 1e12}
             res["adaptive_model"] = dict(model, note="a_d: measured decode step us per KV token; t_block: block bytes / "
                                          "measured H2D rate, plus one layer chunk of pipeline fill")
-        for r in w.victims:
-            assert lib.swap_out(r) == 0, lib.last_error()
-        assert lib.sync() == 0
+        if mode == "pipelined":
+            res.update(offload_rates(torch, B, lib, w, batch, sub_batch(q, len(batch)), sub_batch(out, len(batch)),
+                                     reload_bytes))
+        else:
+            for r in w.victims:
+                assert lib.swap_out(r) == 0, lib.last_error()
+            assert lib.sync() == 0
         for budget in budgets:
             # (1) reload alone, no attention: the transfer time the decode steps have to hide
             for r in w.victims:
@@ -473,8 +483,45 @@ def overlap_sweep(torch, B, K, V, peaks_hbm):
                 assert lib.swap_out(r) == 0
             assert lib.sync() == 0
         lib.destroy()
-    res["recompute_arm"] = recompute_arm(B, w, res)
+    if w.name == "overlap" and "pipelined_adaptive" in res:
+        res["recompute_arm"] = recompute_arm(B, w, res)
     return res
+
+
+def offload_rates(torch, B, lib, w, batch, q_b, out_b, nbytes):
+    """Swap-out of the workload's victims, alone and then under running decode steps; leaves them on the host."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    stream = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    e0.record()
+    for r in w.victims:
+        assert lib.swap_out(r) == 0, lib.last_error()
+    assert lib.sync() == 0
+    e1.record(); e1.synchronize()
+    alone_ms = e0.elapsed_time(e1)
+    for r in w.victims:
+        assert lib.swap_in_begin(r) == 0, lib.last_error()
+    rc, _, _ = lib.step(None, None, [], -1)
+    assert rc == 0 and lib.sync() == 0, lib.last_error()
+    torch.cuda.synchronize()
+    e0.record()
+    for r in w.victims:
+        assert lib.swap_out(r) == 0, lib.last_error()
+    steps = 0
+    while True:
+        rc, _, _ = lib.step(q_b, out_b, batch, 0)
+        assert rc == 0, lib.last_error()
+        stream.synchronize()
+        steps += 1
+        lib.poll()
+        if all(lib.block_table(r)[1] == B.PS_REQ_HOST for r in w.victims):
+            break
+    e1.record(); e1.synchronize()
+    under_ms = e0.elapsed_time(e1)
+    assert lib.sync() == 0
+    return {"offload_alone_gbs": nbytes / alone_ms / 1e6, "offload_under_decode_gbs": nbytes / under_ms / 1e6,
+            "offload_bytes": nbytes, "decode_steps_during_offload": steps,
+            "decode_step_us_during_offload": under_ms / steps * 1e3}
 
 
 def recompute_arm(B, w, res):
@@ -581,6 +628,126 @@ def kernel_rates(torch, B, lib, sh, nb, n_blocks=2048, iters=20):
     res["payload_bytes_per_launch"] = payload
     res["launches_timed"] = iters
     return res
+
+
+def long_context_leg(torch, B, hbm_peak):
+    """70B-shaped KV (80 layers, block 32): decode batch 64 x 4096 tokens, one 32k-token request (10 GiB) offloaded
+    under decode and reloaded layer-pipelined across steps."""
+    w = wl.long_context()
+    sh = w.shape
+    K, V = fill_pools(torch, sh.num_layers, sh.num_gpu_blocks, sh.block_size, sh.num_kv_heads, sh.head_dim, w.seed)
+    torch.cuda.synchronize()
+    res = overlap_sweep(torch, B, K, V, hbm_peak, w=w,
+                        label="long_context: decode batch 64 x 4096 tokens, one 32768-token request of 10 GiB",
+                        pipelined_budgets=[256 * wl.MiB, "adaptive", -1], sync_budgets=[256 * wl.MiB])
+    del K, V
+    return res
+
+
+def churn_leg(torch, B, hbm_peak, steps):
+    """Qwen3-32B-shaped KV (64 layers), 256 live requests of 512-16k tokens on an oversubscribed instance: every
+    step swaps out 2-16 low-priority residents and swaps in 2-16 host-resident requests (a seeded script clipped
+    to capacity), unlimited copy budget, decode over whoever is resident.  Reports the sustained two-way rate
+    over the host link and how much longer a step takes than decoding the same set with no swap."""
+    w = wl.churn(steps=steps)
+    sh = w.shape
+    host_bytes = 12 * wl.GiB
+    init, script = wl.churn_script(w, host_bytes)
+    K, V = fill_pools(torch, sh.num_layers, sh.num_gpu_blocks, sh.block_size, sh.num_kv_heads, sh.head_dim, w.seed)
+    torch.cuda.synchronize()
+    nreq = len(w.ctx_lens)
+    lib = make_ctx(B, w, K, V, sh.num_gpu_blocks, max_batch=nreq, host_pool_bytes=2 * host_bytes)
+    for r in init["host"]:                           # host-resident requests pass through the device first
+        assert lib.kv_alloc(r, w.ctx_lens[r]) == 0, lib.last_error()
+        assert lib.swap_out(r) == 0, lib.last_error()
+        assert lib.sync() == 0
+    for r in init["resident"]:
+        assert lib.kv_alloc(r, w.ctx_lens[r]) == 0, lib.last_error()
+    known = sorted(init["host"] + init["resident"])
+    g = torch.Generator(device="cuda")
+    g.manual_seed(w.seed)
+    q = torch.randn((sh.num_layers, nreq, sh.num_q_heads, sh.head_dim), generator=g, device="cuda",
+                    dtype=torch.float32).to(torch.bfloat16)
+    out = torch.zeros_like(q)
+    duplex_gbs = B.ps_link_probe(256 << 20, 2, 5)
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    q_l, out_l = sub_batch(q, len(known)), sub_batch(out, len(known))
+    for _ in range(3):
+        rc, mask, _ = lib.step(q_l, out_l, known, 0)
+        assert rc == 0, lib.last_error()
+    torch.cuda.synchronize()
+    bytes_out = bytes_in = n_out = n_in = decoded = 0
+    step_ms = []
+    bound_ms = 0.0                                   # per step the busier direction at half the two-way rate
+    e0.record()
+    for stp in script:
+        assert lib.sync() == 0                       # the previous step's swaps have completed
+        o0, i0 = bytes_out, bytes_in
+        for r in stp["out"]:
+            if lib.swap_out(r) == 0:
+                bytes_out += sh.blocks_for(w.ctx_lens[r]) * sh.block_bytes
+                n_out += 1
+        for r in stp["inn"]:
+            if lib.swap_in_begin(r) == 0:
+                bytes_in += sh.blocks_for(w.ctx_lens[r]) * sh.block_bytes
+                n_in += 1
+        bound_ms += max(bytes_out - o0, bytes_in - i0) / (duplex_gbs / 2) / 1e6
+        s0.record()
+        rc, mask, st = lib.step(q_l, out_l, known, -1)
+        assert rc == 0, lib.last_error()
+        s1.record()
+        stream.synchronize()
+        step_ms.append(s0.elapsed_time(s1))
+        decoded += sum(mask)
+    assert lib.sync() == 0
+    e1.record(); e1.synchronize()
+    total_ms = e0.elapsed_time(e1)
+    resident = [r for r in known if lib.block_table(r)[1] == B.PS_REQ_RESIDENT]
+    q_r, out_r = sub_batch(q, len(resident)), sub_batch(out, len(resident))
+    rf = decode_roofline(torch, lib, sh, w.ctx_lens, resident, q_r, out_r, steps=3)
+    lib.destroy()
+    del K, V
+    return {
+        "workload": f"churn: 64 layers, {nreq} live requests (512-16k tokens), {len(known)} of them holding KV, "
+                    f"{steps} scripted steps, unlimited copy budget, device pool 96 GiB, host images 12 GiB planned",
+        "steps": steps, "swap_outs": n_out, "swap_ins": n_in, "bytes_out": bytes_out, "bytes_in": bytes_in,
+        "two_way_gbs": (bytes_out + bytes_in) / total_ms / 1e6, "link_two_way_peak_gbs": duplex_gbs,
+        "frac_of_two_way_peak": (bytes_out + bytes_in) / total_ms / 1e6 / duplex_gbs,
+        "schedule_bound_ms": bound_ms, "total_ms": total_ms, "frac_of_schedule_bound": bound_ms / total_ms,
+        "schedule_bound": "the swaps of a step complete in that step, so a step cannot end before its busier "
+                          "direction has crossed the link at half the measured two-way rate",
+        "step_ms_mean_with_swaps": total_ms / steps, "compute_stream_step_ms_mean": float(np.mean(step_ms)),
+        "decode_step_ms_no_swap": rf["step_us"] / 1e3, "requests_decoding_at_end": len(resident),
+        "decoded_request_steps": decoded, "attn_gbs": rf["gbs"], "attn_frac_of_hbm": rf["gbs"] / hbm_peak,
+    }
+
+
+def run_extra(args):
+    """The other workloads of the evaluation, one JSON line each (single GPU; not the headline line)."""
+    import torch
+
+    from paper_2512_12928_b200 import binding as B
+    from paper_2512_12928_b200 import build as ps_build
+    torch.cuda.set_device(0)
+    ps_build.build()
+    B.load()
+    hbm_peak, peak_kind = read_peaks()
+    sampler = ClockSampler(0)
+    sampler.start()
+    if args.workload == "long_context":
+        detail = long_context_leg(torch, B, hbm_peak)
+        value = detail["pipelined_adaptive"]["reload_under_decode_gbs"]
+        metric = "reload GB/s under decode (adaptive copy budget); hidden fraction in detail"
+    else:
+        detail = churn_leg(torch, B, hbm_peak, args.churn_steps)
+        value = detail["two_way_gbs"]
+        metric = "sustained swap-out + swap-in GB/s over the host link under decode"
+    clocks = sampler.stop()
+    print(json.dumps({"metric": metric, "value": value, "unit": UNIT, "n_gpus": 1, "higher_is_better": True,
+                      "dtype": "bf16", "data": "synthetic", "config": {"workload": args.workload},
+                      "peak_kind": peak_kind, "clocks": clocks, "detail": detail}))
 
 
 def run_gpu(args):
@@ -761,9 +928,14 @@ def main():
     ap.add_argument("--budget-mib", type=int, default=-1, help="copy budget per step in MiB for phase B (-1 = unlimited)")
     ap.add_argument("--no-overlap", action="store_true", help="skip the overlap budget sweep")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    ap.add_argument("--workload", default="llama8b_swap", choices=["llama8b_swap", "long_context", "churn"],
+                    help="llama8b_swap is the headline line; the others print a line of their own (one GPU)")
+    ap.add_argument("--churn-steps", type=int, default=100)
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload != "llama8b_swap":
+        run_extra(args)
     else:
         run_gpu(args)
 
