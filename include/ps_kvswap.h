@@ -202,6 +202,17 @@ int32_t ps_swap_out(ps_ctx* ctx, int64_t req);
  * Errors: PS_ERR_STATE, PS_ERR_INVALID, PS_ERR_HOST_NOMEM, PS_ERR_CUDA. */
 int32_t ps_offload_progress(ps_ctx* ctx, int64_t req, int32_t n_off, int32_t* issued_blocks);
 
+/* ps_offload_progress for a whole batch, e.g. once after every decode step: request reqs[i] with its own
+ * threshold n_off[i] (the paper's n_off^r: smaller for lower-priority requests, which are more likely to be
+ * preempted).  Entries that are unknown or not RESIDENT are skipped.  *issued_blocks (may be NULL) = blocks
+ * issued over the batch.  The entries are taken in order and the call stops at the first failing one
+ * (typically PS_ERR_HOST_NOMEM): copies issued for earlier entries stay issued, the failing entry and the
+ * later ones are untouched.
+ * Errors: PS_ERR_INVALID (null arrays with batch > 0, a non-positive threshold), and those of
+ * ps_offload_progress. */
+int32_t ps_offload_sweep(ps_ctx* ctx, const int64_t* reqs, const int32_t* n_off, int32_t batch,
+                         int64_t* issued_blocks);
+
 /* b_host of Section 4.3 for one request: blocks whose offload has been issued, and blocks whose copy has
  * been seen complete (as of the last ps_poll / ps_step / ps_sync).  Either pointer may be NULL. */
 int32_t ps_host_blocks(ps_ctx* ctx, int64_t req, int32_t* issued, int32_t* on_host);

@@ -206,6 +206,23 @@ class PsOracle:
         rc = self._offload_segment(r, lo, lo + groups * n_off)
         return rc, (groups * n_off if rc == OK else 0)
 
+    def offload_sweep(self, reqs: Sequence[int], n_off: Sequence[int]):
+        """The same trigger over a batch, request r with its own threshold n_off^r ("Asynchronous Offloading":
+        lower-priority requests get smaller thresholds).  Requests that are not resident are skipped; stops at
+        the first failure.  Returns (status, blocks copied)."""
+        if any(n <= 0 for n in n_off):
+            return ERR_INVALID, 0
+        total = 0
+        for req, n in zip(reqs, n_off):
+            r = self.reqs.get(req)
+            if r is None or r.state != ST_RESIDENT:
+                continue
+            rc, issued = self.offload_progress(req, n)
+            total += issued
+            if rc != OK:
+                return rc, total
+        return OK, total
+
     def host_blocks(self, req: int) -> int:
         """b_host of Section 4.3: blocks of the request that have a copy on host."""
         return self._host_issued(self.reqs[req])

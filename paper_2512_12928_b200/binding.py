@@ -32,7 +32,7 @@ EXPORTS = [
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
     "ps_decode_attn_static", "ps_copy_budget", "ps_offload_progress", "ps_host_blocks", "ps_host_segment",
     "ps_select_victims", "ps_copy_condition", "ps_order_queue", "ps_estimate_batch", "ps_resume_cost",
-    "ps_reload_fence",
+    "ps_reload_fence", "ps_offload_sweep",
 ]
 
 
@@ -141,6 +141,7 @@ def load() -> C.CDLL:
         "ps_trace_read": (i32, [vp, C.POINTER(PsTraceSpan), i32, p32]),
         "ps_offload_progress": (i32, [vp, i64, i32, p32]),
         "ps_host_blocks": (i32, [vp, i64, p32, p32]),
+        "ps_offload_sweep": (i32, [vp, p64, p32, i32, p64]),
         "ps_host_segment": (i32, [vp, i64, i32, C.POINTER(vp), p64, p32, p32, p32]),
         "ps_select_victims": (i32, [vp, p64, i32, C.POINTER(C.c_double), C.c_double, C.c_double, i32, p64, i32, p32, p32]),
         "ps_copy_condition": (i32, [i32, i32, i32, i32, i32, C.c_double, p32]),
@@ -334,6 +335,13 @@ class KVSwap:
         n = C.c_int32()
         rc = self.lib.ps_offload_progress(self.h, req, n_off, C.byref(n))
         return rc, n.value
+
+    def offload_sweep(self, reqs: Sequence[int], n_off: Sequence[int]):
+        """Proactive offload over a batch with per-request thresholds: (status, blocks issued)."""
+        total = C.c_int64()
+        thr = (C.c_int32 * max(len(n_off), 1))(*[int(v) for v in n_off])
+        rc = self.lib.ps_offload_sweep(self.h, _i64_array(reqs), thr, len(reqs), C.byref(total))
+        return rc, total.value
 
     def host_blocks(self, req: int) -> Tuple[int, int]:
         a, b = C.c_int32(), C.c_int32()

@@ -226,6 +226,26 @@ int32_t ps_offload_progress(ps_ctx* ctx, int64_t req, int32_t n_off, int32_t* is
     return PS_OK;
 }
 
+int32_t ps_offload_sweep(ps_ctx* ctx, const int64_t* reqs, const int32_t* n_off, int32_t batch,
+                         int64_t* issued_blocks) {
+    if (!ctx) return PS_ERR_INVALID;
+    if (issued_blocks) *issued_blocks = 0;
+    if (batch < 0 || (batch > 0 && (!reqs || !n_off))) return ctx->fail(PS_ERR_INVALID, "ps_offload_sweep: bad argument");
+    for (int32_t i = 0; i < batch; ++i)
+        if (n_off[i] <= 0) return ctx->fail(PS_ERR_INVALID, "ps_offload_sweep: thresholds must be positive");
+    int64_t total = 0;
+    for (int32_t i = 0; i < batch; ++i) {
+        auto it = ctx->reqs.find(reqs[i]);
+        if (it == ctx->reqs.end() || it->second.state != PS_REQ_RESIDENT) continue;
+        int32_t issued = 0;
+        int32_t rc = ps_offload_progress(ctx, reqs[i], n_off[i], &issued);
+        total += issued;
+        if (issued_blocks) *issued_blocks = total;
+        if (rc != PS_OK) return rc;
+    }
+    return PS_OK;
+}
+
 int32_t ps_host_blocks(ps_ctx* ctx, int64_t req, int32_t* issued, int32_t* on_host) {
     if (!ctx) return PS_ERR_INVALID;
     auto it = ctx->reqs.find(req);

@@ -4,7 +4,8 @@ Two loops.  (1) A caller-driven layer loop (Appendix B): reload chunks issued pe
 attention the forward pass appends the new token's K and V to every request, the readmitted ones included,
 which is what ps_reload_fence is for.  (2) The paper's closed loop (Sections 4.2-4.3): the queue is ordered,
 victims are taken from its tail when the pool is short, requests are readmitted from its head, the copy
-budget is chosen per step, ps_step reloads and decodes, decoding appends tokens.  In both, the CPU checker
+budget is chosen per step, ps_step reloads and decodes, decoding appends tokens, filled blocks are offloaded
+ahead of eviction.  In both, the CPU checker
 replays the same calls; block tables, pool bytes and attention outputs must agree.
 """
 import numpy as np
@@ -148,7 +149,7 @@ def test_closed_loop_with_real_bytes():
     next_id = 100
     cases = set()
     last_run = {}
-    decoded_total = evicted_total = reloaded_total = finished_total = 0
+    decoded_total = evicted_total = reloaded_total = finished_total = ahead_total = 0
     for rnd in range(36):
         now += 60.0
         queue = [r for r in ids if r in orc.reqs or r <= rnd or r >= 100]
@@ -174,6 +175,7 @@ def test_closed_loop_with_real_bytes():
                 assert (victims, freed) == want_v
                 victims = [v for v in victims if sorted_q.index(v) > sorted_q.index(r)]
                 for v in victims:
+                    ahead_total += len(lib.host_segments(v)) > 0      # proactive copies: only the tail is left to move
                     assert p.both("swap_out", v) == B.PS_OK
                     evicted_total += 1
                 p.sync()
@@ -217,9 +219,12 @@ def test_closed_loop_with_real_bytes():
                 weight[next_id] = float(rng.choice([1.0, 2.0]))
                 deadline[next_id] = now + float(rng.uniform(200, 3000))
                 next_id += 1
-        p.assert_tables_equal([r for r in sorted_q if r in orc.reqs])
+        # proactive offloading after the step: low-weight requests, the likelier victims, copy more often
+        holders = [r for r in sorted_q if r in orc.reqs]
+        assert p.both("offload_sweep", holders, [2 if weight[r] == 1.0 else 4 for r in holders])[0] == B.PS_OK
+        p.assert_tables_equal(holders)
         orc.check_invariants()
     p.sync()
     p.assert_pools_equal()
-    assert decoded_total > 100 and evicted_total > 5 and reloaded_total > 5 and finished_total > 5
+    assert decoded_total > 100 and evicted_total > 5 and reloaded_total > 5 and finished_total > 5 and ahead_total > 3
     assert {21, 22} <= cases

@@ -147,6 +147,43 @@ def test_library_host_logic_matches_checker_on_a_random_script():
     orc.check_invariants()
 
 
+def test_batch_sweep_with_per_request_thresholds_equals_the_single_calls():
+    """A sweep with thresholds n_off^r is the per-request trigger applied in order; requests that are not
+    resident are skipped; a host pool that fills up stops the sweep where it stands."""
+    sh = wl.KVShape(2, 2, 4, 64, 8, 128)
+    order = np.random.default_rng(5).permutation(sh.num_gpu_blocks)
+    mk = lambda host: B.KVSwap(num_layers=2, num_kv_heads=2, num_q_heads=4, head_dim=64, block_size=8, num_gpu_blocks=128,
+                               max_blocks_per_req=64, host_pool_bytes=host, initial_free_order=order,
+                               flags=B.PS_FLAG_BOOKKEEPING_ONLY)
+    lib, ref = mk(1 << 40), mk(1 << 40)
+    orc = po.PsOracle(2, 2, 4, 64, 8, 128, order)
+    tokens = {1: 100, 2: 37, 3: 8, 4: 64, 5: 90}
+    for x in (lib, ref, orc):
+        for r, n in tokens.items():
+            assert x.kv_alloc(r, n) == 0
+        assert x.swap_out(4) == 0                                  # request 4 is not resident during the sweep
+    reqs, thr = [1, 2, 99, 3, 4, 5], [5, 2, 1, 1, 1, 3]              # 99 is unknown
+    # hand count: 100 tokens = 12 full blocks -> 2 groups of 5 = 10; 37 -> 4 full -> 4; 8 -> 1 full -> 1; 90 -> 11 -> 9
+    assert orc.offload_sweep(reqs, thr) == (po.OK, 24)
+    assert lib.offload_sweep(reqs, thr) == (B.PS_OK, 24)
+    singles = sum(ref.offload_progress(r, n)[1] for r, n in zip(reqs, thr) if r in (1, 2, 3, 5))
+    assert singles == 24
+    for r in (1, 2, 3, 5):
+        assert lib.host_blocks(r)[0] == ref.host_blocks(r)[0] == orc.host_blocks(r)
+        assert lib.host_segments(r)[0][2:] == ref.host_segments(r)[0][2:]
+    assert lib.offload_sweep(reqs, thr) == (B.PS_OK, 0) and orc.offload_sweep(reqs, thr) == (po.OK, 0)   # nothing new
+    for x in (lib, orc):                                           # decode goes on: more blocks fill up
+        assert x.kv_alloc(2, 37 + 16) == 0
+    assert lib.offload_sweep([2], [2]) == (B.PS_OK, 2) and orc.offload_sweep([2], [2]) == (po.OK, 2)
+    assert lib.offload_sweep([1], [0])[0] == B.PS_ERR_INVALID and orc.offload_sweep([1], [0])[0] == po.ERR_INVALID
+    # a host pool of 12 blocks: the first request's 10 blocks fit, the second one's 4 do not
+    small = mk(12 * sh.block_bytes)
+    for r, n in tokens.items():
+        assert small.kv_alloc(r, n) == 0
+    assert small.offload_sweep([1, 2, 3], [5, 2, 1]) == (B.PS_ERR_HOST_NOMEM, 10)
+    assert small.host_blocks(1)[0] == 10 and small.host_blocks(2)[0] == 0 and small.host_blocks(3)[0] == 0
+
+
 # ------------------------------------------------------------------------------------------------- GPU
 
 @pytest.mark.gpu
