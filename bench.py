@@ -19,7 +19,7 @@ roofline, the gather / scatter kernels against HBM, the budget sweep of the over
 CPU checker timed on the host cores.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-overlap]
-  python bench.py --workload long_context | churn      (the other full-size workloads, a line of their own)
+  python bench.py --workload long_context | churn | decode_shapes   (other workloads, a line of their own)
 """
 from __future__ import annotations
 
@@ -724,6 +724,40 @@ def churn_leg(torch, B, hbm_peak, steps):
     }
 
 
+def decode_shapes_leg(torch, B, hbm_peak):
+    """Decode attention alone for the KV shapes of the paper's model families under tensor parallelism: 8 / 4 / 2 / 1
+    KV heads per GPU (8B-like 32 layers G = 4; Qwen2-7B-like 28 layers G = 7 and its 2- and 4-way shards).
+    Batch 128, lognormal contexts (mean 2048, cap 8192); in-step rate (ps_step) and one launch per call."""
+    rows = []
+    nb = 24576
+    for L, Hkv, Hq in [(32, 8, 32), (28, 4, 28), (28, 2, 14), (28, 1, 7)]:
+        sh = wl.KVShape(L, Hkv, Hq, 128, 16, nb)
+        rng = np.random.default_rng(wl.SEED_BASE + 9)
+        ctx = wl.lognormal_ctx(rng, 128, 2048.0, 0.8, 8192)
+        w = wl.Workload("decode_shapes", 9, sh, wl.SEED_BASE + 9, ctx, [], rng.permutation(nb).astype(np.int32),
+                        decode_batch=128)
+        K, V = fill_pools(torch, L, nb, sh.block_size, Hkv, sh.head_dim, w.seed)
+        lib = make_ctx(B, w, K, V, nb, max_batch=128, host_pool_bytes=64 << 20)
+        for r, n in wl.build_order_round_robin(w):
+            assert lib.kv_alloc(r, n) == 0, lib.last_error()
+        reqs = list(range(128))
+        g = torch.Generator(device="cuda")
+        g.manual_seed(w.seed)
+        q = torch.randn((L, 128, Hq, sh.head_dim), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        out = torch.zeros_like(q)
+        time_decode_steps(torch, lib, reqs, q, out, 3)
+        rf = decode_roofline(torch, lib, sh, ctx, reqs, q, out, steps=5)
+        sg = single_launch_rate(torch, lib, sh, ctx, reqs, q, out)
+        rows.append({"layers": L, "kv_heads": Hkv, "q_heads": Hq, "bytes_per_launch": rf["algorithmic_bytes_per_launch"],
+                     "in_step_gbs": rf["gbs"], "in_step_frac_of_hbm": rf["gbs"] / hbm_peak,
+                     "in_step_us_per_launch": rf["us_per_layer"], "single_launch_gbs": sg["gbs"],
+                     "single_launch_us": sg["us_per_launch"]})
+        lib.destroy()
+        del K, V, lib, q, out
+        torch.cuda.empty_cache()
+    return {"workload": "decode attention alone, batch 128, lognormal contexts, four KV shapes", "shapes": rows}
+
+
 def run_extra(args):
     """The other workloads of the evaluation, one JSON line each (single GPU; not the headline line)."""
     import torch
@@ -740,6 +774,10 @@ def run_extra(args):
         detail = long_context_leg(torch, B, hbm_peak)
         value = detail["pipelined_adaptive"]["reload_under_decode_gbs"]
         metric = "reload GB/s under decode (adaptive copy budget); hidden fraction in detail"
+    elif args.workload == "decode_shapes":
+        detail = decode_shapes_leg(torch, B, hbm_peak)
+        value = detail["shapes"][1]["in_step_gbs"]
+        metric = "decode attention GB/s of KV read, 28 layers x 4 KV heads x 28 query heads (in ps_step)"
     else:
         detail = churn_leg(torch, B, hbm_peak, args.churn_steps)
         value = detail["two_way_gbs"]
@@ -928,7 +966,7 @@ def main():
     ap.add_argument("--budget-mib", type=int, default=-1, help="copy budget per step in MiB for phase B (-1 = unlimited)")
     ap.add_argument("--no-overlap", action="store_true", help="skip the overlap budget sweep")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
-    ap.add_argument("--workload", default="llama8b_swap", choices=["llama8b_swap", "long_context", "churn"],
+    ap.add_argument("--workload", default="llama8b_swap", choices=["llama8b_swap", "long_context", "churn", "decode_shapes"],
                     help="llama8b_swap is the headline line; the others print a line of their own (one GPU)")
     ap.add_argument("--churn-steps", type=int, default=100)
     args = ap.parse_args()
