@@ -18,8 +18,9 @@ What it follows (ProServe, Section 4.3 "Efficient Block Management", and Appendi
 * A per-step host-to-device copy budget B_copy (in blocks) is consumed in queue order at request
   granularity: all missing blocks b_miss of a request if they fit, otherwise a partial copy with
   the residual budget ("Put it Together"; Alg. 1: GetCopyBudget, ConsumeCopyBudget).  -> `step_plan`, `step`.
-  The beta admission test of that paragraph depends on the scheduler's computable-token count and
-  is not modelled: a partial copy is always allowed and a request decodes only once complete.
+  The beta admission test of that paragraph (SatisfyCopyCondition) depends on the scheduler's
+  computable-token count: `step_plan` applies it to the requests for which the caller supplies that
+  count and always allows the partial copy for the others; a request decodes only once complete.
 * The number of blocks to reload per step, B_copy, follows the three-case procedure of "Adaptive
   Copy-Budget Control" with the decode latency model of Section 4.1.  -> `copy_budget`.
 * The computation the reload overlaps with is the decode forward; its KV-consuming part is
@@ -325,12 +326,17 @@ class PsOracle:
             return 0
         return len(r.table) - min(r.layer_done)
 
-    def step_plan(self, copy_budget_bytes: int) -> List[Tuple[int, int, int]]:
+    def step_plan(self, copy_budget_bytes: int, rule: Optional[Dict[int, Tuple[int, int]]] = None,
+                  beta: Optional[float] = None) -> List[Tuple[int, int, int]]:
         """Consume the budget over the reload queue in order; returns (req, blk_lo, blk_hi) per request.
 
         Budget in blocks = floor(bytes / block_bytes) with a block spanning all layers; negative
-        means unlimited.  A request whose missing blocks fit is copied whole, otherwise it gets
-        what is left and the round ends.
+        means unlimited.  A request whose missing blocks fit is copied whole.  The first one that does
+        not fit gets what is left -- always, when `rule` does not list it; when rule[req] =
+        (l_comp, l_comp_max) is given, only if the partial-copy test of "Put it Together" passes
+        (`copy_condition` with the residual budget), otherwise the request is skipped this round and
+        the scheduler proceeds to the next request with the budget unchanged (Alg. 1: `continue`
+        after SatisfyCopyCondition fails).
         """
         left = None if copy_budget_bytes < 0 else copy_budget_bytes // self.block_bytes
         plan = []
@@ -340,24 +346,29 @@ class PsOracle:
             miss = len(r.table) - lo
             if miss == 0:
                 continue
-            take = miss if left is None else min(miss, left)
-            if take == 0:
+            if left is not None and left == 0:
                 break
+            take = miss
+            if left is not None and miss > left:
+                if rule is not None and req in rule:
+                    l_comp, l_comp_max = rule[req]
+                    if not copy_condition(l_comp, l_comp_max, miss, left, self.S, beta):
+                        continue
+                take = left
             plan.append((req, lo, lo + take))
             if left is not None:
                 left -= take
-                if left == 0:
-                    break
         return plan
 
     def step(self, copy_budget_bytes: int, reqs: Optional[Sequence[int]] = None,
-             q_bits: Optional[np.ndarray] = None):
+             q_bits: Optional[np.ndarray] = None, rule: Optional[Dict[int, Tuple[int, int]]] = None,
+             beta: Optional[float] = None):
         """One engine step: reload under the budget (every layer), then decode the complete requests.
 
         Returns (plan, decoded mask, out) with out float64 [L][B][Hq][D] (rows of requests that
         did not decode are NaN) or None when no queries were given.
         """
-        plan = self.step_plan(copy_budget_bytes)
+        plan = self.step_plan(copy_budget_bytes, rule, beta)
         for req, lo, hi in plan:
             for l in range(self.L):
                 rc = self.swap_in_layer(req, l, lo, hi)

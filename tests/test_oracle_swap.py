@@ -184,6 +184,73 @@ def test_budget_schedule_golden(repo_root):
         o.check_invariants()
 
 
+def test_swap_in_begin_of_a_request_without_blocks_is_resident_at_once():
+    """Section 4.3 "Pipelined Reloading": a readmitted request's KV must be restored before computation can
+    proceed; a request with no tokens has nothing to restore, so it is RESIDENT as soon as it is readmitted:
+    it never sits in the reload queue (where no budget could ever complete it) and holds no host bytes."""
+    o, _ = small_oracle(with_data=True, host_pool_bytes=1 << 20)
+    assert o.kv_alloc(0, 0) == po.OK and o.kv_alloc(1, 9) == po.OK
+    assert o.swap_out(0) == po.OK and o.swap_out(1) == po.OK
+    o.reap()
+    assert o.block_table(0) == ([], po.ST_HOST)
+    used_by_1 = o.host_used
+    assert used_by_1 == 3 * o.block_bytes                 # the empty image of request 0 holds nothing
+    free_before = o.num_free_blocks()
+    assert o.swap_in_begin(1) == po.OK and o.swap_in_begin(0) == po.OK
+    assert o.block_table(0) == ([], po.ST_RESIDENT)
+    assert list(o.in_fifo) == [1]                          # FIFO unchanged by the empty request
+    assert o.host_used == used_by_1 and o.num_free_blocks() == free_before - 3
+    assert o.missing_blocks(0) == 0
+    assert o.step_plan(-1) == [(1, 0, 3)]
+    assert o.swap_in_begin(0) == po.ERR_STATE              # already resident
+    assert o.kv_alloc(0, 5) == po.OK                       # and it can grow like any resident request
+    o.step(-1)
+    assert o.host_used == 0
+    o.check_invariants()
+
+
+def test_ruled_budget_schedule_golden(repo_root):
+    """The partial-copy admission test while the budget is consumed: hand-worked schedules."""
+    g = json.load(open(os.path.join(repo_root, "tests", "golden", "budget_schedule.json")))
+    for case in g["ruled_cases"]:
+        o = po.PsOracle(**g["shape"])
+        for req, n in g["queue_tokens"]:
+            assert o.kv_alloc(req, n) == po.OK
+        for req, _ in g["queue_tokens"]:
+            assert o.swap_out(req) == po.OK
+        o.reap()
+        for req, _ in g["queue_tokens"]:
+            assert o.swap_in_begin(req) == po.OK
+        rule = {int(k): tuple(v) for k, v in case["rule"].items()}
+        for want in case["steps"]:
+            plan, _, _ = o.step(case["budget_bytes"], rule=rule, beta=case["beta"])
+            assert [list(p) for p in plan] == want, (case["_derivation"], plan, want)
+        o.check_invariants()
+
+
+def test_ruled_plan_equals_plain_plan_when_every_partial_copy_is_allowed():
+    """With l_comp at the round's limit for every request the rule never bites: same plans as without it."""
+    rng = np.random.default_rng(5)
+    for trial in range(20):
+        a, _ = small_oracle(with_data=False, nb=64)
+        b, _ = small_oracle(with_data=False, nb=64)
+        ids = list(range(5))
+        for r in ids:
+            n = int(rng.integers(1, 40))
+            for o in (a, b):
+                assert o.kv_alloc(r, n) == po.OK
+        for o in (a, b):
+            for r in ids:
+                assert o.swap_out(r) == po.OK
+            o.reap()
+            for r in ids:
+                assert o.swap_in_begin(r) == po.OK
+        budget = int(rng.integers(1, 6)) * a.block_bytes
+        rule = {r: (7, 7) for r in ids}
+        for _ in range(12):
+            assert a.step(budget)[0] == b.step(budget, rule=rule, beta=2.0)[0]
+
+
 def test_tiny_workload_script_round_trip():
     w = wl.tiny()
     K, V = wl.make_pools_numpy(w)
