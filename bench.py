@@ -610,7 +610,7 @@ def kernel_rates(torch, B, lib, sh, nb, n_blocks=2048, iters=20):
     payload = n_blocks * sh.layer_block_bytes
 
     def launch(i, direction):
-        rc = lib.lib.ps_copy_blocks(lib.h, i % sh.num_layers, ids, n_blocks, C.c_void_p(stage.data_ptr()), direction)
+        rc = lib.lib.ps_copy_blocks(lib.h, i % sh.num_layers, 1, ids, n_blocks, C.c_void_p(stage.data_ptr()), direction)
         assert rc == 0, lib.last_error()
 
     for name, direction in (("gather", 0), ("scatter", 1)):   # the scatter overwrites pool blocks: run last

@@ -23,7 +23,8 @@
  *     ps_create was called; "host pointer" = ordinary process memory unless it says pinned.
  *   - One caller thread per context.  All GPU work is asynchronous with respect to the host
  *     unless a function says it waits.  Asynchronous CUDA failures surface as PS_ERR_CUDA (and
- *     kernel-side id checks as PS_ERR_BOUNDS) from the next ps_poll / ps_sync / ps_step.
+ *     kernel-side id checks as PS_ERR_BOUNDS, a kernel-side wait that ran out as PS_ERR_TIMEOUT) from the
+ *     next ps_poll / ps_sync / ps_step.
  *   - Layouts.  bf16 everywhere.  Per layer there is one K pool and one V pool, each
  *     [num_gpu_blocks][block_size][num_kv_heads][head_dim]; the "slab" of a block is its
  *     block_size*num_kv_heads*head_dim contiguous elements in one pool.  The host image of a
@@ -51,7 +52,8 @@ enum ps_status {
     PS_ERR_HOST_NOMEM = -3,  /* host pool cannot hold the image */
     PS_ERR_STATE = -4,       /* request is in the wrong state for this call */
     PS_ERR_BUSY = -5,        /* a transfer of this request is still in flight */
-    PS_ERR_TIMEOUT = -6,     /* bounded host wait ran out */
+    PS_ERR_TIMEOUT = -6,     /* a bounded wait ran out: ps_sync's on the host, or one inside the attention
+                                kernel (then the launches in flight produced undefined outputs) */
     PS_ERR_CUDA = -7,        /* a CUDA call failed; see ps_last_error */
     PS_ERR_BOUNDS = -8       /* a kernel met a block id outside the pool and skipped it */
 };
@@ -99,7 +101,11 @@ typedef struct ps_config {
     int32_t flags;               /* OR of ps_flags */
     int32_t attn_kernel;         /* ps_attn_kernel */
     int32_t kv_split_tokens;     /* tokens per split-KV work item; 0 = chosen per batch */
-    int32_t reserved0;
+    int32_t layer_chunk_bytes;   /* ps_step reloads in layer chunks (Appendix B: one completion event per layer
+                                    chunk): consecutive layers share one host copy, one scatter launch and one
+                                    event until the chunk carries this many bytes, because a single layer's share
+                                    of a small copy budget is too small for the copy engine to reach link rate.
+                                    0 = 2 MiB; negative = always one layer per chunk */
     int64_t host_pool_bytes;     /* capacity for host images */
     int64_t staging_bytes;       /* device staging per direction (split into 4 slots); 0 = 256 MiB */
     const int32_t* initial_free_order; /* host pointer to a permutation of 0..M-1: the order in
@@ -189,9 +195,9 @@ int32_t ps_num_free_blocks(ps_ctx* ctx, int32_t* out);
  * Errors: PS_ERR_STATE, PS_ERR_HOST_NOMEM, PS_ERR_INVALID, PS_ERR_CUDA. */
 int32_t ps_swap_out(ps_ctx* ctx, int64_t req);
 
-/* Proactive incremental offloading (Section 4.3 "Asynchronous Offloading": a copy is triggered for every
- * n_off newly generated blocks of a request, with a smaller n_off for requests that are more likely to be
- * preempted).  If the RESIDENT request has at least n_off blocks that are completely filled
+/* Proactive incremental offloading (Section 4.3 "Asynchronous Offloading"): offloads a request's filled blocks
+ * in groups of n_off ahead of any eviction; the caller passes a smaller n_off for requests it expects to
+ * preempt sooner.  If the RESIDENT request has at least n_off blocks that are completely filled
  * (n_tokens / block_size) and not yet offloaded, the largest whole number of groups of n_off such blocks
  * is copied to the host as a new image segment, asynchronously and ordered after the work already
  * enqueued on the compute stream; the request stays RESIDENT and keeps decoding and growing.  Filled
@@ -345,6 +351,39 @@ int32_t ps_decode_attn_static(const void* kpool, const void* vpool, const void* 
 int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs,
                 int32_t batch, int64_t copy_budget_bytes, int32_t* decoded_mask, ps_step_stats* stats);
 
+/* ps_step with the partial-copy admission test of Section 4.3 "Put it Together" (Alg. 1, SatisfyCopyCondition)
+ * applied while the budget is consumed.  When the residual budget b_rem does not cover the b_miss missing blocks
+ * of a queued request that `rule` lists, the request receives the residual only if ps_copy_condition(l_comp,
+ * l_comp_max, b_miss, b_rem, block_size, beta) allows it; otherwise it is skipped in this step and the next
+ * request of the reload queue is tried with the budget unchanged.  Requests that `rule` does not list, and every
+ * request when rule == NULL, follow ps_step's reduced rule (the residual is always given).
+ *   rule->reqs[i]       : request id
+ *   rule->l_comp[i]     : tokens the scheduler could still compute for it in this round after a partial copy
+ *                         (0 for a request that only decodes: it cannot run before its last block is back)
+ *   rule->l_comp_max[i] : the round's computable-token limit for it
+ * Errors: those of ps_step; PS_ERR_INVALID for beta <= 1, null arrays with n > 0, negative counts. */
+typedef struct ps_copy_rule {
+    double beta;
+    int32_t n;
+    int32_t reserved0;
+    const int64_t* reqs;
+    const int32_t* l_comp;
+    const int32_t* l_comp_max;
+} ps_copy_rule;
+int32_t ps_step_ruled(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs,
+                      int32_t batch, int64_t copy_budget_bytes, const ps_copy_rule* rule, int32_t* decoded_mask,
+                      ps_step_stats* stats);
+
+/* ps_step for callers whose queries and outputs live in HOST memory: copies q_host to a device buffer of the
+ * context on the compute stream, runs the step, and copies the outputs back, all asynchronously on the compute
+ * stream (synchronise that stream, or call ps_sync, before reading out_host).
+ *   q_host, out_host : host, bf16 [num_layers][batch][num_q_heads][head_dim]; pinned memory keeps the copies
+ *                      asynchronous.  Rows of out_host whose request did not decode are zero.
+ * The context's two device buffers ([num_layers][max_batch][num_q_heads][head_dim] each) are allocated by the
+ * first call.  Errors: those of ps_step; PS_ERR_INVALID (batch 0, null buffers, bookkeeping-only context). */
+int32_t ps_step_host(ps_ctx* ctx, const void* q_host, void* out_host, const int64_t* reqs, int32_t batch,
+                     int64_t copy_budget_bytes, int32_t* decoded_mask, ps_step_stats* stats);
+
 /* ---- adaptive copy budget (Section 4.3 "Adaptive Copy-Budget Control") -------------------- */
 
 /* Latency model of one decode step and of the host link, in microseconds (Section 4.1: a decode request
@@ -379,8 +418,7 @@ int32_t ps_copy_budget(ps_ctx* ctx, const int64_t* reqs, int32_t batch, const ps
 
 /* ---- eviction policy and partial-copy admission (Section 4.3) ----------------------------- */
 
-/* "Eviction Policy": when device memory is saturated, evict requests near the tail of the sorted queue,
- * except those whose waiting time is close to the starvation threshold.
+/* Victim choice under memory pressure (Section 4.3 "Eviction Policy").
  *   queue      : host array of n request ids in the scheduler's order, head (next to run) first
  *   waited_us  : host array of n waiting times
  *   tau_us     : the starvation threshold; near_frac in (0, 1]: "close to" means waited >= near_frac * tau
@@ -494,13 +532,20 @@ int32_t ps_trace_read(ps_ctx* ctx, ps_trace_span* out, int32_t cap, int32_t* n);
  * Allocates and frees its own buffers; needs no context. */
 int32_t ps_link_probe(int64_t bytes, int32_t direction, int32_t iters, double* gb_per_s);
 
-/* On-device gather / scatter of `n_blocks` blocks of one layer between the pools and a contiguous
- * device buffer, without any host transfer: the kernels of ps_swap_out / ps_swap_in_layer alone,
- * for measuring them against HBM bandwidth.  `staging` is a device pointer with room for
- * n_blocks * 2 slabs ([n][K,V][slab]); ids is a host array of n_blocks block ids.  Runs on the
- * compute stream.  direction 0 = gather (pool -> staging), 1 = scatter (staging -> pool). */
-int32_t ps_copy_blocks(ps_ctx* ctx, int32_t layer, const int32_t* ids, int32_t n_blocks, void* staging,
-                       int32_t direction);
+/* The gather kernel of ps_swap_out (direction 0: pools -> staging) or the scatter kernel of ps_swap_in_layer /
+ * ps_step (direction 1: staging -> pools) alone, without any host transfer, on the compute stream: the same
+ * kernels in the launch shape the swap path gives them, for measuring them against HBM bandwidth.  One launch
+ * moves `n_blocks` blocks of the layers [layer, layer + n_layers); `staging` is a device pointer with room for
+ * n_layers * n_blocks * 2 slabs, laid out [n_layers][n_blocks][K,V][slab]; ids is a host array of n_blocks
+ * block ids.  n_layers > 1 is the shape of a reload's layer chunk under a small copy budget. */
+int32_t ps_copy_blocks(ps_ctx* ctx, int32_t layer, int32_t n_layers, const int32_t* ids, int32_t n_blocks,
+                       void* staging, int32_t direction);
+
+/* Test hook: writes `value` into the context's kernel status word as a kernel would (1 = a copy kernel met a
+ * bad block id, 2 = an attention kernel did, 3 = a bounded wait inside the attention kernel ran out; on a device
+ * context 3 also leaves the kernel's chunk and arrival counters dirty, as CTAs that gave up would).  The next
+ * ps_poll / ps_step / ps_sync then reports it.  Lets the error path be exercised without making a kernel fail. */
+int32_t ps_inject_status(ps_ctx* ctx, int32_t value);
 
 #ifdef __cplusplus
 }

@@ -32,7 +32,7 @@ EXPORTS = [
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
     "ps_decode_attn_static", "ps_copy_budget", "ps_offload_progress", "ps_host_blocks", "ps_host_segment",
     "ps_select_victims", "ps_copy_condition", "ps_order_queue", "ps_estimate_batch", "ps_resume_cost",
-    "ps_reload_fence", "ps_offload_sweep",
+    "ps_reload_fence", "ps_offload_sweep", "ps_step_ruled", "ps_step_host", "ps_inject_status",
 ]
 
 
@@ -41,7 +41,7 @@ class PsConfig(C.Structure):
         ("num_layers", C.c_int32), ("num_kv_heads", C.c_int32), ("num_q_heads", C.c_int32),
         ("head_dim", C.c_int32), ("block_size", C.c_int32), ("num_gpu_blocks", C.c_int32),
         ("max_blocks_per_req", C.c_int32), ("max_batch", C.c_int32), ("flags", C.c_int32),
-        ("attn_kernel", C.c_int32), ("kv_split_tokens", C.c_int32), ("reserved0", C.c_int32),
+        ("attn_kernel", C.c_int32), ("kv_split_tokens", C.c_int32), ("layer_chunk_bytes", C.c_int32),
         ("host_pool_bytes", C.c_int64), ("staging_bytes", C.c_int64),
         ("initial_free_order", C.POINTER(C.c_int32)),
     ]
@@ -75,6 +75,11 @@ class PsProfile(C.Structure):
 class PsBudgetModel(C.Structure):
     _fields_ = [("a_d_us_per_token", C.c_double), ("b_d_us", C.c_double), ("t_c_us", C.c_double),
                 ("t_block_us", C.c_double), ("t_budget_us", C.c_double)]
+
+
+class PsCopyRule(C.Structure):
+    _fields_ = [("beta", C.c_double), ("n", C.c_int32), ("reserved0", C.c_int32), ("reqs", C.POINTER(C.c_int64)),
+                ("l_comp", C.POINTER(C.c_int32)), ("l_comp_max", C.POINTER(C.c_int32))]
 
 
 class PsSchedParams(C.Structure):
@@ -136,7 +141,10 @@ def load() -> C.CDLL:
         "ps_launch_count": (i32, [vp, p64]),
         "ps_get_profile": (i32, [vp, C.POINTER(PsProfile), i32]),
         "ps_link_probe": (i32, [i64, i32, i32, C.POINTER(C.c_double)]),
-        "ps_copy_blocks": (i32, [vp, i32, p32, i32, vp, i32]),
+        "ps_copy_blocks": (i32, [vp, i32, i32, p32, i32, vp, i32]),
+        "ps_inject_status": (i32, [vp, i32]),
+        "ps_step_ruled": (i32, [vp, vp, vp, p64, i32, i64, C.POINTER(PsCopyRule), p32, C.POINTER(PsStepStats)]),
+        "ps_step_host": (i32, [vp, vp, vp, p64, i32, i64, p32, C.POINTER(PsStepStats)]),
         "ps_trace": (i32, [vp, i32]),
         "ps_trace_read": (i32, [vp, C.POINTER(PsTraceSpan), i32, p32]),
         "ps_offload_progress": (i32, [vp, i64, i32, p32]),
@@ -245,7 +253,7 @@ class KVSwap:
                  num_gpu_blocks: int, max_blocks_per_req: int, max_batch: int = 0, host_pool_bytes: int = 0,
                  staging_bytes: int = 0, initial_free_order=None, k_pools=None, v_pools=None, flags: int = 0,
                  attn_kernel: int = PS_ATTN_AUTO, kv_split_tokens: int = 0, host_pool_ptr: int = 0,
-                 compute_stream: Optional[int] = None):
+                 compute_stream: Optional[int] = None, layer_chunk_bytes: int = 0):
         self.lib = load()
         self.L = num_layers
         self.Hq, self.D = num_q_heads, head_dim
@@ -254,6 +262,7 @@ class KVSwap:
         cfg.head_dim, cfg.block_size, cfg.num_gpu_blocks = head_dim, block_size, num_gpu_blocks
         cfg.max_blocks_per_req, cfg.max_batch, cfg.flags = max_blocks_per_req, max_batch, flags
         cfg.attn_kernel, cfg.kv_split_tokens = attn_kernel, kv_split_tokens
+        cfg.layer_chunk_bytes = layer_chunk_bytes
         cfg.host_pool_bytes, cfg.staging_bytes = host_pool_bytes, staging_bytes
         self._order = None
         if initial_free_order is not None:
@@ -394,6 +403,36 @@ class KVSwap:
                               copy_budget_bytes, mask, C.byref(st))
         return rc, list(mask[: len(reqs)]), st.as_dict()
 
+    def step_ruled(self, q_all, out_all, reqs: Sequence[int], copy_budget_bytes: int, beta: float,
+                   rule_reqs: Sequence[int], l_comp: Sequence[int], l_comp_max: Sequence[int]):
+        """ps_step with the partial-copy admission test: (status, decoded mask list, stats dict)."""
+        arr = _i64_array(reqs)
+        mask = (C.c_int32 * max(len(reqs), 1))()
+        st = PsStepStats()
+        n = len(rule_reqs)
+        rr = _i64_array(rule_reqs)
+        lc = (C.c_int32 * max(n, 1))(*[int(v) for v in l_comp])
+        lm = (C.c_int32 * max(n, 1))(*[int(v) for v in l_comp_max])
+        rule = PsCopyRule(beta, n, 0, C.cast(rr, C.POINTER(C.c_int64)), C.cast(lc, C.POINTER(C.c_int32)),
+                          C.cast(lm, C.POINTER(C.c_int32)))
+        rc = self.lib.ps_step_ruled(self.h, C.c_void_p(q_all.data_ptr()) if q_all is not None else None,
+                                    C.c_void_p(out_all.data_ptr()) if out_all is not None else None, arr, len(reqs),
+                                    copy_budget_bytes, C.byref(rule), mask, C.byref(st))
+        return rc, list(mask[: len(reqs)]), st.as_dict()
+
+    def step_host(self, q_host, out_host, reqs: Sequence[int], copy_budget_bytes: int):
+        """ps_step with queries and outputs in host memory (tensors with data_ptr(), e.g. pinned CPU tensors):
+        (status, decoded mask list, stats dict).  Asynchronous: synchronise the compute stream before reading."""
+        arr = _i64_array(reqs)
+        mask = (C.c_int32 * max(len(reqs), 1))()
+        st = PsStepStats()
+        rc = self.lib.ps_step_host(self.h, C.c_void_p(q_host.data_ptr()), C.c_void_p(out_host.data_ptr()), arr,
+                                   len(reqs), copy_budget_bytes, mask, C.byref(st))
+        return rc, list(mask[: len(reqs)]), st.as_dict()
+
+    def inject_status(self, value: int) -> int:
+        return self.lib.ps_inject_status(self.h, value)
+
     def copy_budget(self, reqs: Sequence[int], *, a_d: float, b_d: float, t_c: float, t_block: float, t_budget: float):
         """Adaptive copy budget for the coming step: (status, blocks, bytes, case 1 / 21 / 22); times in us."""
         m = PsBudgetModel(a_d, b_d, t_c, t_block, t_budget)
@@ -444,6 +483,6 @@ class KVSwap:
         self._ck(self.lib.ps_trace_read(self.h, buf, n.value, C.byref(n)), "ps_trace_read")
         return [(TRACE_KINDS[s.kind], s.tag, s.start_us, s.end_us) for s in buf[: n.value]]
 
-    def copy_blocks(self, layer: int, ids: Sequence[int], staging, direction: int) -> int:
+    def copy_blocks(self, layer: int, ids: Sequence[int], staging, direction: int, n_layers: int = 1) -> int:
         arr = (C.c_int32 * max(len(ids), 1))(*[int(v) for v in ids])
-        return self.lib.ps_copy_blocks(self.h, layer, arr, len(ids), C.c_void_p(staging.data_ptr()), direction)
+        return self.lib.ps_copy_blocks(self.h, layer, n_layers, arr, len(ids), C.c_void_p(staging.data_ptr()), direction)

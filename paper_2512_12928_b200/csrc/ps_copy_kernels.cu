@@ -6,6 +6,11 @@
 // staging range that the copy engine filled back into freshly allocated blocks (Section 4.3,
 // "Asynchronous Offloading" and "Pipelined Reloading").  Pure byte movement: HBM-bound, 16-byte
 // coalesced accesses, several independent loads in flight per thread.
+//
+// Both directions walk the same "image range": slab s of the range belongs to layer
+// layer0 + s / (2 n), logical block (s % (2 n)) / 2 and tensor s & 1 (K, V), where n is the number
+// of block ids.  The staging side is contiguous in s; the pool side is pool[layer][tensor] at block
+// ids[j].  A block id is the same in every layer, so one id list serves a whole group of layers.
 #include "ps_internal.h"
 
 namespace ps {
@@ -39,63 +44,45 @@ __device__ __forceinline__ void copy_piece(const uint4* __restrict__ src, uint4*
     }
 }
 
-__global__ void __launch_bounds__(kCopyThreads)
-gather_image_kernel(const uint4* const* __restrict__ kpools, const uint4* const* __restrict__ vpools,
-                    const int32_t* __restrict__ table, int32_t n_blk, int64_t slab_begin, uint4* __restrict__ dst,
-                    int32_t slab_vec, int32_t pieces, int32_t num_blocks, int32_t* status) {
-    const int64_t local = blockIdx.x / pieces;
+// One CTA per 16 KiB piece of a slab.  kScatter = false: pool -> staging; true: staging -> pool.
+template <bool kScatter>
+__device__ __forceinline__ void image_copy(uint4* const* __restrict__ kpools, uint4* const* __restrict__ vpools,
+                                           const int32_t* __restrict__ ids, int32_t n, int32_t layer0,
+                                           int64_t slab_begin, uint4* __restrict__ staging, int32_t slab_vec,
+                                           int32_t pieces, int32_t num_blocks, int32_t* status) {
+    const int64_t local = blockIdx.x / pieces;  // slab inside this launch; staging is addressed from it
     const int piece = blockIdx.x - (int)(local * pieces);
     const int64_t s = slab_begin + local;
-    const int64_t per_layer = 2 * (int64_t)n_blk;
+    const int64_t per_layer = 2 * (int64_t)n;
     const int l = (int)(s / per_layer);
     const int rem = (int)(s - (int64_t)l * per_layer);
-    const int j = rem >> 1;
-    const int id = table[j];
+    const int id = ids[rem >> 1];
     if ((unsigned)id >= (unsigned)num_blocks) {
         if (threadIdx.x == 0) *(volatile int32_t*)status = 1;
         return;
     }
-    const uint4* pool = (rem & 1) ? vpools[l] : kpools[l];
-    copy_piece(pool + (int64_t)id * slab_vec, dst + local * slab_vec, piece * kPieceVec, slab_vec);
-}
-
-// kScatter = false: pool -> pairs; true: pairs -> pool.
-template <bool kScatter>
-__global__ void __launch_bounds__(kCopyThreads)
-layer_copy_kernel(uint4* __restrict__ kpool, uint4* __restrict__ vpool, const int32_t* __restrict__ ids,
-                  uint4* __restrict__ pairs, int32_t slab_vec, int32_t pieces, int32_t num_blocks, int32_t* status) {
-    const int local = blockIdx.x / pieces;  // slab index inside the pair array: 2 i + t
-    const int piece = blockIdx.x - local * pieces;
-    const int id = ids[local >> 1];
-    if ((unsigned)id >= (unsigned)num_blocks) {
-        if (threadIdx.x == 0) *(volatile int32_t*)status = 1;
-        return;
-    }
-    uint4* pool_slab = ((local & 1) ? vpool : kpool) + (int64_t)id * slab_vec;
-    uint4* pair_slab = pairs + (int64_t)local * slab_vec;
+    uint4* pool_slab = ((rem & 1) ? vpools[layer0 + l] : kpools[layer0 + l]) + (int64_t)id * slab_vec;
+    uint4* stage_slab = staging + local * slab_vec;
     if (kScatter)
-        copy_piece(pair_slab, pool_slab, piece * kPieceVec, slab_vec);
+        copy_piece(stage_slab, pool_slab, piece * kPieceVec, slab_vec);
     else
-        copy_piece(pool_slab, pair_slab, piece * kPieceVec, slab_vec);
+        copy_piece(pool_slab, stage_slab, piece * kPieceVec, slab_vec);
 }
 
-struct ParamIds {
-    int32_t ids[kMaxParamIds];
-};
+__global__ void __launch_bounds__(kCopyThreads)
+gather_image_kernel(uint4* const* __restrict__ kpools, uint4* const* __restrict__ vpools,
+                    const int32_t* __restrict__ ids, int32_t n, int32_t layer0, int64_t slab_begin,
+                    uint4* __restrict__ staging, int32_t slab_vec, int32_t pieces, int32_t num_blocks,
+                    int32_t* status) {
+    image_copy<false>(kpools, vpools, ids, n, layer0, slab_begin, staging, slab_vec, pieces, num_blocks, status);
+}
 
 __global__ void __launch_bounds__(kCopyThreads)
-scatter_param_ids_kernel(uint4* __restrict__ kpool, uint4* __restrict__ vpool, const __grid_constant__ ParamIds ids,
-                         const uint4* __restrict__ pairs, int32_t slab_vec, int32_t pieces, int32_t num_blocks,
-                         int32_t* status) {
-    const int local = blockIdx.x / pieces;
-    const int piece = blockIdx.x - local * pieces;
-    const int id = ids.ids[local >> 1];
-    if ((unsigned)id >= (unsigned)num_blocks) {
-        if (threadIdx.x == 0) *(volatile int32_t*)status = 1;
-        return;
-    }
-    uint4* pool_slab = ((local & 1) ? vpool : kpool) + (int64_t)id * slab_vec;
-    copy_piece(pairs + (int64_t)local * slab_vec, pool_slab, piece * kPieceVec, slab_vec);
+scatter_image_kernel(uint4* const* __restrict__ kpools, uint4* const* __restrict__ vpools,
+                     const int32_t* __restrict__ ids, int32_t n, int32_t layer0, int64_t slab_begin,
+                     uint4* __restrict__ staging, int32_t slab_vec, int32_t pieces, int32_t num_blocks,
+                     int32_t* status) {
+    image_copy<true>(kpools, vpools, ids, n, layer0, slab_begin, staging, slab_vec, pieces, num_blocks, status);
 }
 
 __global__ void __launch_bounds__(256)
@@ -108,41 +95,22 @@ inline int pieces_for(int32_t slab_vec) { return (slab_vec + kPieceVec - 1) / kP
 
 }  // namespace
 
-cudaError_t launch_gather_image(const void* const* d_kpools, const void* const* d_vpools, const int32_t* d_table,
-                                int32_t n_blk, int64_t slab_begin, int64_t slab_count, void* dst, int32_t slab_vec,
-                                int32_t num_blocks, int32_t* d_status, cudaStream_t stream) {
+cudaError_t launch_image_copy(bool scatter, void* const* d_kpools, void* const* d_vpools, const int32_t* d_ids,
+                              int32_t n, int32_t layer0, int64_t slab_begin, int64_t slab_count, void* staging,
+                              int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream) {
     if (slab_count <= 0) return cudaSuccess;
+    if (n <= 0) return cudaErrorInvalidValue;
     const int pieces = pieces_for(slab_vec);
     const int64_t grid = slab_count * pieces;
     if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
-    gather_image_kernel<<<(unsigned)grid, kCopyThreads, 0, stream>>>(
-        (const uint4* const*)d_kpools, (const uint4* const*)d_vpools, d_table, n_blk, slab_begin, (uint4*)dst,
-        slab_vec, pieces, num_blocks, d_status);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_scatter_layer(void* kpool, void* vpool, const int32_t* d_ids, int32_t n, const void* src,
-                                 int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream) {
-    if (n <= 0) return cudaSuccess;
-    const int pieces = pieces_for(slab_vec);
-    const int64_t grid = 2LL * n * pieces;
-    if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
-    layer_copy_kernel<true><<<(unsigned)grid, kCopyThreads, 0, stream>>>(
-        (uint4*)kpool, (uint4*)vpool, d_ids, (uint4*)const_cast<void*>(src), slab_vec, pieces, num_blocks, d_status);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_scatter_layer_ids(void* kpool, void* vpool, const int32_t* h_ids, int32_t n, const void* src,
-                                     int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream) {
-    if (n <= 0) return cudaSuccess;
-    if (n > kMaxParamIds) return cudaErrorInvalidValue;
-    ParamIds ids;
-    for (int32_t i = 0; i < n; ++i) ids.ids[i] = h_ids[i];
-    for (int32_t i = n; i < kMaxParamIds; ++i) ids.ids[i] = 0;
-    const int pieces = pieces_for(slab_vec);
-    const int64_t grid = 2LL * n * pieces;
-    scatter_param_ids_kernel<<<(unsigned)grid, kCopyThreads, 0, stream>>>(
-        (uint4*)kpool, (uint4*)vpool, ids, (const uint4*)src, slab_vec, pieces, num_blocks, d_status);
+    if (scatter)
+        scatter_image_kernel<<<(unsigned)grid, kCopyThreads, 0, stream>>>(
+            (uint4* const*)d_kpools, (uint4* const*)d_vpools, d_ids, n, layer0, slab_begin, (uint4*)staging, slab_vec,
+            pieces, num_blocks, d_status);
+    else
+        gather_image_kernel<<<(unsigned)grid, kCopyThreads, 0, stream>>>(
+            (uint4* const*)d_kpools, (uint4* const*)d_vpools, d_ids, n, layer0, slab_begin, (uint4*)staging, slab_vec,
+            pieces, num_blocks, d_status);
     return cudaGetLastError();
 }
 
@@ -153,18 +121,6 @@ cudaError_t launch_upload(void* dst, const void* src_mapped, size_t bytes, cudaS
     const int64_t want = (n_vec + 255) / 256;
     const unsigned grid = (unsigned)(want < 64 ? want : 64);
     upload_kernel<<<grid, 256, 0, stream>>>((uint4*)dst, (const uint4*)src_mapped, n_vec);
-    return cudaGetLastError();
-}
-
-cudaError_t launch_gather_layer(const void* kpool, const void* vpool, const int32_t* d_ids, int32_t n, void* dst,
-                                int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream) {
-    if (n <= 0) return cudaSuccess;
-    const int pieces = pieces_for(slab_vec);
-    const int64_t grid = 2LL * n * pieces;
-    if (grid > 0x7fffffffLL) return cudaErrorInvalidValue;
-    layer_copy_kernel<false><<<(unsigned)grid, kCopyThreads, 0, stream>>>(
-        (uint4*)const_cast<void*>(kpool), (uint4*)const_cast<void*>(vpool), d_ids, (uint4*)dst, slab_vec, pieces,
-        num_blocks, d_status);
     return cudaGetLastError();
 }
 

@@ -5,6 +5,7 @@
 #include <chrono>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <deque>
 #include <map>
@@ -161,16 +162,24 @@ struct ps_ctx {
     cudaEvent_t e_gathered[kSlots]{}, e_drained[kSlots]{}, e_loaded[kSlots]{}, e_scattered[kSlots]{};
     bool out_used[kSlots]{}, in_used[kSlots]{};
     uint64_t out_next = 0, in_next = 0;
-    std::vector<cudaEvent_t> ev_in;  // per layer
+    int in_slot = -1;        // reload staging: the slot being filled and the bytes used in it (pieces are packed)
+    int64_t in_fill = 0;
+    std::vector<cudaEvent_t> ev_in;      // completion events of layer chunks, indexed by the chunk's first layer
+    std::vector<int32_t> ev_of_layer;    // per layer: first layer of the chunk that last reloaded into it
+    int64_t chunk_min_bytes = 0;         // layers are grouped into one chunk until a chunk carries this many bytes
+    int64_t max_pitch = 0;               // largest row pitch of a strided copy
     cudaEvent_t e_mark = nullptr, e_mark2 = nullptr, e_fork = nullptr, e_join = nullptr;
     int32_t* status = nullptr;  // mapped pinned word written by kernels on a bad block id
     int32_t* d_status = nullptr;
     Tracker t_d2h, t_scatter, t_compute;
-    Arena a_gather, a_meta, a_ids;
+    Arena a_gather, a_meta, a_ids, a_scatter;
+    std::vector<int32_t> scatter_ids_cache;  // ids of the last reload-plan upload and where they sit in a_scatter
+    size_t scatter_ids_off = 0;
     std::vector<int32_t> ids_cache;  // ids of the last ps_copy_blocks upload and where they sit in a_ids
     size_t ids_cache_off = 0;
     std::vector<cudaEvent_t> ev_pool, ev_pool_timing;
     std::deque<std::pair<uint64_t, std::pair<int64_t, int64_t>>> img_release;  // in_ticket -> (off, bytes)
+    std::deque<std::pair<uint64_t, std::pair<int64_t, int64_t>>> host_release;  // t_d2h ticket -> (off, bytes)
     std::vector<int64_t> gated_reqs;
     // split-KV scratch: sets 0 and 1 are used alternately by the launches on the compute stream (consecutive
     // launches of a step may overlap), set 2 by the launches on the reload lane
@@ -183,6 +192,8 @@ struct ps_ctx {
     int attn_kernel = 1;
     int32_t num_sms = 1;
     BatchMeta meta;
+    char* io_q = nullptr;    // ps_step_host: device copies of the queries and of the outputs (allocated on first use)
+    char* io_out = nullptr;
 
     // measurement
     int64_t launches = 0;
@@ -261,12 +272,13 @@ int32_t do_poll(ps_ctx* ctx, int32_t* n_reaped);
 // swap-out and swap-in issue (ps_swap.cu)
 int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi);
 int32_t order_scatter_after_compute(ps_ctx* ctx);
-int32_t issue_reload_layer(ps_ctx* ctx, int32_t layer, const std::vector<PlanEntry>& plan);
+int32_t upload_plan_ids(ps_ctx* ctx, const std::vector<PlanEntry>& plan, const int32_t** d_ids);
+int32_t issue_reload_group(ps_ctx* ctx, int32_t l0, int32_t g, const std::vector<PlanEntry>& plan, const int32_t* d_ids);
 int32_t note_layer_issued(ps_ctx* ctx, int64_t id, Req& r, int32_t layer, int32_t hi);
 int32_t missing_of(const Req& r);
 
 // copy-budget consumption and the attention batch (ps_step.cu)
-std::vector<PlanEntry> make_plan(ps_ctx* ctx, int64_t copy_budget_bytes);
+std::vector<PlanEntry> make_plan(ps_ctx* ctx, int64_t copy_budget_bytes, const ps_copy_rule* rule);
 int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::vector<char>& active,
                       const std::vector<char>& gated, bool want_lanes, bool contended);
 int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, float* lse, cudaEvent_t wait_event,

@@ -10,32 +10,20 @@ namespace ps {
 
 // A "slab" is one block of one layer in one pool: slab_vec 16-byte vectors, contiguous.
 //
-// Gather: image slab s (s in [slab_begin, slab_begin + slab_count)) of a request with n_blk blocks
-// lives at layer l = s / (2 n_blk), logical block j = (s % (2 n_blk)) / 2, tensor t = s & 1
-// (0 = K, 1 = V); it is copied from pool[l][t] + table[j] * slab to dst + (s - slab_begin) * slab.
-cudaError_t launch_gather_image(const void* const* d_kpools, const void* const* d_vpools, const int32_t* d_table,
-                                int32_t n_blk, int64_t slab_begin, int64_t slab_count, void* dst, int32_t slab_vec,
-                                int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
-
-// Scatter for one layer: src holds n consecutive (K slab, V slab) pairs; pair i goes to block
-// d_ids[i] of kpool / vpool.
-cudaError_t launch_scatter_layer(void* kpool, void* vpool, const int32_t* d_ids, int32_t n, const void* src,
-                                 int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
-
-// Same, with the block ids passed by value in the kernel parameters (no descriptor upload at all);
-// h_ids is a host array, n <= kMaxParamIds per call.
-constexpr int kMaxParamIds = 960;
-cudaError_t launch_scatter_layer_ids(void* kpool, void* vpool, const int32_t* h_ids, int32_t n, const void* src,
-                                     int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
+// Image range over n block ids and the layers from layer0 on: slab s lives at layer layer0 + s / (2 n),
+// logical block j = (s % (2 n)) / 2, tensor t = s & 1 (0 = K, 1 = V).  The launch moves slabs
+// [slab_begin, slab_begin + slab_count) between pool[layer][t] + d_ids[j] * slab and
+// staging + (s - slab_begin) * slab: pool -> staging (gather, swap-out) or staging -> pool (scatter,
+// swap-in).  d_kpools / d_vpools are device arrays of the per-layer pool pointers, d_ids a device array.
+// An id outside [0, num_blocks) sets *d_status to 1 and its slabs are skipped.
+cudaError_t launch_image_copy(bool scatter, void* const* d_kpools, void* const* d_vpools, const int32_t* d_ids,
+                              int32_t n, int32_t layer0, int64_t slab_begin, int64_t slab_count, void* staging,
+                              int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
 
 // Copies `bytes` (a multiple of 16) from mapped pinned host memory (device view src) to device
 // memory with a small kernel, so that descriptor uploads never queue behind bulk transfers in a
 // copy engine.
 cudaError_t launch_upload(void* dst, const void* src_mapped, size_t bytes, cudaStream_t stream);
-
-// Gather for one layer into the same pair layout (the inverse of launch_scatter_layer).
-cudaError_t launch_gather_layer(const void* kpool, const void* vpool, const int32_t* d_ids, int32_t n, void* dst,
-                                int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
 
 // ---- paged decode attention --------------------------------------------------------------------
 

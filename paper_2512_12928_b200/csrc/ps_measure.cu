@@ -3,12 +3,12 @@
 
 extern "C" {
 
-int32_t ps_copy_blocks(ps_ctx* ctx, int32_t layer, const int32_t* ids, int32_t n_blocks, void* staging,
-                       int32_t direction) {
+int32_t ps_copy_blocks(ps_ctx* ctx, int32_t layer, int32_t n_layers, const int32_t* ids, int32_t n_blocks,
+                       void* staging, int32_t direction) {
     if (!ctx) return PS_ERR_INVALID;
     if (ctx->bk) return ctx->fail(PS_ERR_INVALID, "ps_copy_blocks: context holds no device (bookkeeping only)");
-    if (layer < 0 || layer >= ctx->cfg.num_layers || !ids || n_blocks < 0 || n_blocks > ctx->cfg.num_gpu_blocks ||
-        !staging || (direction != 0 && direction != 1))
+    if (layer < 0 || n_layers < 1 || layer + n_layers > ctx->cfg.num_layers || !ids || n_blocks < 0 ||
+        n_blocks > ctx->cfg.num_gpu_blocks || !staging || (direction != 0 && direction != 1))
         return ctx->fail(PS_ERR_INVALID, "ps_copy_blocks: bad argument");
     if (n_blocks == 0) return PS_OK;
     for (int32_t i = 0; i < n_blocks; ++i)
@@ -27,17 +27,31 @@ int32_t ps_copy_blocks(ps_ctx* ctx, int32_t layer, const int32_t* ids, int32_t n
         ctx->ids_cache_off = ioff;
     }
     const int32_t* d_ids = (const int32_t*)(ctx->a_ids.d + ioff);
-    const int64_t bytes = (int64_t)n_blocks * ctx->layer_block_bytes;
-    if (direction == 0) {
-        ProfScope prof(ctx, kProfGather, ctx->compute, bytes);
-        CK(ps::launch_gather_layer(ctx->kpools[(size_t)layer], ctx->vpools[(size_t)layer], d_ids, n_blocks, staging,
-                                   ctx->slab_vec, ctx->cfg.num_gpu_blocks, ctx->d_status, ctx->compute));
-    } else {
-        ProfScope prof(ctx, kProfScatter, ctx->compute, bytes);
-        CK(ps::launch_scatter_layer(ctx->kpools[(size_t)layer], ctx->vpools[(size_t)layer], d_ids, n_blocks, staging,
-                                    ctx->slab_vec, ctx->cfg.num_gpu_blocks, ctx->d_status, ctx->compute));
+    const int64_t bytes = (int64_t)n_layers * n_blocks * ctx->layer_block_bytes;
+    {
+        // the launch swap-out (direction 0) and swap-in (direction 1) make, on the compute stream
+        ProfScope prof(ctx, direction == 0 ? kProfGather : kProfScatter, ctx->compute, bytes);
+        CK(ps::launch_image_copy(direction == 1, ctx->d_kpools, ctx->d_vpools, d_ids, n_blocks, layer, 0,
+                                 2LL * n_blocks * n_layers, staging, ctx->slab_vec, ctx->cfg.num_gpu_blocks, ctx->d_status,
+                                 ctx->compute));
     }
     ctx->launches++;
+    return PS_OK;
+}
+
+int32_t ps_inject_status(ps_ctx* ctx, int32_t value) {
+    if (!ctx || !ctx->status) return PS_ERR_INVALID;
+    if (value < 1 || value > 3) return ctx->fail(PS_ERR_INVALID, "ps_inject_status: value must be 1, 2 or 3");
+    if (value == 3 && !ctx->bk) {
+        // what CTAs that gave up leave behind: chunk and arrival counters that were not re-armed
+        const size_t done_bytes = (size_t)std::max(ctx->cfg.max_batch, 1) * ctx->cfg.num_kv_heads * sizeof(int32_t);
+        for (int i = 0; i < 3; ++i) {
+            cudaStream_t st = i == 2 ? ctx->s_lane : ctx->compute;
+            if (ctx->d_sched[i]) CK(cudaMemsetAsync(ctx->d_sched[i], 0x01, 4 * sizeof(int32_t), st));
+            if (ctx->d_row_done[i]) CK(cudaMemsetAsync(ctx->d_row_done[i], 0x01, done_bytes, st));
+        }
+    }
+    *(volatile int32_t*)ctx->status = value;
     return PS_OK;
 }
 

@@ -11,7 +11,8 @@
 //   s_h2d    : pinned host -> staging copies.        s_scatter : scatter kernels of swap-in.
 // Each direction owns kSlots staging slots; two events per slot hand a slot back and forth between
 // the kernel stream and the copy-engine stream, so the copy engine never waits for a kernel launch
-// and a kernel never reads a slot the engine is still filling.
+// and a kernel never reads a slot the engine is still filling.  Reload pieces smaller than a slot are
+// packed into the current slot one after the other.
 #include "ps_ctx.h"
 
 namespace psrt {
@@ -156,10 +157,28 @@ void push_table(ps_ctx* ctx, std::vector<int32_t>& table) {
     ctx->table_epoch++;
 }
 
+// Kernels report through one mapped word: 1 = a copy kernel met a block id outside the pool, 2 = an attention
+// kernel did, 3 = a bounded wait inside the tensor-core attention kernel ran out and its CTAs left early.
+// After 3 the launch's outputs are undefined and its CTAs did not re-arm the kernel's chunk and arrival
+// counters, so these are cleared on their streams before anything else is launched over them.
 int32_t check_status_word(ps_ctx* ctx) {
     if (ctx->status && *(volatile int32_t*)ctx->status != 0) {
         const int v = *(volatile int32_t*)ctx->status;
         *(volatile int32_t*)ctx->status = 0;
+        if (v == 3) {
+            if (!ctx->bk) {
+                const size_t done_bytes = (size_t)std::max(ctx->cfg.max_batch, 1) * ctx->cfg.num_kv_heads * sizeof(int32_t);
+                for (int i = 0; i < 3; ++i) {
+                    cudaStream_t st = i == 2 ? ctx->s_lane : ctx->compute;
+                    if (ctx->d_sched[i]) CK(cudaMemsetAsync(ctx->d_sched[i], 0, 4 * sizeof(int32_t), st));
+                    if (ctx->d_row_done[i]) CK(cudaMemsetAsync(ctx->d_row_done[i], 0, done_bytes, st));
+                }
+            }
+            ctx->meta.valid = false;
+            return ctx->fail(PS_ERR_TIMEOUT,
+                             "attention kernel: a bounded wait on a shared-memory barrier ran out; the outputs of the "
+                             "launches in flight are undefined; the kernel's counters have been reset");
+        }
         return ctx->fail(PS_ERR_BOUNDS, v == 2 ? "attention kernel met a block id outside the pool"
                                                : "copy kernel met a block id outside the pool");
     }
@@ -177,6 +196,10 @@ int32_t do_poll(ps_ctx* ctx, int32_t* n_reaped) {
         r.state = PS_REQ_HOST;
         ctx->out_fifo.pop_front();
         ++reaped;
+    }
+    while (!ctx->host_release.empty() && ctx->host_release.front().first <= ctx->t_d2h.done) {
+        ctx->hpool.release(ctx->host_release.front().second.first, ctx->host_release.front().second.second);
+        ctx->host_release.pop_front();
     }
     rc = tracker_poll(ctx, ctx->t_scatter);
     if (rc != PS_OK) return rc;
@@ -221,6 +244,9 @@ void destroy_ctx(ps_ctx* ctx) {
         arena_free(ctx->a_gather);
         arena_free(ctx->a_meta);
         arena_free(ctx->a_ids);
+        arena_free(ctx->a_scatter);
+        if (ctx->io_q) cudaFree(ctx->io_q);
+        if (ctx->io_out) cudaFree(ctx->io_out);
         if (ctx->stage_out) cudaFree(ctx->stage_out);
         if (ctx->stage_in) cudaFree(ctx->stage_in);
         if (ctx->d_kpools) cudaFree(ctx->d_kpools);
@@ -231,9 +257,11 @@ void destroy_ctx(ps_ctx* ctx) {
             if (ctx->d_row_done[i]) cudaFree(ctx->d_row_done[i]);
         }
         if (ctx->status) cudaFreeHost(ctx->status);
+        ctx->status = nullptr;
         if (ctx->own_host_pool && ctx->host_pool) cudaFreeHost(ctx->host_pool);
         cudaGetLastError();
     }
+    if (ctx->bk && ctx->status) free(ctx->status);
     delete ctx;
 }
 
@@ -306,7 +334,11 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
         }
     }
     ctx->hpool.init(cfg->host_pool_bytes);
+    ctx->chunk_min_bytes = cfg->layer_chunk_bytes == 0 ? (2LL << 20) : std::max<int64_t>(cfg->layer_chunk_bytes, 0);
+    ctx->ev_of_layer.resize((size_t)cfg->num_layers);
+    for (int32_t l = 0; l < cfg->num_layers; ++l) ctx->ev_of_layer[(size_t)l] = l;
     if (ctx->bk) {
+        ctx->status = (int32_t*)calloc(16, sizeof(int32_t));  // no kernel writes it; the status path stays testable
         *out = ctx;
         return PS_OK;
     }
@@ -387,6 +419,13 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     const size_t desc_chunk = std::max<size_t>((size_t)cfg->max_blocks_per_req * 4 * 8, 1 << 20);
     CKR(arena_init(ctx, ctx->a_gather, desc_chunk, 4, ctx->s_gather));
     CKR(arena_init(ctx, ctx->a_ids, (size_t)cfg->num_gpu_blocks * 4, 4, ctx->compute));  // ps_copy_blocks
+    CKR(arena_init(ctx, ctx->a_scatter, (size_t)cfg->num_gpu_blocks * 4, 4, ctx->s_scatter));  // reload plans
+    {
+        int dev = 0, pitch = 0;
+        CKC(cudaGetDevice(&dev));
+        CKC(cudaDeviceGetAttribute(&pitch, cudaDevAttrMaxPitch, dev));
+        ctx->max_pitch = pitch;
+    }
 
     // split-KV scratch
     ctx->attn_kernel = PS_ATTN_SIMT;

@@ -5,9 +5,12 @@
 
 namespace psrt {
 
-// Copy-budget consumption (Alg. 1, ConsumeCopyBudget, reduced to the byte budget): FIFO, whole request if it
-// fits, otherwise the residual.
-std::vector<PlanEntry> make_plan(ps_ctx* ctx, int64_t copy_budget_bytes) {
+// Copy-budget consumption (Alg. 1, ConsumeCopyBudget, with the byte budget turned into blocks): FIFO, whole
+// request if it fits, otherwise the residual -- always (rule == nullptr or the request is not listed in it), or
+// only if SatisfyCopyCondition holds for the request (Section 4.3 "Put it Together": l_comp reaches the round's
+// limit, or l_comp / ((b_miss - B_rem) * s_blk) > beta); a request that fails the test is skipped for this
+// round and the next one in the queue is tried with the budget unchanged.
+std::vector<PlanEntry> make_plan(ps_ctx* ctx, int64_t copy_budget_bytes, const ps_copy_rule* rule) {
     std::vector<PlanEntry> plan;
     const bool unlimited = copy_budget_bytes < 0;
     int64_t left = unlimited ? 0 : copy_budget_bytes / ctx->block_bytes;
@@ -16,15 +19,38 @@ std::vector<PlanEntry> make_plan(ps_ctx* ctx, int64_t copy_budget_bytes) {
         const int32_t miss = missing_of(r);
         if (miss == 0) continue;
         const int32_t lo = (int32_t)r.table.size() - miss;
-        const int64_t take = unlimited ? miss : std::min<int64_t>(miss, left);
-        if (take == 0) break;
-        plan.push_back({id, lo, lo + (int32_t)take});
-        if (!unlimited) {
-            left -= take;
-            if (left == 0) break;
+        if (!unlimited && left == 0) break;
+        int64_t take = miss;
+        if (!unlimited && miss > left) {
+            bool allowed = true;
+            if (rule != nullptr)
+                for (int32_t k = 0; k < rule->n; ++k)
+                    if (rule->reqs[k] == id) {
+                        int32_t ok = 1;
+                        ps_copy_condition(rule->l_comp[k], rule->l_comp_max[k], miss, (int32_t)left, ctx->cfg.block_size,
+                                          rule->beta, &ok);
+                        allowed = ok != 0;
+                        break;
+                    }
+            if (!allowed) continue;
+            take = left;
         }
+        plan.push_back({id, lo, lo + (int32_t)take});
+        if (!unlimited) left -= take;
     }
     return plan;
+}
+
+// Layers per chunk for a step that reloads n_blocks blocks: one layer's share of the step (n_blocks * layer
+// block bytes) may be far below what a copy engine needs to run at link rate, so consecutive layers are
+// grouped until a chunk carries chunk_min_bytes (Appendix B speaks of a completion event per layer *chunk*).
+// A chunk must fit a staging slot.
+int32_t layers_per_chunk(const ps_ctx* ctx, int64_t n_blocks) {
+    const int64_t per_layer = n_blocks * ctx->layer_block_bytes;
+    if (ctx->chunk_min_bytes <= 0 || per_layer <= 0 || per_layer >= ctx->chunk_min_bytes) return 1;
+    int64_t g = (ctx->chunk_min_bytes + per_layer - 1) / per_layer;
+    g = std::min<int64_t>(g, ctx->slot_bytes / per_layer);
+    return (int32_t)std::max<int64_t>(1, std::min<int64_t>(g, ctx->cfg.num_layers));
 }
 
 // ---- attention batch ------------------------------------------------------------------------------------
@@ -342,14 +368,22 @@ int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, flo
     int32_t rc = prepare_batch(ctx, reqs, batch, active, gated, /*want_lanes=*/false, /*contended=*/false);
     if (rc != PS_OK) return rc;
     int32_t launched = 0;
-    return launch_layer_attn(ctx, layer, q, out, lse, ctx->meta.n_gated_rows ? ctx->ev_in[(size_t)layer] : nullptr,
+    return launch_layer_attn(ctx, layer, q, out, lse,
+                             ctx->meta.n_gated_rows ? ctx->ev_in[(size_t)ctx->ev_of_layer[(size_t)layer]] : nullptr,
                              /*follows_own=*/false, &launched);
 }
 
-int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs, int32_t batch,
-                int64_t copy_budget_bytes, int32_t* decoded_mask, ps_step_stats* stats) {
-    if (!ctx) return PS_ERR_INVALID;
+static int32_t step_impl(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs,
+                         int32_t batch, int64_t copy_budget_bytes, const ps_copy_rule* rule, int32_t* decoded_mask,
+                         ps_step_stats* stats) {
     if (batch < 0 || (batch > 0 && !reqs)) return ctx->fail(PS_ERR_INVALID, "ps_step: bad batch");
+    if (rule != nullptr && (!(rule->beta > 1.0) || rule->n < 0 ||
+                            (rule->n > 0 && (!rule->reqs || !rule->l_comp || !rule->l_comp_max))))
+        return ctx->fail(PS_ERR_INVALID, "ps_step_ruled: beta must exceed 1 and the rule's arrays must be given");
+    if (rule != nullptr)
+        for (int32_t k = 0; k < rule->n; ++k)
+            if (rule->l_comp[k] < 0 || rule->l_comp_max[k] < 0)
+                return ctx->fail(PS_ERR_INVALID, "ps_step_ruled: negative token count in the rule");
     const bool want_attn = q_all_layers != nullptr || out_all_layers != nullptr;
     if (want_attn && (ctx->bk || !q_all_layers || !out_all_layers || batch > ctx->cfg.max_batch))
         return ctx->fail(PS_ERR_INVALID, "ps_step: attention needs q and out on a device context, batch <= max_batch");
@@ -360,7 +394,7 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
     st.swapouts_reaped = reaped;
 
     // 1. the copy budget is consumed over the reload queue
-    const std::vector<PlanEntry> plan = make_plan(ctx, copy_budget_bytes);
+    const std::vector<PlanEntry> plan = make_plan(ctx, copy_budget_bytes, rule);
     std::vector<char> completes(plan.size(), 0);
     for (size_t i = 0; i < plan.size(); ++i) {
         st.blocks_copied += plan[i].hi - plan[i].lo;
@@ -398,17 +432,34 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
         st.gated = ctx->meta.n_gated_rows;
     }
 
-    // 3. per layer: reload chunk on the copy streams, then that layer's attention on the compute stream
+    // 3. the step's layer chunks: first_of[l] = size of the chunk that starts at layer l, else 0.  When rows of
+    // the batch wait for this step's reload, the first chunk is a single layer, so that their first layer
+    // starts after the smallest possible transfer.
+    std::vector<int32_t> first_of((size_t)L, 0);
+    const int32_t* d_ids = nullptr;
     if (!plan.empty()) {
         rc = order_scatter_after_compute(ctx);
         if (rc != PS_OK) return rc;
-    }
-    const bool sync_reload = (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) != 0 || !attn;
-    if (sync_reload)
-        for (int l = 0; l < L; ++l) {
-            rc = issue_reload_layer(ctx, l, plan);
-            if (rc != PS_OK) return rc;
+        rc = upload_plan_ids(ctx, plan, &d_ids);
+        if (rc != PS_OK) return rc;
+        const int32_t g = layers_per_chunk(ctx, st.blocks_copied);
+        int32_t l = 0;
+        if (g > 1 && attn && ctx->meta.n_gated_rows > 0) first_of[(size_t)l++] = 1;
+        while (l < L) {
+            first_of[(size_t)l] = std::min<int32_t>(g, L - l);
+            l += first_of[(size_t)l];
         }
+    }
+
+    // 4. per layer: its reload chunk (if one starts here) on the copy streams, then the layer's attention on
+    // the compute stream
+    const bool sync_reload = (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) != 0 || !attn;
+    if (sync_reload && !plan.empty())
+        for (int l = 0; l < L; ++l)
+            if (first_of[(size_t)l] > 0) {
+                rc = issue_reload_group(ctx, l, first_of[(size_t)l], plan, d_ids);
+                if (rc != PS_OK) return rc;
+            }
     if (attn) {
         const int64_t layer_bytes = (int64_t)batch * ctx->cfg.num_q_heads * ctx->cfg.head_dim * 2;
         const bool any_gated = ctx->meta.n_gated_rows > 0;
@@ -418,16 +469,16 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
             CK(cudaStreamWaitEvent(ctx->s_lane, ctx->e_fork, 0));
         }
         for (int l = 0; l < L; ++l) {
-            if (!sync_reload) {
-                rc = issue_reload_layer(ctx, l, plan);
+            if (!sync_reload && !plan.empty() && first_of[(size_t)l] > 0) {
+                rc = issue_reload_group(ctx, l, first_of[(size_t)l], plan, d_ids);
                 if (rc != PS_OK) return rc;
             }
             cudaEvent_t wait = nullptr;
             if (any_gated) {
                 if (!sync_reload)
-                    wait = ctx->ev_in[(size_t)l];
+                    wait = ctx->ev_in[(size_t)ctx->ev_of_layer[(size_t)l]];
                 else if (l == 0)
-                    wait = ctx->ev_in[(size_t)L - 1];  // the whole reload, once, before the first layer
+                    wait = ctx->ev_in[(size_t)ctx->ev_of_layer[(size_t)L - 1]];  // the whole reload, once, before the first layer
             }
             int32_t launched = 0;
             rc = launch_layer_attn(ctx, l, (const char*)q_all_layers + l * layer_bytes,
@@ -440,7 +491,7 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
         }
     }
 
-    // 4. request states follow what was issued
+    // 5. request states follow what was issued
     for (size_t i = 0; i < plan.size(); ++i) {
         Req& r = ctx->reqs[plan[i].req];
         for (int l = 0; l < L; ++l) {
@@ -461,6 +512,44 @@ int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, con
     }
     st.kernel_launches = (int32_t)(ctx->launches - launches_before);
     if (stats) *stats = st;
+    return PS_OK;
+}
+
+int32_t ps_step(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs, int32_t batch,
+                int64_t copy_budget_bytes, int32_t* decoded_mask, ps_step_stats* stats) {
+    if (!ctx) return PS_ERR_INVALID;
+    return step_impl(ctx, q_all_layers, out_all_layers, reqs, batch, copy_budget_bytes, nullptr, decoded_mask, stats);
+}
+
+int32_t ps_step_ruled(ps_ctx* ctx, const void* q_all_layers, void* out_all_layers, const int64_t* reqs, int32_t batch,
+                      int64_t copy_budget_bytes, const ps_copy_rule* rule, int32_t* decoded_mask, ps_step_stats* stats) {
+    if (!ctx) return PS_ERR_INVALID;
+    return step_impl(ctx, q_all_layers, out_all_layers, reqs, batch, copy_budget_bytes, rule, decoded_mask, stats);
+}
+
+int32_t ps_step_host(ps_ctx* ctx, const void* q_host, void* out_host, const int64_t* reqs, int32_t batch,
+                     int64_t copy_budget_bytes, int32_t* decoded_mask, ps_step_stats* stats) {
+    if (!ctx) return PS_ERR_INVALID;
+    if (ctx->bk) return ctx->fail(PS_ERR_INVALID, "ps_step_host: context holds no device (bookkeeping only)");
+    if (batch <= 0 || batch > ctx->cfg.max_batch || !q_host || !out_host || !reqs)
+        return ctx->fail(PS_ERR_INVALID, "ps_step_host: needs q, out and 1 <= batch <= max_batch");
+    const size_t row = (size_t)ctx->cfg.num_q_heads * ctx->cfg.head_dim * 2;
+    const size_t bytes = (size_t)ctx->cfg.num_layers * batch * row;
+    if (ctx->io_q == nullptr) {  // first use: device buffers for the largest batch
+        const size_t cap = (size_t)ctx->cfg.num_layers * ctx->cfg.max_batch * row;
+        CK(cudaMalloc((void**)&ctx->io_q, cap));
+        cudaError_t e = cudaMalloc((void**)&ctx->io_out, cap);
+        if (e != cudaSuccess) {
+            cudaFree(ctx->io_q);
+            ctx->io_q = nullptr;
+            return ctx->fail_cuda(e, "cudaMalloc(step output buffer)");
+        }
+    }
+    CK(cudaMemcpyAsync(ctx->io_q, q_host, bytes, cudaMemcpyHostToDevice, ctx->compute));
+    CK(cudaMemsetAsync(ctx->io_out, 0, bytes, ctx->compute));
+    int32_t rc = step_impl(ctx, ctx->io_q, ctx->io_out, reqs, batch, copy_budget_bytes, nullptr, decoded_mask, stats);
+    if (rc != PS_OK) return rc;
+    CK(cudaMemcpyAsync(out_host, ctx->io_out, bytes, cudaMemcpyDeviceToHost, ctx->compute));
     return PS_OK;
 }
 

@@ -16,58 +16,122 @@ int32_t order_scatter_after_compute(ps_ctx* ctx) {
     return PS_OK;
 }
 
-// Issues the reload of one layer for a list of (request, block range); records ev_in[layer].
-int32_t issue_reload_layer(ps_ctx* ctx, int32_t layer, const std::vector<PlanEntry>& plan) {
+// Uploads the block ids of a reload plan (plan order) to the device on the scatter stream and returns where
+// they sit.  A block id is the same in every layer, so one upload serves all the layer chunks of a step; a
+// repeat of the previous upload (the caller-driven layer loop over one block range) reuses it.
+int32_t upload_plan_ids(ps_ctx* ctx, const std::vector<PlanEntry>& plan, const int32_t** d_ids) {
+    *d_ids = nullptr;
+    if (ctx->bk || plan.empty()) return PS_OK;
+    std::vector<int32_t> ids;
+    for (const PlanEntry& e : plan) {
+        const Req& r = ctx->reqs[e.req];
+        ids.insert(ids.end(), r.table.begin() + e.lo, r.table.begin() + e.hi);
+    }
+    if (ids.empty()) return PS_OK;
+    if (ids != ctx->scatter_ids_cache) {
+        size_t off = 0;
+        int32_t rc = arena_alloc(ctx, ctx->a_scatter, ids.size() * 4, &off);
+        if (rc != PS_OK) return rc;
+        memcpy(ctx->a_scatter.h + off, ids.data(), ids.size() * 4);
+        CK(ps::launch_upload(ctx->a_scatter.d + off, ctx->a_scatter.hd + off, (size_t)round_up((int64_t)ids.size() * 4, 16),
+                             ctx->s_scatter));
+        ctx->launches++;
+        ctx->scatter_ids_cache.swap(ids);
+        ctx->scatter_ids_off = off;
+    }
+    *d_ids = (const int32_t*)(ctx->a_scatter.d + ctx->scatter_ids_off);
+    return PS_OK;
+}
+
+// Issues one layer chunk of a reload plan: layers [l0, l0 + g) of every (request, block range) of the plan.
+// Host image -> staging on the H2D stream (per request and image segment one copy: a contiguous range for
+// g = 1, a strided one of g rows otherwise, since a layer's blocks are contiguous in the image and the
+// layers are a fixed stride apart), then one scatter launch per staging piece on the scatter stream, then
+// the chunk's completion event (Appendix B: one event per layer chunk), which every layer of the chunk
+// refers to.  d_ids: the plan's ids on the device (upload_plan_ids).  Pieces are packed into the current
+// staging slot while they fit, so small chunks never wait for a slot.
+int32_t issue_reload_group(ps_ctx* ctx, int32_t l0, int32_t g, const std::vector<PlanEntry>& plan,
+                           const int32_t* d_ids) {
     if (ctx->bk || plan.empty()) return PS_OK;
     const int64_t Bl = ctx->layer_block_bytes;
-    const int64_t cap = ctx->slot_bytes / Bl;  // pairs per slot
+    int64_t left = 0;
+    for (const PlanEntry& e : plan) left += e.hi - e.lo;
+    if (left == 0) return PS_OK;
+    const int64_t cap = std::max<int64_t>(ctx->slot_bytes / (g * Bl), 1);  // blocks per staging piece
     size_t i = 0;
     int32_t lo = plan[0].lo;
-    std::vector<int32_t> ids;
-    while (i < plan.size()) {
-        const int slot = (int)(ctx->in_next++ % kSlots);
-        char* sp = ctx->stage_in + (int64_t)slot * ctx->slot_bytes;
-        if (ctx->in_used[slot]) CK(cudaStreamWaitEvent(ctx->s_h2d, ctx->e_scattered[slot], 0));
+    int64_t id_off = 0;
+    while (left > 0) {
+        while (i < plan.size() && lo >= plan[i].hi) {
+            ++i;
+            if (i < plan.size()) lo = plan[i].lo;
+        }
+        const int64_t n_c = std::min(cap, left);
+        const int64_t bytes = g * n_c * Bl;
+        if (ctx->in_slot < 0 || ctx->in_fill + bytes > ctx->slot_bytes) {
+            ctx->in_slot = (int)(ctx->in_next++ % kSlots);
+            ctx->in_fill = 0;
+            if (ctx->in_used[ctx->in_slot]) CK(cudaStreamWaitEvent(ctx->s_h2d, ctx->e_scattered[ctx->in_slot], 0));
+        }
+        const int slot = ctx->in_slot;
+        char* sp = ctx->stage_in + (int64_t)slot * ctx->slot_bytes + ctx->in_fill;
+        ctx->in_fill += bytes;
         int64_t used = 0;
-        ids.clear();
-        while (i < plan.size() && used < cap) {
+        while (used < n_c) {
             Req& r = ctx->reqs[plan[i].req];
-            const int64_t take = std::min<int64_t>(plan[i].hi - lo, cap - used);
-            // one contiguous host range per (segment, layer): a run of blocks is cut at segment borders
+            const int64_t take = std::min<int64_t>(plan[i].hi - lo, n_c - used);
+            if (take <= 0) {  // an empty range in the plan
+                ++i;
+                lo = plan[i].lo;
+                continue;
+            }
+            // a run of blocks is cut at the borders of the image's segments
             for (int64_t j = lo, done = 0; done < take;) {
                 const Req::Seg* sg = nullptr;
                 for (const Req::Seg& c : r.segs)
                     if (j >= c.lo && j < c.hi) sg = &c;
                 if (sg == nullptr) return ctx->fail(PS_ERR_STATE, "reload: block outside the host image");
                 const int64_t piece = std::min<int64_t>(take - done, sg->hi - j);
-                const char* src = ctx->host_pool + sg->off + ((int64_t)layer * (sg->hi - sg->lo) + (j - sg->lo)) * Bl;
-                ProfScope prof(ctx, kProfH2D, ctx->s_h2d, piece * Bl, layer);
-                CK(cudaMemcpyAsync(sp + (used + done) * Bl, src, (size_t)(piece * Bl), cudaMemcpyHostToDevice, ctx->s_h2d));
+                const int64_t seg_pitch = (int64_t)(sg->hi - sg->lo) * Bl;  // bytes between layers in the image
+                const char* src = ctx->host_pool + sg->off + (int64_t)l0 * seg_pitch + (j - sg->lo) * Bl;
+                char* dst = sp + (used + done) * Bl;
+                ProfScope prof(ctx, kProfH2D, ctx->s_h2d, g * piece * Bl, l0);
+                if (g == 1) {
+                    CK(cudaMemcpyAsync(dst, src, (size_t)(piece * Bl), cudaMemcpyHostToDevice, ctx->s_h2d));
+                } else if (seg_pitch <= ctx->max_pitch && n_c * Bl <= ctx->max_pitch) {
+                    CK(cudaMemcpy2DAsync(dst, (size_t)(n_c * Bl), src, (size_t)seg_pitch, (size_t)(piece * Bl), (size_t)g,
+                                         cudaMemcpyHostToDevice, ctx->s_h2d));
+                } else {
+                    for (int32_t l = 0; l < g; ++l)
+                        CK(cudaMemcpyAsync(dst + l * n_c * Bl, src + l * seg_pitch, (size_t)(piece * Bl),
+                                           cudaMemcpyHostToDevice, ctx->s_h2d));
+                }
                 j += piece;
                 done += piece;
             }
-            for (int64_t j = lo; j < lo + take; ++j) ids.push_back(r.table[(size_t)j]);
             used += take;
             lo += (int32_t)take;
-            if (lo >= plan[i].hi) {
+            if (lo >= plan[i].hi && used < n_c) {
                 ++i;
-                if (i < plan.size()) lo = plan[i].lo;
+                lo = plan[i].lo;
             }
         }
         CK(cudaEventRecord(ctx->e_loaded[slot], ctx->s_h2d));
         CK(cudaStreamWaitEvent(ctx->s_scatter, ctx->e_loaded[slot], 0));
-        for (size_t c0 = 0; c0 < ids.size(); c0 += ps::kMaxParamIds) {
-            const int32_t n = (int32_t)std::min<size_t>(ps::kMaxParamIds, ids.size() - c0);
-            ProfScope prof(ctx, kProfScatter, ctx->s_scatter, (int64_t)n * Bl, layer);
-            CK(ps::launch_scatter_layer_ids(ctx->kpools[layer], ctx->vpools[layer], ids.data() + c0, n,
-                                            sp + (int64_t)c0 * Bl, ctx->slab_vec, ctx->cfg.num_gpu_blocks,
-                                            ctx->d_status, ctx->s_scatter));
+        {
+            ProfScope prof(ctx, kProfScatter, ctx->s_scatter, bytes, l0);
+            CK(ps::launch_image_copy(/*scatter=*/true, ctx->d_kpools, ctx->d_vpools, d_ids + id_off, (int32_t)n_c, l0, 0,
+                                     2 * n_c * g, sp, ctx->slab_vec, ctx->cfg.num_gpu_blocks, ctx->d_status,
+                                     ctx->s_scatter));
             ctx->launches++;
         }
         CK(cudaEventRecord(ctx->e_scattered[slot], ctx->s_scatter));
         ctx->in_used[slot] = true;
+        id_off += n_c;
+        left -= n_c;
     }
-    CK(cudaEventRecord(ctx->ev_in[layer], ctx->s_scatter));
+    CK(cudaEventRecord(ctx->ev_in[(size_t)l0], ctx->s_scatter));
+    for (int32_t l = l0; l < l0 + g; ++l) ctx->ev_of_layer[(size_t)l] = l0;
     return PS_OK;
 }
 
@@ -139,8 +203,16 @@ int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi) {
             return rc;
         }
         memcpy(ctx->a_gather.h + toff, r.table.data() + lo, (size_t)n_blk * 4);
+        // On a failure after the first copy into the range was enqueued, the range must not be handed out
+        // again before those copies have ended: it is parked behind a ticket of the D2H stream.
+        bool copies_enqueued = false;
         auto bail = [&](cudaError_t ce, const char* what) {
-            ctx->hpool.release(off, bytes);
+            uint64_t ticket = 0;
+            if (!copies_enqueued)
+                ctx->hpool.release(off, bytes);
+            else if (tracker_mark(ctx, ctx->t_d2h, &ticket) == PS_OK)
+                ctx->host_release.push_back({ticket, {off, bytes}});
+            // (if not even the ticket could be recorded the range stays reserved: a leak, never a reuse)
             return ctx->fail_cuda(ce, what);
         };
         e = ps::launch_upload(ctx->a_gather.d + toff, ctx->a_gather.hd + toff, (size_t)round_up(n_blk * 4, 16),
@@ -159,9 +231,9 @@ int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi) {
             }
             {
                 ProfScope prof(ctx, kProfGather, ctx->s_gather, cnt * ctx->slab_bytes);
-                e = ps::launch_gather_image((const void* const*)ctx->d_kpools, (const void* const*)ctx->d_vpools,
-                                            (const int32_t*)(ctx->a_gather.d + toff), (int32_t)n_blk, s0, cnt, sp,
-                                            ctx->slab_vec, ctx->cfg.num_gpu_blocks, ctx->d_status, ctx->s_gather);
+                e = ps::launch_image_copy(/*scatter=*/false, ctx->d_kpools, ctx->d_vpools,
+                                          (const int32_t*)(ctx->a_gather.d + toff), (int32_t)n_blk, 0, s0, cnt, sp,
+                                          ctx->slab_vec, ctx->cfg.num_gpu_blocks, ctx->d_status, ctx->s_gather);
                 ctx->launches++;
             }
             if (e == cudaSuccess) e = cudaEventRecord(ctx->e_gathered[slot], ctx->s_gather);
@@ -171,6 +243,7 @@ int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi) {
                 ProfScope prof(ctx, kProfD2H, ctx->s_d2h, cnt * ctx->slab_bytes);
                 e = cudaMemcpyAsync(ctx->host_pool + off + s0 * ctx->slab_bytes, sp, (size_t)(cnt * ctx->slab_bytes),
                                     cudaMemcpyDeviceToHost, ctx->s_d2h);
+                copies_enqueued |= e == cudaSuccess;
             }
             if (e == cudaSuccess) e = cudaEventRecord(ctx->e_drained[slot], ctx->s_d2h);
             if (e != cudaSuccess) return bail(e, "device-to-host copy");
@@ -179,7 +252,11 @@ int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi) {
     }
     Req::Seg sg{lo, hi, off, bytes, 0};
     int32_t rc = tracker_mark(ctx, ctx->t_d2h, &sg.ticket);
-    if (rc != PS_OK) return rc;
+    if (rc != PS_OK) {
+        // copies into the range may be in flight and there is no ticket to wait for: the range stays
+        // reserved until ps_destroy rather than being reused under them
+        return rc;
+    }
     r.segs.push_back(sg);
     r.host_issued = hi;
     return PS_OK;
@@ -350,7 +427,11 @@ int32_t ps_swap_in_layer(ps_ctx* ctx, int64_t req, int32_t layer, int32_t blk_lo
     if (blk_hi > blk_lo) {
         int32_t rc = order_scatter_after_compute(ctx);
         if (rc != PS_OK) return rc;
-        rc = issue_reload_layer(ctx, layer, {{req, blk_lo, blk_hi}});
+        const std::vector<PlanEntry> plan{{req, blk_lo, blk_hi}};
+        const int32_t* d_ids = nullptr;
+        rc = upload_plan_ids(ctx, plan, &d_ids);
+        if (rc != PS_OK) return rc;
+        rc = issue_reload_group(ctx, layer, 1, plan, d_ids);
         if (rc != PS_OK) return rc;
     }
     return note_layer_issued(ctx, req, r, layer, blk_hi);
@@ -360,9 +441,13 @@ int32_t ps_reload_fence(ps_ctx* ctx, int32_t layer) {
     if (!ctx) return PS_ERR_INVALID;
     if (layer < -1 || layer >= ctx->cfg.num_layers) return ctx->fail(PS_ERR_INVALID, "ps_reload_fence: layer out of range");
     if (ctx->bk) return PS_OK;
-    // the layer's event was last recorded behind its most recent scatter, and the scatter stream runs in order
+    // the event of the layer's chunk was last recorded behind its most recent scatter, and the scatter stream
+    // runs in order
     const int lo = layer < 0 ? 0 : layer, hi = layer < 0 ? ctx->cfg.num_layers : layer + 1;
-    for (int l = lo; l < hi; ++l) CK(cudaStreamWaitEvent(ctx->compute, ctx->ev_in[(size_t)l], 0));
+    for (int l = lo; l < hi; ++l) {
+        if (l > lo && ctx->ev_of_layer[(size_t)l] == ctx->ev_of_layer[(size_t)l - 1]) continue;  // same layer chunk
+        CK(cudaStreamWaitEvent(ctx->compute, ctx->ev_in[(size_t)ctx->ev_of_layer[(size_t)l]], 0));
+    }
     return PS_OK;
 }
 

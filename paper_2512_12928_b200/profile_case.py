@@ -1,8 +1,12 @@
 """Small, self-contained cases of the three kernels for profilers and quick timing.
 
     python -m paper_2512_12928_b200.profile_case attn    [--iters N] [--batch B] [--ctx T] [--q-heads H] [--kv-heads H] [--simt | --rows]
-    python -m paper_2512_12928_b200.profile_case gather  [--iters N] [--blocks K]
-    python -m paper_2512_12928_b200.profile_case scatter [--iters N] [--blocks K]
+    python -m paper_2512_12928_b200.profile_case gather  [--iters N] [--blocks K] [--layers L] [--chunk-layers G]
+    python -m paper_2512_12928_b200.profile_case scatter [--iters N] [--blocks K] [--layers L] [--chunk-layers G]
+
+gather / scatter launch the kernels of the swap path (gather_image_kernel, scatter_image_kernel) through
+ps_copy_blocks: K blocks of G consecutive layers per launch, the shape of a staging slot (large K) or of a
+reload's layer chunk under a small copy budget (small K, G > 1).
 
 The cases keep the Llama-3-8B KV shape (8 KV heads, head_dim 128, block 16) but only two layers and
 a pool of a few GiB, so that a profiler that saves and restores device memory between passes stays
@@ -31,11 +35,13 @@ def main():
     ap.add_argument("--q-heads", type=int, default=32)
     ap.add_argument("--kv-heads", type=int, default=8)
     ap.add_argument("--blocks", type=int, default=2048)
+    ap.add_argument("--layers", type=int, default=2, help="layers of the case's pools")
+    ap.add_argument("--chunk-layers", type=int, default=1, help="gather / scatter: layers moved by one launch")
     ap.add_argument("--simt", action="store_true")
     ap.add_argument("--rows", action="store_true", help="tensor-core kernel fed by per-row bulk copies")
     args = ap.parse_args()
 
-    L, Hkv, D, S = 2, args.kv_heads, 128, 16
+    L, Hkv, D, S = max(args.layers, args.chunk_layers), args.kv_heads, 128, 16
     nblk_req = (args.ctx + S - 1) // S
     nb = max(args.batch * nblk_req + 64, 2 * args.blocks + 64)
     sh = wl.KVShape(L, Hkv, args.q_heads, D, S, nb)
@@ -75,19 +81,21 @@ def main():
         direction = 0 if args.case == "gather" else 1
         ids = np.random.default_rng(2).permutation(nb)[: args.blocks].astype(np.int32)
         arr = (C.c_int32 * args.blocks)(*[int(v) for v in ids])
-        stage = torch.zeros((args.blocks, 2, S, Hkv, D), dtype=torch.bfloat16, device="cuda")
+        nl = args.chunk_layers
+        stage = torch.zeros((nl, args.blocks, 2, S, Hkv, D), dtype=torch.bfloat16, device="cuda")
         for i in range(3):
-            assert lib.lib.ps_copy_blocks(lib.h, i % L, arr, args.blocks, C.c_void_p(stage.data_ptr()), direction) == 0
+            assert lib.lib.ps_copy_blocks(lib.h, (i % (L - nl + 1)), nl, arr, args.blocks, C.c_void_p(stage.data_ptr()), direction) == 0
         torch.cuda.synchronize()
         e0.record()
         for i in range(args.iters):
-            assert lib.lib.ps_copy_blocks(lib.h, i % L, arr, args.blocks, C.c_void_p(stage.data_ptr()), direction) == 0
+            assert lib.lib.ps_copy_blocks(lib.h, (i % (L - nl + 1)), nl, arr, args.blocks, C.c_void_p(stage.data_ptr()), direction) == 0
         e1.record()
         e1.synchronize()
         ms = e0.elapsed_time(e1) / args.iters
-        payload = args.blocks * sh.layer_block_bytes
+        payload = nl * args.blocks * sh.layer_block_bytes
         res.update(us_per_launch=ms * 1e3, payload_bytes_per_launch=payload, gb_per_s_read_plus_write=2 * payload / ms / 1e6,
-                   blocks=args.blocks)
+                   blocks=args.blocks, chunk_layers=nl,
+                   kernel="gather_image_kernel" if direction == 0 else "scatter_image_kernel")
     assert lib.sync() == 0, lib.last_error()
     lib.destroy()
     print(json.dumps(res))

@@ -109,6 +109,58 @@ def test_budget_schedule_golden_through_the_library(repo_root):
             assert st["h2d_bytes"] == sum(hi - lo for _, lo, hi in want) * g["block_bytes"]
 
 
+def test_ruled_budget_schedule_golden_through_the_library(repo_root):
+    """ps_step_ruled: the partial-copy admission test applied while the budget is consumed."""
+    g = json.load(open(os.path.join(repo_root, "tests", "golden", "budget_schedule.json")))
+    sh = wl.KVShape(**g["shape"])
+    for case in g["ruled_cases"]:
+        lib, orc = make_pair(sh, None)
+        for req, n in g["queue_tokens"]:
+            assert lib.kv_alloc(req, n) == orc.kv_alloc(req, n) == B.PS_OK
+        for req, _ in g["queue_tokens"]:
+            assert lib.swap_out(req) == orc.swap_out(req) == B.PS_OK
+        assert lib.sync() == B.PS_OK
+        orc.reap()
+        for req, _ in g["queue_tokens"]:
+            assert lib.swap_in_begin(req) == orc.swap_in_begin(req) == B.PS_OK
+        ids = [r for r, _ in g["queue_tokens"]]
+        rule = {int(k): tuple(v) for k, v in case["rule"].items()}
+        rr = sorted(rule)
+        for want in case["steps"]:
+            before = {r: lib.missing_blocks(r) for r in ids}
+            rc, mask, st = lib.step_ruled(None, None, ids, case["budget_bytes"], case["beta"], rr,
+                                          [rule[r][0] for r in rr], [rule[r][1] for r in rr])
+            assert rc == B.PS_OK, lib.last_error()
+            plan, omask, _ = orc.step(case["budget_bytes"], ids, rule=rule, beta=case["beta"])
+            got = {r: before[r] - lib.missing_blocks(r) for r in ids if before[r] != lib.missing_blocks(r)}
+            assert got == {r: hi - lo for r, lo, hi in want} == {r: hi - lo for r, lo, hi in plan}
+            assert mask == omask
+            same_tables(lib, orc, ids)
+    lib, _ = make_pair(sh, None)
+    assert lib.step_ruled(None, None, [], 0, 1.0, [], [], [])[0] == B.PS_ERR_INVALID      # beta must exceed 1
+    assert lib.step_ruled(None, None, [], 0, 2.0, [1], [-1], [0])[0] == B.PS_ERR_INVALID
+
+
+def test_kernel_status_word_is_reported_with_its_own_code_and_text():
+    """What a kernel writes into the status word surfaces from the next poll: a bad block id as
+    PS_ERR_BOUNDS, a wait that ran out inside the attention kernel as PS_ERR_TIMEOUT.  The word is written
+    by a test hook: no kernel is made to fail."""
+    sh = wl.KVShape(2, 2, 4, 64, 16, 8)
+    lib, _ = make_pair(sh, None)
+    assert lib.poll() == 0
+    for value, code, text in ((1, B.PS_ERR_BOUNDS, "copy kernel"), (2, B.PS_ERR_BOUNDS, "attention kernel met"),
+                              (3, B.PS_ERR_TIMEOUT, "bounded wait")):
+        assert lib.inject_status(value) == B.PS_OK
+        with pytest.raises(B.PsError) as e:
+            lib.poll()
+        assert e.value.code == code and text in str(e.value), str(e.value)
+        assert lib.poll() == 0                      # reported once, then clear
+    assert lib.inject_status(3) == B.PS_OK
+    assert lib.step(None, None, [], 0)[0] == B.PS_ERR_TIMEOUT
+    assert lib.sync() == B.PS_OK
+    assert lib.inject_status(0) == B.PS_ERR_INVALID and lib.inject_status(4) == B.PS_ERR_INVALID
+
+
 def test_random_script_against_checker():
     """A long seeded mix of alloc / grow / free / swap-out / reap / swap-in / cancel / budgeted steps."""
     sh = wl.KVShape(3, 2, 4, 64, 8, 96)
