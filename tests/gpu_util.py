@@ -27,7 +27,7 @@ class Pair:
 
     def __init__(self, sh: wl.KVShape, free_order, K: np.ndarray, V: np.ndarray, *, max_batch=64,
                  host_pool_bytes=None, staging_bytes=0, flags=0, attn_kernel=B.PS_ATTN_AUTO, kv_split_tokens=0,
-                 max_blocks_per_req=None):
+                 max_blocks_per_req=None, layer_chunk_bytes=0):
         self.sh = sh
         self.Kd = bits_to_dev(K)           # [L][nb][S][Hkv][D]
         self.Vd = bits_to_dev(V)
@@ -40,7 +40,8 @@ class Pair:
                             host_pool_bytes=host_pool_bytes, staging_bytes=staging_bytes,
                             initial_free_order=free_order, k_pools=[self.Kd[l] for l in range(sh.num_layers)],
                             v_pools=[self.Vd[l] for l in range(sh.num_layers)], flags=flags,
-                            attn_kernel=attn_kernel, kv_split_tokens=kv_split_tokens)
+                            attn_kernel=attn_kernel, kv_split_tokens=kv_split_tokens,
+                            layer_chunk_bytes=layer_chunk_bytes)
         self.orc = po.PsOracle(sh.num_layers, sh.num_kv_heads, sh.num_q_heads, sh.head_dim, sh.block_size,
                                sh.num_gpu_blocks, free_order, K.copy(), V.copy())
 
