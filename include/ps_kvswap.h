@@ -532,6 +532,13 @@ int32_t ps_trace_read(ps_ctx* ctx, ps_trace_span* out, int32_t cap, int32_t* n);
  * Allocates and frees its own buffers; needs no context. */
 int32_t ps_link_probe(int64_t bytes, int32_t direction, int32_t iters, double* gb_per_s);
 
+/* Device-memory bandwidth probe with a plain streaming kernel of this library: best of `iters` passes over
+ * `bytes` (a multiple of 16, at least 1 MiB; use more than the L2 holds), timed with CUDA events on the default
+ * stream.  mode 0 = read only (the traffic pattern of decode attention: KV is read, almost nothing written),
+ * mode 1 = copy (bytes read + bytes written are counted, the accounting of a gather or scatter).  *gb_per_s in
+ * 1e9 bytes/s.  Allocates and frees its own buffers; needs no context. */
+int32_t ps_hbm_probe(int64_t bytes, int32_t mode, int32_t iters, double* gb_per_s);
+
 /* The gather kernel of ps_swap_out (direction 0: pools -> staging) or the scatter kernel of ps_swap_in_layer /
  * ps_step (direction 1: staging -> pools) alone, without any host transfer, on the compute stream: the same
  * kernels in the launch shape the swap path gives them, for measuring them against HBM bandwidth.  One launch

@@ -32,7 +32,7 @@ EXPORTS = [
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
     "ps_decode_attn_static", "ps_copy_budget", "ps_offload_progress", "ps_host_blocks", "ps_host_segment",
     "ps_select_victims", "ps_copy_condition", "ps_order_queue", "ps_estimate_batch", "ps_resume_cost",
-    "ps_reload_fence", "ps_offload_sweep", "ps_step_ruled", "ps_step_host", "ps_inject_status",
+    "ps_reload_fence", "ps_offload_sweep", "ps_step_ruled", "ps_step_host", "ps_inject_status", "ps_hbm_probe",
 ]
 
 
@@ -141,6 +141,7 @@ def load() -> C.CDLL:
         "ps_launch_count": (i32, [vp, p64]),
         "ps_get_profile": (i32, [vp, C.POINTER(PsProfile), i32]),
         "ps_link_probe": (i32, [i64, i32, i32, C.POINTER(C.c_double)]),
+        "ps_hbm_probe": (i32, [i64, i32, i32, C.POINTER(C.c_double)]),
         "ps_copy_blocks": (i32, [vp, i32, i32, p32, i32, vp, i32]),
         "ps_inject_status": (i32, [vp, i32]),
         "ps_step_ruled": (i32, [vp, vp, vp, p64, i32, i64, C.POINTER(PsCopyRule), p32, C.POINTER(PsStepStats)]),
@@ -176,6 +177,15 @@ def ps_link_probe(nbytes: int, direction: int, iters: int = 10) -> float:
     rc = load().ps_link_probe(nbytes, direction, iters, C.byref(out))
     if rc != PS_OK:
         raise PsError(rc, "ps_link_probe", load().ps_last_error(None).decode())
+    return out.value
+
+
+def ps_hbm_probe(nbytes: int, mode: int, iters: int = 5) -> float:
+    """Device-memory rate of a plain streaming kernel in GB/s (1e9): 0 = read only, 1 = copy (read + written)."""
+    out = C.c_double(0.0)
+    rc = load().ps_hbm_probe(nbytes, mode, iters, C.byref(out))
+    if rc != PS_OK:
+        raise PsError(rc, "ps_hbm_probe", load().ps_last_error(None).decode())
     return out.value
 
 

@@ -125,3 +125,47 @@ cudaError_t launch_upload(void* dst, const void* src_mapped, size_t bytes, cudaS
 }
 
 }  // namespace ps
+
+// ---- plain streaming kernels for the bandwidth probe -------------------------------------------------
+namespace ps {
+namespace {
+
+// Every thread streams 16-byte vectors with a grid stride, four loads in flight, and folds them into one
+// word that is stored at the end (so the loads cannot be dropped).  kCopy also stores every vector.
+template <bool kCopy>
+__global__ void __launch_bounds__(256)
+stream_probe_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, int64_t n_vec, uint32_t* __restrict__ sink) {
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t acc = 0;
+    for (; i + 3 * stride < n_vec; i += 4 * stride) {
+        uint4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) v[u] = ld_stream(src + i + u * stride);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (kCopy) dst[i + u * stride] = v[u];
+            acc ^= v[u].x ^ v[u].y ^ v[u].z ^ v[u].w;
+        }
+    }
+    for (; i < n_vec; i += stride) {
+        const uint4 v = ld_stream(src + i);
+        if (kCopy) dst[i] = v;
+        acc ^= v.x ^ v.y ^ v.z ^ v.w;
+    }
+    if (!kCopy) sink[(int64_t)blockIdx.x * blockDim.x + threadIdx.x] = acc;
+}
+
+}  // namespace
+
+cudaError_t launch_stream_probe(bool copy, const void* src, void* dst, int64_t bytes, uint32_t* sink, int32_t ctas,
+                                cudaStream_t stream) {
+    if (bytes <= 0 || bytes % 16 || ctas <= 0) return cudaErrorInvalidValue;
+    if (copy)
+        stream_probe_kernel<true><<<(unsigned)ctas, 256, 0, stream>>>((const uint4*)src, (uint4*)dst, bytes / 16, sink);
+    else
+        stream_probe_kernel<false><<<(unsigned)ctas, 256, 0, stream>>>((const uint4*)src, (uint4*)dst, bytes / 16, sink);
+    return cudaGetLastError();
+}
+
+}  // namespace ps

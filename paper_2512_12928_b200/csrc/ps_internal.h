@@ -25,6 +25,11 @@ cudaError_t launch_image_copy(bool scatter, void* const* d_kpools, void* const* 
 // copy engine.
 cudaError_t launch_upload(void* dst, const void* src_mapped, size_t bytes, cudaStream_t stream);
 
+// Streams `bytes` (a multiple of 16) of src with `ctas` CTAs of 256 threads: read-only (every thread folds what
+// it read into one word of sink, which holds ctas * 256 words) or as a copy into dst.  For the bandwidth probe.
+cudaError_t launch_stream_probe(bool copy, const void* src, void* dst, int64_t bytes, uint32_t* sink, int32_t ctas,
+                                cudaStream_t stream);
+
 // ---- paged decode attention --------------------------------------------------------------------
 
 // One split-KV work item: tokens [t_begin, t_end) of batch row b.  `part` indexes the partial

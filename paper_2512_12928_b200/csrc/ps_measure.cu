@@ -55,6 +55,54 @@ int32_t ps_inject_status(ps_ctx* ctx, int32_t value) {
     return PS_OK;
 }
 
+int32_t ps_hbm_probe(int64_t bytes, int32_t mode, int32_t iters, double* gb_per_s) {
+    if (bytes < (1 << 20) || bytes % 16 || iters <= 0 || !gb_per_s || mode < 0 || mode > 1) return PS_ERR_INVALID;
+    void *src = nullptr, *dst = nullptr;
+    uint32_t* sink = nullptr;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    int32_t rc = PS_OK;
+    double best = 0.0;
+    int dev = 0, sms = 0;
+#define CKP(call)                        \
+    do {                                 \
+        if ((call) != cudaSuccess) {     \
+            rc = PS_ERR_CUDA;            \
+            create_error() = #call;      \
+            goto done;                   \
+        }                                \
+    } while (0)
+    CKP(cudaGetDevice(&dev));
+    CKP(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    {
+        const int32_t ctas = sms * 8;  // 2048 threads per SM, four 16-byte loads in flight each
+        CKP(cudaMalloc(&src, (size_t)bytes));
+        CKP(cudaMemset(src, 1, (size_t)bytes));
+        if (mode == 1) CKP(cudaMalloc(&dst, (size_t)bytes));
+        CKP(cudaMalloc((void**)&sink, (size_t)ctas * 256 * sizeof(uint32_t)));
+        CKP(cudaEventCreate(&e0));
+        CKP(cudaEventCreate(&e1));
+        for (int it = 0; it < iters + 1; ++it) {  // first pass warms up
+            CKP(cudaEventRecord(e0, 0));
+            CKP(ps::launch_stream_probe(mode == 1, src, dst, bytes, sink, ctas, 0));
+            CKP(cudaEventRecord(e1, 0));
+            CKP(cudaEventSynchronize(e1));
+            float ms = 0.f;
+            CKP(cudaEventElapsedTime(&ms, e0, e1));
+            if (it > 0 && ms > 0.f) best = std::max(best, (mode == 1 ? 2.0 : 1.0) * (double)bytes / (ms * 1e-3) / 1e9);
+        }
+        *gb_per_s = best;
+    }
+done:
+#undef CKP
+    if (e0) cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (src) cudaFree(src);
+    if (dst) cudaFree(dst);
+    if (sink) cudaFree(sink);
+    cudaGetLastError();
+    return rc;
+}
+
 int32_t ps_link_probe(int64_t bytes, int32_t direction, int32_t iters, double* gb_per_s) {
     if (bytes <= 0 || iters <= 0 || !gb_per_s || direction < 0 || direction > 2) return PS_ERR_INVALID;
     void *h0 = nullptr, *h1 = nullptr, *d0 = nullptr, *d1 = nullptr;
