@@ -156,8 +156,8 @@ def oracle_swap_pass(n_req: int = 4, ctx: int = 2048, seed: int = 0):
     sh = wl.KVShape(32, 8, 32, 128, 16, n_req * (ctx // 16) + 64)
     rng = np.random.default_rng(seed)
     dims = (sh.num_layers, sh.num_gpu_blocks, sh.block_size, sh.num_kv_heads, sh.head_dim)
-    K = rng.integers(0, 65536, size=dims, dtype=np.uint16)
-    V = rng.integers(0, 65536, size=dims, dtype=np.uint16)
+    K = wl.randn_bf16_bits(rng, dims)              # N(0,1) as bf16, like every other input
+    V = wl.randn_bf16_bits(rng, dims)
     orc = po.PsOracle(sh.num_layers, sh.num_kv_heads, sh.num_q_heads, sh.head_dim, sh.block_size,
                       sh.num_gpu_blocks, rng.permutation(sh.num_gpu_blocks), K, V)
     grown = 0
@@ -177,7 +177,33 @@ def oracle_swap_pass(n_req: int = 4, ctx: int = 2048, seed: int = 0):
     return one_pass, nbytes, orc, sh
 
 
-def time_oracle(target_s: float = 10.0):
+def oracle_attention_step(step_layers: int, step_tokens: int, n_layers: int = 2, n_req: int = 8, ctx: int = 2048):
+    """The checker's fp64 decode attention on n_layers x n_req requests of ctx tokens (8B KV shape, 32 query
+    heads), and its linear extrapolation to a whole decode step of step_layers layers over step_tokens KV tokens
+    (attention is linear in both).  NumPy's BLAS may use every host core the process is allowed."""
+    from oracle import ps_oracle as po
+    sh = wl.KVShape(n_layers, 8, 32, 128, 16, n_req * (ctx // 16) + 16)
+    rng = np.random.default_rng(2)
+    dims = (sh.num_layers, sh.num_gpu_blocks, sh.block_size, sh.num_kv_heads, sh.head_dim)
+    orc = po.PsOracle(sh.num_layers, sh.num_kv_heads, sh.num_q_heads, sh.head_dim, sh.block_size, sh.num_gpu_blocks,
+                      rng.permutation(sh.num_gpu_blocks), wl.randn_bf16_bits(rng, dims), wl.randn_bf16_bits(rng, dims))
+    for r in range(n_req):
+        assert orc.kv_alloc(r, ctx) == 0
+    q = wl.randn_bf16_bits(rng, (n_layers, n_req, sh.num_q_heads, sh.head_dim))
+    reqs = list(range(n_req))
+    t0 = time.perf_counter()
+    for l in range(n_layers):
+        orc.decode_attn(l, q[l], reqs)
+    sample_s = time.perf_counter() - t0
+    scale = (step_layers / n_layers) * (step_tokens / (n_req * ctx))
+    return {"attn_sample_s": sample_s,
+            "attn_sample": f"fp64 decode attention, {n_layers} layers x {n_req} requests x {ctx} tokens x 32 query heads",
+            "attn_step_s_extrapolated": sample_s * scale,
+            "attn_step_extrapolation": f"sample x ({step_layers} / {n_layers} layers) x ({step_tokens} / {n_req * ctx} KV "
+                                       f"tokens) = x {scale:.1f}: one decode step of the bench's 64 requests"}
+
+
+def time_oracle(target_s: float = 10.0, step_layers: int = 32, step_tokens: int = 0):
     one_pass, nbytes, orc, sh = oracle_swap_pass()
     one_pass()                                   # touch the pages once
     t0 = time.perf_counter()
@@ -188,19 +214,17 @@ def time_oracle(target_s: float = 10.0):
         if time.perf_counter() - t0 >= target_s:
             break
     dt = time.perf_counter() - t0
-    # a small attention sample for context (fp64 checker, 4 requests x 1 layer)
-    q = wl.randn_bf16_bits(np.random.default_rng(1), (4, sh.num_q_heads, sh.head_dim))
-    t1 = time.perf_counter()
-    orc.decode_attn(0, q, [0, 1, 2, 3])
-    attn_s = time.perf_counter() - t1
-    return {
+    del orc
+    cores = len(os.sched_getaffinity(0))
+    res = {
         "value": n * nbytes / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
         "sample": f"{n} passes of swap-out + reap + unbudgeted swap-in of 4 requests x 2048 tokens "
                   f"(8B KV shape, {nbytes / 2**30:.2f} GiB moved per pass) in {dt:.1f} s, single thread",
-        "attn_sample_s": attn_s,
-        "attn_sample": "fp64 decode attention, 1 layer x 4 requests x 2048 tokens x 32 query heads",
-        "host_cores_available": len(os.sched_getaffinity(0)),
+        "host_cores_available": cores, "attn_blas_threads_allowed": cores,
     }
+    if step_tokens > 0:
+        res.update(oracle_attention_step(step_layers, step_tokens))
+    return res
 
 
 def run_reference(args):
@@ -269,13 +293,14 @@ def swap_workload_step(torch, B, lib, w, q, out, q_res, out_res, budget, e2e_buf
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
 
     def decode(reqs, qq, oo, bud):
-        if e2e_bufs is not None:                     # end-to-end: queries come from pinned host memory each step
-            qq.copy_(sub_batch(e2e_bufs["q_host"], qq.shape[1]), non_blocking=True)
-        rc, mask, st = lib.step(qq, oo, reqs, bud)
+        if e2e_bufs is not None:
+            # end-to-end: queries and outputs live in pinned HOST memory; ps_step_host makes both copies
+            qh, oh = e2e_bufs[qq.shape[1]]
+            rc, mask, st = lib.step_host(qh, oh, reqs, bud)
+        else:
+            rc, mask, st = lib.step(qq, oo, reqs, bud)
         if rc != 0:
             raise RuntimeError(f"ps_step: {rc} {lib.last_error()}")
-        if e2e_bufs is not None:                     # ... and the step's result goes back to the host
-            sub_batch(e2e_bufs["out_host"], oo.shape[1]).copy_(oo, non_blocking=True)
         stream.synchronize()                         # an engine reads the step's result before the next step
         return mask, st
 
@@ -378,6 +403,8 @@ def overlap_sweep(torch, B, K, V, peaks_hbm, w=None, label=None, pipelined_budge
         sync_budgets = [256 * wl.MiB, -1]
     for mode in ("pipelined", "sync_reload"):
         flags = B.PS_FLAG_SYNC_RELOAD if mode == "sync_reload" else 0
+        if not (pipelined_budgets if mode == "pipelined" else sync_budgets):
+            continue
         lib = make_ctx(B, w, K, V, nb, max_batch=len(w.ctx_lens), host_pool_bytes=host_bytes, flags=flags)
         for r, n in wl.build_order_round_robin(w):
             assert lib.kv_alloc(r, n) == 0, lib.last_error()
@@ -404,6 +431,10 @@ def overlap_sweep(torch, B, K, V, peaks_hbm, w=None, label=None, pipelined_budge
             link_gbs = B.ps_link_probe(256 << 20, 0, 5)
             model = {"a_d": rf["step_us"] / sum(w.ctx_lens[r] for r in batch), "b_d": 0.0, "t_c": 0.0,
                      "t_block": sh.block_bytes / (link_gbs * 1e3) * (1.0 + 1.0 / sh.num_layers), "t_budget": 1e12}
+            # the largest budget whose transfer fits under a decode step: link rate x step time, less the
+            # first layer chunk, which nothing can hide
+            res["hideable_budget_mib"] = link_gbs * 1e3 * rf["step_us"] * (1.0 - 1.0 / sh.num_layers) / wl.MiB
+            res["link_h2d_gbs_256mib_probe"] = link_gbs
             res["adaptive_model"] = dict(model, note="a_d: measured decode step us per KV token; t_block: block bytes / "
                                          "measured H2D rate, plus one layer chunk of pipeline fill")
         if mode == "pipelined":
@@ -433,6 +464,22 @@ def overlap_sweep(torch, B, K, V, peaks_hbm, w=None, label=None, pipelined_budge
                 rc, _, _ = lib.step(None, None, [], step_budget(all_reqs))
                 assert rc == 0, lib.last_error()
                 assert lib.sync() == 0
+            e1.record(); e1.synchronize()
+            alone_stepwise_ms = e0.elapsed_time(e1)
+            chosen.clear()
+            for r in w.victims:
+                assert lib.swap_out(r) == 0
+            assert lib.sync() == 0
+            # (1b) the same steps issued back to back, one wait at the end: the transfer without a host round
+            # trip per step (the denominator of the hidden fraction)
+            for r in w.victims:
+                assert lib.swap_in_begin(r) == 0
+            torch.cuda.synchronize()
+            e0.record()
+            while any(lib.missing_blocks(r) for r in w.victims):
+                rc, _, _ = lib.step(None, None, [], step_budget(all_reqs))
+                assert rc == 0, lib.last_error()
+            assert lib.sync() == 0
             e1.record(); e1.synchronize()
             alone_ms = e0.elapsed_time(e1)
             chosen.clear()
@@ -476,6 +523,10 @@ def overlap_sweep(torch, B, K, V, peaks_hbm, w=None, label=None, pipelined_budge
             res[key] = {"steps": n_steps, "step_us_with_reload": with_ms / n_steps * 1e3,
                         "step_us_no_reload": without_ms / n_steps * 1e3,
                         "reload_alone_ms": alone_ms, "reload_alone_gbs": reload_bytes / alone_ms / 1e6,
+                        "reload_alone_stepwise_ms": alone_stepwise_ms,
+                        "reload_alone_stepwise_gbs": reload_bytes / alone_stepwise_ms / 1e6,
+                        "hidden_frac_vs_stepwise": (1.0 - max(0.0, with_ms - without_ms) / alone_stepwise_ms)
+                        if alone_stepwise_ms > 0 else None,
                         "reload_under_decode_gbs": reload_bytes / with_ms / 1e6, "hidden_frac": hidden}
             if budget == "adaptive":
                 res[key]["chosen_budget_mib_per_step"] = [round(c / wl.MiB, 1) for c in chosen]
@@ -596,41 +647,49 @@ def proactive_offload_leg(torch, B, lib, w, n_off=16):
             "background_copy_ms": background_ms}
 
 
-def kernel_rates(torch, B, lib, sh, nb, n_blocks=2048, iters=20):
-    """Gather / scatter kernels alone (no host link): payload read once + written once per launch.
-
-    The launches are enqueued back to back (the ids are marshalled once), so the GPU never waits for the
-    host; the time per launch includes the small upload kernel that carries the ids."""
+def kernel_rates(torch, B, lib, sh, nb, hbm_peak, iters=20):
+    """The swap path's own kernels alone (no host link), in the launch shapes the path gives them: payload read
+    once + written once per launch.  gather_image_kernel at the size of a staging slot (64 MiB over 8 layers
+    of a request), scatter_image_kernel at the layer chunks ps_step issues for 16 / 64 / 256 MiB per step and
+    for an unlimited budget.  Launches are enqueued back to back (the ids are uploaded once)."""
     import ctypes as C
     rng = np.random.default_rng(3)
-    ids = (C.c_int32 * n_blocks)(*[int(v) for v in rng.permutation(nb)[:n_blocks]])
-    stage = torch.empty((n_blocks, 2, sh.block_size, sh.num_kv_heads, sh.head_dim), dtype=torch.bfloat16, device="cuda")
+    Bl = sh.layer_block_bytes
+    cases = [("gather_slot_64mib", 0, 128, 8), ("scatter_slot_64mib", 1, 1024, 1),
+             ("scatter_chunk_256mib_step", 1, 256 * wl.MiB // sh.block_bytes, 1),
+             ("scatter_chunk_64mib_step", 1, 64 * wl.MiB // sh.block_bytes, 1),
+             ("scatter_chunk_16mib_step", 1, 16 * wl.MiB // sh.block_bytes, 4)]
     res = {}
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    payload = n_blocks * sh.layer_block_bytes
+    for name, direction, n_blocks, n_layers in cases:          # scatters overwrite pool blocks: the caller runs this last
+        ids = (C.c_int32 * n_blocks)(*[int(v) for v in rng.permutation(nb)[:n_blocks]])
+        stage = torch.empty((n_layers, n_blocks, 2, sh.block_size, sh.num_kv_heads, sh.head_dim), dtype=torch.bfloat16,
+                            device="cuda")
+        payload = n_layers * n_blocks * Bl
 
-    def launch(i, direction):
-        rc = lib.lib.ps_copy_blocks(lib.h, i % sh.num_layers, 1, ids, n_blocks, C.c_void_p(stage.data_ptr()), direction)
-        assert rc == 0, lib.last_error()
+        def launch(i):
+            rc = lib.lib.ps_copy_blocks(lib.h, (i * n_layers) % (sh.num_layers - n_layers + 1), n_layers, ids, n_blocks,
+                                        C.c_void_p(stage.data_ptr()), direction)
+            assert rc == 0, lib.last_error()
 
-    for name, direction in (("gather", 0), ("scatter", 1)):   # the scatter overwrites pool blocks: run last
         for i in range(3):
-            launch(i, direction)
+            launch(i)
         torch.cuda.synchronize()
         e0.record()
         for i in range(iters):
-            launch(i, direction)
+            launch(i)
         e1.record(); e1.synchronize()
         ms = e0.elapsed_time(e1) / iters
-        res[name + "_gbs_rw"] = 2 * payload / ms / 1e6
-        res[name + "_us"] = ms * 1e3
-    res["blocks_per_launch"] = n_blocks
-    res["payload_bytes_per_launch"] = payload
+        res[name] = {"kernel": "gather_image_kernel" if direction == 0 else "scatter_image_kernel",
+                     "blocks": n_blocks, "layers": n_layers, "payload_bytes_per_launch": payload,
+                     "us_per_launch": ms * 1e3, "gbs_rw": 2 * payload / ms / 1e6,
+                     "frac_of_hbm": 2 * payload / ms / 1e6 / hbm_peak}
+        del stage
     res["launches_timed"] = iters
     return res
 
 
-def long_context_leg(torch, B, hbm_peak):
+def long_context_leg(torch, B, hbm_peak, compact=False):
     """70B-shaped KV (80 layers, block 32): decode batch 64 x 4096 tokens, one 32k-token request (10 GiB) offloaded
     under decode and reloaded layer-pipelined across steps."""
     w = wl.long_context()
@@ -639,7 +698,8 @@ def long_context_leg(torch, B, hbm_peak):
     torch.cuda.synchronize()
     res = overlap_sweep(torch, B, K, V, hbm_peak, w=w,
                         label="long_context: decode batch 64 x 4096 tokens, one 32768-token request of 10 GiB",
-                        pipelined_budgets=[256 * wl.MiB, "adaptive", -1], sync_budgets=[256 * wl.MiB])
+                        pipelined_budgets=[256 * wl.MiB, "adaptive"] if compact else [256 * wl.MiB, "adaptive", -1],
+                        sync_budgets=[] if compact else [256 * wl.MiB])
     del K, V
     return res
 
@@ -798,6 +858,8 @@ def run_gpu(args):
 
     rank, world, local_rank = replicas.env()
     torch.cuda.set_device(local_rank)
+    if world > 1:
+        replicas.bind_near_gpu(local_rank)           # pinned host pools from the memory nearest to this GPU's link
     group = replicas.Group("nccl", torch.device("cuda", local_rank))
     if rank == 0:
         ps_build.build()
@@ -825,10 +887,12 @@ def run_gpu(args):
                     dtype=torch.float32).to(torch.bfloat16)
     out = torch.zeros_like(q)
     budget = args.budget_mib * wl.MiB if args.budget_mib >= 0 else -1
-    e2e_bufs = {"q_host": q.cpu().pin_memory(), "out_host": torch.zeros_like(q, device="cpu").pin_memory()}
     n_res = nreq - len(w.victims)
     q_res = sub_batch(q, n_res).clone()
     out_res = torch.zeros_like(q_res)
+    # end-to-end arm: queries and outputs in pinned host memory, one pair of buffers per batch size
+    e2e_bufs = {nreq: (q.cpu().pin_memory(), torch.zeros_like(q, device="cpu").pin_memory()),
+                n_res: (q_res.cpu().pin_memory(), torch.zeros_like(q_res, device="cpu").pin_memory())}
 
     def fresh_ctx(flags):
         lib = make_ctx(B, w, K, V, sh.num_gpu_blocks, max_batch=nreq, host_pool_bytes=victim_bytes + (256 << 20),
@@ -871,18 +935,20 @@ def run_gpu(args):
     rf_single = single_launch_rate(torch, lib, sh, w.ctx_lens, all_reqs, q, out)
     clocks = sampler.stop()
 
-    # ---- end-to-end arm: queries from pinned host memory and outputs back to it, every decode step
+    # ---- end-to-end arm: the same pass through ps_step_host (host buffers in, host buffers out)
     e2e_recs = [swap_workload_step(torch, B, lib, w, q, out, q_res, out_res, budget, e2e_bufs)
                 for _ in range(max(1, min(args.steps, 2)))]
     e2e_ms = sum(r["out_ms"] + r["in_ms"] for r in e2e_recs)
-    e2e_steps = sum(r["steps_out"] + r["steps_in"] for r in e2e_recs) / len(e2e_recs)
     (e2e_ms,) = group.max_over_ranks([e2e_ms])
-    q_bytes = q.numel() * 2
+    row_bytes = sh.num_layers * sh.num_q_heads * sh.head_dim * 2
+    io_bytes = sum(r["steps_out"] * n_res + r["steps_in"] * nreq for r in e2e_recs) * row_bytes / len(e2e_recs)
     e2e = {"value": 2 * victim_bytes * len(e2e_recs) * world / e2e_ms / 1e6, "unit": UNIT,
-           "h2d_bytes_per_step": int(victim_bytes + e2e_steps * q_bytes),
-           "d2h_bytes_per_step": int(victim_bytes + e2e_steps * q_bytes),
-           "note": "host images live in pinned host memory by definition; this arm adds the per-decode-step "
-                   "upload of the queries from pinned host memory and the download of the attention output"}
+           "h2d_bytes_per_step": int(victim_bytes + io_bytes), "d2h_bytes_per_step": int(victim_bytes + io_bytes),
+           "api": "ps_step_host: queries from and outputs to pinned host memory through the C ABI, every decode step",
+           "decode_steps_per_pass": sum(r["steps_out"] + r["steps_in"] for r in e2e_recs) / len(e2e_recs),
+           "note": "bytes per step = the swapped KV each way (host images live in pinned host memory by "
+                   "definition) + the queries (up) / outputs (down) of every decode step: 48 rows while the "
+                   "offload drains, 64 rows in the reload step"}
 
     result = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -897,8 +963,11 @@ def run_gpu(args):
         "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches),
         "wall_ms": wall_ms,
     }
+    flat = {}                                        # scalars that go into the roofline object (see below)
     if rank == 0:
         ratio = read_traffic_ratio()
+        read_peak = B.ps_hbm_probe(4 << 30, 0, 5)
+        copy_peak = B.ps_hbm_probe(2 << 30, 1, 5)
         result["roofline"] = {
             "kernel": "decode_attn_mma_kernel (paged GQA decode attention, split-KV combined in the kernel)",
             "bound": "hbm", "achieved": rf_all["gbs"], "peak": hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth",
@@ -906,15 +975,17 @@ def run_gpu(args):
             "traffic": ratio * rf_all["algorithmic_bytes_per_launch"] if ratio else None,
             "algorithmic_bytes_per_launch": rf_all["algorithmic_bytes_per_launch"],
             "us_per_launch": rf_all["us_per_layer"], "launches_per_layer": rf_all["launches_per_layer"],
-            "how": "CUDA events around 5 decode-only steps (32 launches each, all 64 requests) on the compute "
-                   "stream, as ps_step issues them: the queries of all layers are inputs, so the launches of "
-                   "consecutive layers are independent and overlap head to tail (programmatic dependent launch)",
-            "single_launch": {"gbs": rf_single["gbs"], "us_per_launch": rf_single["us_per_launch"],
-                              "frac": rf_single["gbs"] / hbm_peak,
-                              "how": "ps_decode_attn, one layer per call, back to back, no overlap between layers"},
+            "how": "CUDA events around 5 decode-only ps_step calls (32 launches each, 64 requests); launches of "
+                   "consecutive layers overlap head to tail",
             "frac_of_nominal_8TBs": rf_all["gbs"] / 8000.0,
-            "batch_of_48_residents": {"gbs": rf_res["gbs"], "us_per_launch": rf_res["us_per_layer"],
-                                      "frac": rf_res["gbs"] / hbm_peak},
+            # the kernel only reads: a read-only stream of this library's probe kernel, measured in this run,
+            # is the like-for-like ceiling (the copy peak counts read + written bytes)
+            "read_peak_gbs": read_peak, "frac_of_read_peak": rf_all["gbs"] / read_peak,
+            "probe_copy_peak_gbs": copy_peak,
+            "single_launch_gbs": rf_single["gbs"], "single_launch_us": rf_single["us_per_launch"],
+            "single_launch_frac": rf_single["gbs"] / hbm_peak,
+            "single_launch_frac_of_read_peak": rf_single["gbs"] / read_peak,
+            "residents48_gbs": rf_res["gbs"], "residents48_us_per_launch": rf_res["us_per_layer"],
         }
         result["swap"] = {
             "swap_out_gbs": victim_bytes * args.steps / out_ms / 1e6, "swap_in_gbs": victim_bytes * args.steps / in_ms / 1e6,
@@ -925,13 +996,27 @@ def run_gpu(args):
             "decode_step_us_no_swap": rf_res["step_us"],
             "link": link,
         }
-    if rank == 0:
+        sw = result["swap"]
+        flat.update({"swap_out_gbs": sw["swap_out_gbs"], "swap_in_gbs": sw["swap_in_gbs"],
+                     "swap_out_frac_of_link": sw["swap_out_frac_of_link"],
+                     "swap_in_frac_of_link": sw["swap_in_frac_of_link"], "link_h2d_gbs": link["h2d_gbs"],
+                     "link_d2h_gbs": link["d2h_gbs"], "link_duplex_sum_gbs": link["duplex_sum_gbs"],
+                     "decode_step_us_during_swap_out": sw["decode_step_us_during_out"],
+                     "decode_step_us_no_swap_48req": sw["decode_step_us_no_swap"]})
         result["proactive_offload"] = proactive_offload_leg(torch, B, lib, w)
+        # the swap path's own gather / scatter kernels alone (the scatters overwrite pool blocks: last use of lib)
+        kr = kernel_rates(torch, B, lib, sh, sh.num_gpu_blocks, hbm_peak)
+        result["gather_scatter_alone"] = kr
+        for name, row in kr.items():
+            if isinstance(row, dict):
+                flat[name + "_gbs_rw"] = row["gbs_rw"]
+                flat[name + "_frac_of_hbm"] = row["frac_of_hbm"]
+                flat[name + "_us"] = row["us_per_launch"]
     lib.destroy()
     del lib
     if rank == 0:
         # diagnostics pass with per-launch events (not part of any reported rate above): engine and kernel
-        # rates inside a step; the events themselves slow this pass down
+        # rates inside a step, beside attention; the events themselves slow this pass down
         plib = fresh_ctx(B.PS_FLAG_PROFILE)
         swap_workload_step(torch, B, plib, w, q, out, q_res, out_res, budget)
         prof = plib.get_profile(reset=True)
@@ -940,21 +1025,58 @@ def run_gpu(args):
             "h2d_engine_gbs": prof["h2d_bytes"] / prof["h2d_ms"] / 1e6 if prof["h2d_ms"] > 0 else None,
             "gather_in_step_gbs_rw": 2 * prof["gather_bytes"] / prof["gather_ms"] / 1e6 if prof["gather_ms"] > 0 else None,
             "scatter_in_step_gbs_rw": 2 * prof["scatter_bytes"] / prof["scatter_ms"] / 1e6 if prof["scatter_ms"] > 0 else None,
+            "gather_launches": prof["gather_launches"], "scatter_launches": prof["scatter_launches"],
         })
-        kr = kernel_rates(torch, B, plib, sh, sh.num_gpu_blocks)
-        kr["gather_frac_of_hbm"] = kr["gather_gbs_rw"] / hbm_peak
-        kr["scatter_frac_of_hbm"] = kr["scatter_gbs_rw"] / hbm_peak
-        result["gather_scatter_alone"] = kr
+        flat["gather_beside_attention_gbs_rw"] = result["swap"]["gather_in_step_gbs_rw"]
+        flat["scatter_beside_attention_gbs_rw"] = result["swap"]["scatter_in_step_gbs_rw"]
         plib.destroy()
         del plib
     if rank == 0 and not args.no_overlap:
-        result["overlap"] = overlap_sweep(torch, B, K, V, hbm_peak)
+        ov = overlap_sweep(torch, B, K, V, hbm_peak)
+        result["overlap"] = ov
+        flat["overlap_attn_gbs"] = ov["attn_gbs"]
+        flat["overlap_hideable_budget_mib"] = ov["hideable_budget_mib"]
+        for key, tag in (("pipelined_16MiB", "16mib"), ("pipelined_64MiB", "64mib"), ("pipelined_256MiB", "256mib"),
+                         ("pipelined_adaptive", "adaptive"), ("pipelined_unlimited", "unlimited"),
+                         ("sync_reload_256MiB", "sync256mib")):
+            if key in ov:
+                row = ov[key]
+                flat[f"overlap_{tag}_hidden_frac"] = row["hidden_frac"]
+                flat[f"overlap_{tag}_step_us_with_reload"] = row["step_us_with_reload"]
+                flat[f"overlap_{tag}_step_us_no_reload"] = row["step_us_no_reload"]
+                flat[f"overlap_{tag}_reload_alone_gbs"] = row["reload_alone_gbs"]
+                flat[f"overlap_{tag}_reload_alone_frac_of_link"] = row["reload_alone_gbs"] / link["h2d_gbs"]
+    del K, V
+    torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_extra:
+        # the two other full-size workloads, compact: long context (70B shape) and priority churn (32B shape)
+        try:
+            lc = long_context_leg(torch, B, hbm_peak, compact=True)
+            result["long_context"] = lc
+            flat.update({"longctx_offload_under_decode_gbs": lc["offload_under_decode_gbs"],
+                         "longctx_offload_alone_gbs": lc["offload_alone_gbs"],
+                         "longctx_adaptive_hidden_frac": lc["pipelined_adaptive"]["hidden_frac"],
+                         "longctx_adaptive_reload_gbs": lc["pipelined_adaptive"]["reload_under_decode_gbs"],
+                         "longctx_adaptive_step_us_with_reload": lc["pipelined_adaptive"]["step_us_with_reload"],
+                         "longctx_step_us_no_reload": lc["pipelined_adaptive"]["step_us_no_reload"],
+                         "longctx_256mib_hidden_frac": lc["pipelined_256MiB"]["hidden_frac"]})
+        except Exception as e:                       # e.g. the box cannot pin 10 GiB
+            result["long_context"] = {"skipped": repr(e)[:200]}
+        torch.cuda.empty_cache()
+    if rank == 0 and "roofline" in result:
+        result["roofline"].update(flat)
     if rank == 0 and world == 1:
-        del K, V
-        result["cpu_baseline"] = time_oracle(args.cpu_seconds)
+        result["cpu_baseline"] = time_oracle(args.cpu_seconds, sh.num_layers, sum(w.ctx_lens))
     group.close()
     if rank == 0:
         print(json.dumps(result))
+
+
+def spawn_replicas(args):
+    """`python bench.py --gpus N` outside a launcher: starts the N replicas itself (rank 0 prints the line)."""
+    from paper_2512_12928_b200 import replicas
+    rcs = replicas.spawn([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], args.gpus)
+    sys.exit(max(abs(rc) for rc in rcs))
 
 
 def main():
@@ -965,6 +1087,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--budget-mib", type=int, default=-1, help="copy budget per step in MiB for phase B (-1 = unlimited)")
     ap.add_argument("--no-overlap", action="store_true", help="skip the overlap budget sweep")
+    ap.add_argument("--no-extra", action="store_true", help="skip the compact long-context and churn legs")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--workload", default="llama8b_swap", choices=["llama8b_swap", "long_context", "churn", "decode_shapes"],
                     help="llama8b_swap is the headline line; the others print a line of their own (one GPU)")
@@ -972,6 +1095,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_replicas(args)
     elif args.workload != "llama8b_swap":
         run_extra(args)
     else:

@@ -9,13 +9,70 @@ both sides of the timed region and a max-over-ranks of the device times, through
 from __future__ import annotations
 
 import os
-from typing import List, Sequence, Tuple
+import socket
+import subprocess
+import sys
+from typing import List, Optional, Sequence, Tuple
 
 
 def env() -> Tuple[int, int, int]:
     """(rank, world size, local rank) from the launcher's environment (1 process = rank 0 of 1)."""
     return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
             int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def spawn(argv: Sequence[str], n: int, stdout=None) -> List[int]:
+    """Starts n replicas of a command on this node, one process per GPU, with the environment a launcher would
+    give them (RANK = LOCAL_RANK = 0..n-1, WORLD_SIZE = n, rendezvous on 127.0.0.1 at a free port), waits for
+    all of them and returns their exit codes.  What `bench.py --gpus N` does when it was not started by a
+    launcher."""
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for rank in range(n):
+        env = dict(os.environ, RANK=str(rank), LOCAL_RANK=str(rank), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen(list(argv), env=env, stdout=stdout))
+    return [p.wait() for p in procs]
+
+
+def numa_cpus_of_gpu(local_rank: int, sysfs: str = "/sys") -> Optional[List[int]]:
+    """CPUs of the NUMA node the GPU's PCIe slot hangs off, from sysfs, or None when the box does not say
+    (pinned host pools allocated by a process bound to these CPUs land in the memory nearest to the GPU's link)."""
+    try:
+        import torch
+        p = torch.cuda.get_device_properties(local_rank)
+        bus = f"{p.pci_domain_id:04x}:{p.pci_bus_id:02x}:{p.pci_device_id:02x}.0"
+        node = int(open(os.path.join(sysfs, "bus/pci/devices", bus, "numa_node")).read())
+        if node < 0:
+            return None
+        return parse_cpulist(open(os.path.join(sysfs, "devices/system/node", f"node{node}", "cpulist")).read())
+    except Exception:
+        return None
+
+
+def parse_cpulist(text: str) -> List[int]:
+    """'0-3,8,10-11' -> [0, 1, 2, 3, 8, 10, 11]."""
+    cpus: List[int] = []
+    for part in text.strip().split(","):
+        if not part:
+            continue
+        lo, _, hi = part.partition("-")
+        cpus.extend(range(int(lo), int(hi or lo) + 1))
+    return cpus
+
+
+def bind_near_gpu(local_rank: int) -> bool:
+    """Restricts this process to the CPUs near its GPU, if the box exposes them and they are allowed."""
+    cpus = numa_cpus_of_gpu(local_rank)
+    if not cpus:
+        return False
+    allowed = sorted(set(cpus) & os.sched_getaffinity(0))
+    if not allowed:
+        return False
+    os.sched_setaffinity(0, allowed)
+    return True
 
 
 def replica_seed(base_seed: int, rank: int) -> int:

@@ -99,6 +99,45 @@ def test_two_gloo_replicas_are_independent_and_aggregate_like_the_bench(tmp_path
     assert outs[0]["seed"] != outs[1]["seed"]
 
 
+SPAWNED = r"""
+import json, os, sys
+sys.path.insert(0, {root!r})
+from paper_2512_12928_b200 import binding as B, replicas
+g = replicas.Group("gloo")
+rank, world, local = replicas.env()
+lib = B.KVSwap(num_layers=2, num_kv_heads=2, num_q_heads=4, head_dim=64, block_size=16, num_gpu_blocks=32,
+               max_blocks_per_req=8, host_pool_bytes=1 << 20, flags=B.PS_FLAG_BOOKKEEPING_ONLY)
+assert lib.kv_alloc(rank, 40 * (rank + 1)) == 0
+blocks = len(lib.block_table(rank)[0])
+(total,) = g.sum_over_ranks([blocks])
+open(os.path.join({out!r}, f"rank{{rank}}.json"), "w").write(json.dumps(
+    {{"rank": rank, "world": world, "local": local, "addr": os.environ["MASTER_ADDR"], "total": total}}))
+g.close()
+"""
+
+
+def test_spawn_starts_one_replica_per_rank_with_a_launcher_environment(tmp_path):
+    """What `bench.py --gpus N` does without a launcher: N processes with RANK / LOCAL_RANK / WORLD_SIZE and a
+    rendezvous on 127.0.0.1, here with bookkeeping-only contexts over gloo."""
+    from paper_2512_12928_b200 import build as ps_build, replicas
+    ps_build.build()
+    script = tmp_path / "spawned.py"
+    script.write_text(SPAWNED.format(root=ROOT, out=str(tmp_path)))
+    rcs = replicas.spawn([sys.executable, str(script)], 2)
+    assert rcs == [0, 0]
+    outs = [json.loads((tmp_path / f"rank{r}.json").read_text()) for r in range(2)]
+    assert [d["rank"] for d in outs] == [0, 1] and [d["local"] for d in outs] == [0, 1]
+    assert all(d["world"] == 2 and d["addr"] == "127.0.0.1" for d in outs)
+    assert all(d["total"] == 3.0 + 5.0 for d in outs)          # ceil(40 / 16) + ceil(80 / 16) blocks
+
+
+def test_cpulist_parsing_and_missing_numa_information():
+    from paper_2512_12928_b200 import replicas
+    assert replicas.parse_cpulist("0-3,8,10-11\n") == [0, 1, 2, 3, 8, 10, 11]
+    assert replicas.parse_cpulist("") == []
+    assert replicas.numa_cpus_of_gpu(0, sysfs="/nonexistent") is None     # no such box: nothing is bound
+
+
 def test_reference_arm_is_silent_on_other_ranks():
     env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1", MASTER_ADDR="127.0.0.1", MASTER_PORT="1")
     p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
