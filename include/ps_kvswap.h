@@ -403,12 +403,13 @@ typedef struct ps_budget_model {
  *   case 1  T_fwd_min > t_budget        : B_copy = floor(t_budget / t_block)
  *   case 2  T_fwd_min <= t_budget and
  *     2i    T_fwd_min > T_trans_max     : B_copy = all missing blocks
- *     2ii   otherwise                   : binary search for the largest B with
+ *     2ii   otherwise                   : the largest B with
  *                                         B * t_block <= estimated step time after copying B blocks,
  * where "after copying B blocks" means: the requests of `reqs` that are resident now, plus those the
- * reload queue completes when it consumes B blocks in order.  (This library's path has no recomputation,
- * so that estimate grows with B; the search is valid because a block takes longer to copy than to
- * attend to: t_block > a_d * block_size is required in case 2ii, else PS_ERR_INVALID.)
+ * reload queue completes when it consumes B blocks in order.  (The paper finds that B by binary search over a
+ * latency that falls as more is copied.  This library's path has no recomputation: the estimate is a step
+ * function that rises whenever a queued request becomes complete, the test can fail and hold again, so the
+ * intervals between those steps are scanned instead, one closed-form candidate each.)
  *   reqs          : host array, the decode batch of the coming step (as for ps_step)
  *   budget_blocks : B_copy;  budget_bytes : B_copy * bytes of a block over all layers, for ps_step
  *   which_case    : 1, 21 or 22 (may be NULL)

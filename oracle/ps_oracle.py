@@ -418,10 +418,13 @@ class PsOracle:
 
         T_fwd_min: estimated forward time with all host-resident blocks of the queue copied;
         T_trans_max = sum of b_miss * t_block.  (1) T_fwd_min > t_budget: floor(t_budget / t_block).
-        (2) otherwise, (i) T_fwd_min > T_trans_max: all missing blocks; (ii) else binary search for the largest
-        B_copy whose transfer time does not exceed the estimated batch latency.  Reading for this decode-only
-        path (no recomputation): the batch latency after copying B blocks is `step_latency_after`, which
-        grows with B, slower than the transfer time as long as t_block > a_d * s_blk.
+        (2) otherwise, (i) T_fwd_min > T_trans_max: all missing blocks; (ii) else the largest B_copy whose
+        transfer time does not exceed the estimated batch latency.  The paper finds it by binary search,
+        relying on a latency that falls monotonically as more is copied (its engine recomputes what is
+        missing).  Reading for this decode-only path (no recomputation): the batch latency after copying B
+        blocks is `step_latency_after`, a step function that jumps up whenever a queued request becomes
+        complete, so "B * t_block <= latency(B)" can turn false and true again; the definition itself is
+        taken instead: every B from 0 to B_missing is tried and the largest feasible one returned.
         Returns (B_copy, case) with case 1, 21 or 22.
         """
         b_missing = sum(self.missing_blocks(q) for q in self.in_fifo)
@@ -431,15 +434,11 @@ class PsOracle:
             return int(math.floor(t_budget / t_block)), 1
         if t_fwd_min > t_trans_max:
             return b_missing, 21
-        assert t_block > a_d * self.S
-        lo, hi = 0, b_missing
-        while lo < hi:
-            mid = lo + (hi - lo + 1) // 2
-            if mid * t_block <= self.step_latency_after(reqs, mid, a_d, b_d, t_c):
-                lo = mid
-            else:
-                hi = mid - 1
-        return lo, 22
+        best = 0
+        for b in range(b_missing + 1):
+            if b * t_block <= self.step_latency_after(reqs, b, a_d, b_d, t_c):
+                best = b
+        return best, 22
 
     # ------------------------------------------------------------------ eviction policy, partial-copy rule
     def select_victims(self, queue: Sequence[int], waited: Sequence[float], tau: float, near_frac: float,

@@ -52,22 +52,23 @@ int32_t ps_copy_budget(ps_ctx* ctx, const int64_t* reqs, int32_t batch, const ps
         B = missing;
     } else {
         wc = 22;
-        if (!(t_block > a_d * (double)ctx->cfg.block_size))
-            return ctx->fail(PS_ERR_INVALID, "ps_copy_budget: the search needs t_block > a_d * block_size");
-        auto step_time_after = [&](int64_t blocks) {  // requests whose last missing block is among the first `blocks`
-            double t = t_resident;
-            for (size_t i = 0; i < cum_miss.size() && cum_miss[i] <= blocks; ++i) t = t_resident + cum_time[i];
-            return t;
-        };
-        int64_t lo = 0, hi = missing;  // lo is feasible (0 blocks take no time)
-        while (lo < hi) {
-            const int64_t mid = lo + (hi - lo + 1) / 2;
-            if ((double)mid * t_block <= step_time_after(mid))
-                lo = mid;
-            else
-                hi = mid - 1;
+        // The estimated step time after copying B blocks is a step function of B: it jumps up by a request's
+        // decode time when the request's last missing block is among the first B.  "B * t_block <= step time"
+        // can therefore hold again beyond a point where it fails, and a binary search may stop far below the
+        // largest feasible B.  Between two jumps the step time is constant, so the largest feasible B of
+        // every such interval is known in closed form; the answer is the largest over the intervals.
+        const size_t nq = cum_miss.size();
+        for (size_t i = 0; i <= nq; ++i) {  // interval i: the first i queued requests are complete
+            const int64_t lo = i == 0 ? 0 : cum_miss[i - 1];
+            const int64_t hi = i == nq ? missing : cum_miss[i] - 1;
+            if (hi < lo) continue;
+            const double t = t_resident + (i == 0 ? 0.0 : cum_time[i - 1]);
+            int64_t cand = (int64_t)std::floor(t / t_block);
+            while ((double)(cand + 1) * t_block <= t) ++cand;  // the decision is "B * t_block <= t", exactly
+            while (cand > 0 && (double)cand * t_block > t) --cand;
+            cand = std::min(cand, hi);
+            if (cand >= lo && cand > B) B = cand;
         }
-        B = lo;
     }
     *budget_blocks = B;
     if (budget_bytes) *budget_bytes = B * ctx->block_bytes;

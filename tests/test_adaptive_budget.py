@@ -84,7 +84,9 @@ def test_search_equals_exhaustive_scan_and_library_matches_on_random_queues():
         lib.step(None, None, ids, part); orc.step(part, ids)
         batch = [r for r in ids if rng.random() < 0.8] + [999]           # an unknown id is ignored
         a_d = float(rng.uniform(0.001, 0.05)); b_d = float(rng.uniform(0, 3)); t_c = float(rng.uniform(0, 50))
-        t_block = float(rng.uniform(a_d * sh.block_size * 1.01, 5.0))
+        if trial % 2:                                    # large per-request constants: the test is far from monotone
+            b_d = float(rng.uniform(20, 200))
+        t_block = float(rng.uniform(0.05, 5.0))
         b_missing = sum(orc.missing_blocks(r) for r in ids)
         for t_budget in (0.0, float(rng.uniform(0, 200)), 1e9):
             want = orc.copy_budget(batch, a_d, b_d, t_c, t_block, t_budget)
@@ -135,6 +137,25 @@ def test_library_rejects_bad_models():
     assert lib.swap_in_begin(0) == 0
     assert lib.copy_budget([0], a_d=1.0, b_d=0.0, t_c=0.0, t_block=0.0, t_budget=10.0)[0] == B.PS_ERR_INVALID
     assert lib.copy_budget([0], a_d=-1.0, b_d=0.0, t_c=0.0, t_block=1.0, t_budget=10.0)[0] == B.PS_ERR_INVALID
-    # case 2ii with a block that copies faster than it is attended to: the search is not valid
-    rc, _, _, _ = lib.copy_budget([0], a_d=1.0, b_d=0.0, t_c=0.0, t_block=4.0, t_budget=1e9)
-    assert rc == B.PS_ERR_INVALID and "t_block" in lib.last_error()
+    # a block that copies as fast as it is attended to is no longer refused: every interval is scanned
+    rc, blocks, _, case = lib.copy_budget([0], a_d=1.0, b_d=0.0, t_c=0.0, t_block=4.0, t_budget=1e9)
+    assert (rc, blocks, case) == (B.PS_OK, 10, 22)          # 10 blocks * 4 = 40 <= 40 tokens * 1
+
+
+def test_largest_feasible_budget_beyond_a_first_failure(repo_root):
+    """The hand-worked queue on which the feasibility test fails and holds again (a binary search answers 2)."""
+    g = json.load(open(os.path.join(repo_root, "tests", "golden", "adaptive_budget.json")))["non_monotone_case"]
+    lib, orc = make_pair(wl.KVShape(**g["shape"]))
+    for x in (lib, orc):
+        for r, n in g["resident_tokens"] + g["queued_tokens"]:
+            assert x.kv_alloc(r, n) == 0
+        for r, _ in g["queued_tokens"]:
+            assert x.swap_out(r) == 0
+    lib.sync(); orc.reap()
+    for x in (lib, orc):
+        for r, _ in g["queued_tokens"]:
+            assert x.swap_in_begin(r) == 0
+    kw = dict(a_d=g["a_d"], b_d=g["b_d"], t_c=g["t_c"], t_block=g["t_block"], t_budget=g["t_budget"])
+    assert orc.copy_budget(g["batch"], **kw) == (g["blocks"], g["case"])
+    rc, blocks, _, case = lib.copy_budget(g["batch"], **kw)
+    assert (rc, blocks, case) == (B.PS_OK, g["blocks"], g["case"])
