@@ -330,6 +330,12 @@ class KVSwap:
         self._ck(self.lib.ps_block_table(self.h, req, ids, n.value, None, None, None), "ps_block_table")
         return list(ids[: n.value]), st.value
 
+    def req_state(self, req: int) -> int:
+        """ps_req_state of the request, PS_REQ_NONE for an unknown one (no table is copied)."""
+        st = C.c_int32()
+        rc = self.lib.ps_block_table(self.h, req, None, 0, None, C.byref(st), None)
+        return st.value if rc == PS_OK else PS_REQ_NONE
+
     def n_tokens(self, req: int) -> int:
         nt = C.c_int32()
         self._ck(self.lib.ps_block_table(self.h, req, None, 0, None, None, C.byref(nt)), "ps_block_table")

@@ -267,7 +267,10 @@ inline int32_t blocks_for(const ps_ctx* ctx, int32_t n_tokens) {
 }
 void push_table(ps_ctx* ctx, std::vector<int32_t>& table);
 int32_t check_status_word(ps_ctx* ctx);
-int32_t do_poll(ps_ctx* ctx, int32_t* n_reaped);
+// reap_offloads = false: only the side tasks (host images of landed reloads, reload gates, parked ranges);
+// finished offloads give their blocks back in ps_poll / ps_step / ps_sync alone, which report how many, so a
+// caller can follow the free-block count exactly.
+int32_t do_poll(ps_ctx* ctx, int32_t* n_reaped, bool reap_offloads = true);
 
 // swap-out and swap-in issue (ps_swap.cu)
 int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi);

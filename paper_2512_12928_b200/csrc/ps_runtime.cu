@@ -185,11 +185,11 @@ int32_t check_status_word(ps_ctx* ctx) {
     return PS_OK;
 }
 
-int32_t do_poll(ps_ctx* ctx, int32_t* n_reaped) {
+int32_t do_poll(ps_ctx* ctx, int32_t* n_reaped, bool reap_offloads) {
     int32_t reaped = 0;
     int32_t rc = tracker_poll(ctx, ctx->t_d2h);
     if (rc != PS_OK) return rc;
-    while (!ctx->out_fifo.empty()) {
+    while (reap_offloads && !ctx->out_fifo.empty()) {
         Req& r = ctx->reqs[ctx->out_fifo.front()];
         if (r.out_ticket > ctx->t_d2h.done) break;  // offloads complete in issue order
         push_table(ctx, r.table);
@@ -534,12 +534,12 @@ int32_t ps_kv_free(ps_ctx* ctx, int64_t req) {
         return ctx->fail(PS_ERR_BUSY, "ps_kv_free: transfer in flight");
     if (r.state == PS_REQ_RESIDENT) {
         if (r.gated) {
-            int32_t rc = do_poll(ctx, nullptr);
+            int32_t rc = do_poll(ctx, nullptr, /*reap_offloads=*/false);
             if (rc != PS_OK) return rc;
             if (r.gated) return ctx->fail(PS_ERR_BUSY, "ps_kv_free: reload copies still in flight");
         }
         if (!r.segs.empty()) {  // proactive copies: their transfers must have ended before the image goes
-            int32_t rc = do_poll(ctx, nullptr);
+            int32_t rc = do_poll(ctx, nullptr, /*reap_offloads=*/false);
             if (rc != PS_OK) return rc;
             if (r.segs.back().ticket > ctx->t_d2h.done)
                 return ctx->fail(PS_ERR_BUSY, "ps_kv_free: proactive offload still in flight");

@@ -360,7 +360,7 @@ int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, flo
         any_gated |= it->second.gated;
     }
     if (any_gated) {
-        int32_t rc = do_poll(ctx, nullptr);  // the copies may have landed since
+        int32_t rc = do_poll(ctx, nullptr, /*reap_offloads=*/false);  // the copies may have landed since
         if (rc != PS_OK) return rc;
     }
     std::vector<char> active((size_t)batch, 1), gated((size_t)batch, 0);

@@ -182,7 +182,7 @@ int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi) {
     const int64_t bytes = n_blk * ctx->block_bytes;
     int64_t off = ctx->hpool.alloc(bytes);
     if (off < 0) {  // images of reloads that have landed since the last poll may still be held
-        int32_t rc = do_poll(ctx, nullptr);
+        int32_t rc = do_poll(ctx, nullptr, /*reap_offloads=*/false);
         if (rc != PS_OK) return rc;
         off = ctx->hpool.alloc(bytes);
     }
