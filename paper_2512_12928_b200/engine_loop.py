@@ -56,6 +56,15 @@ class LoopParams:
     max_batch: int = 256
 
 
+def config4_params(**over) -> LoopParams:
+    """Knobs for the priority-churn workload at its full shape (64 layers, 4 MiB blocks, steps of about 13 ms):
+    a starvation threshold and lifetimes short enough that evicted requests come back within tens of rounds,
+    which offers the host link a sustained load of about half its rate in each direction."""
+    kw = dict(tau_us=150e3, max_admit=2, gen_tokens=(20, 60), host_budget_bytes=12 << 30)
+    kw.update(over)
+    return LoopParams(**kw)
+
+
 @dataclass
 class StubRequest:
     rid: int
@@ -216,7 +225,10 @@ class SchedulerStub:
         return [ids[i] for i in order], [waited[i] for i in order], t_budget
 
     # ---- one round of the closed loop
-    def round(self, q_all, out_all) -> RoundReport:
+    def round(self, q_all, out_all, on_step=None) -> RoundReport:
+        """One round.  q_all / out_all: device bf16 [L][max_batch][Hq][D] (their first len(batch) rows are used) or
+        None on a context without a device.  on_step(batch, mask, q, out), if given, is called right after the
+        step, before the decoded requests grow by their new token."""
         p, be = self.p, self.be
         be.poll()                                             # finished offloads give their blocks back
         queue, waited, t_budget = self._ordered()
@@ -293,6 +305,8 @@ class SchedulerStub:
         before = {rid: be.missing(rid) for rid in rule}
         mask, stats = be.step(_front(q_all, n), _front(out_all, n), batch, nbytes, p.beta, rule)
         rep = RoundReport(self.now, t_budget, blocks, case, batch, mask, stats, evicted, admitted, readmitted)
+        if on_step is not None:
+            on_step(batch, mask, _front(q_all, n), _front(out_all, n))
         if stats["blocks_copied"] < blocks:                   # budget left over: who was passed over by the rule?
             rep.skipped_by_rule = sum(1 for rid, m in before.items() if m > 0 and be.missing(rid) == m)
         # what the step did to the traffic

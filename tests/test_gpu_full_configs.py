@@ -18,6 +18,8 @@ pytestmark = pytest.mark.gpu
 
 if torch.cuda.is_available():
     from gpu_util import FullSizePair
+    from loop_util import PairedBackend
+    from paper_2512_12928_b200 import engine_loop as el
 
 
 def _queries(sh, n, seed):
@@ -235,4 +237,59 @@ def test_config4_priority_churn_full_shape():
         if rq.state == 3:
             p.assert_image_matches(r)
     assert moved > 0 and ok_out > 50 and ok_in > 50 and decoded > 0
+    p.destroy()
+
+
+def test_config4_closed_loop_driven_by_the_scheduler_stub_full_shape():
+    """Config 4 at its shape (64 layers, 24 576 blocks of 4 MiB, 256 live requests of 512-16k tokens, two
+    priority classes) driven by the paper's closed loop instead of a seeded script: every round the queue is
+    ordered (ps_order_queue), memory pressure evicts from the tail (ps_select_victims, asynchronous offloads
+    reaped when their transfers complete), the head is readmitted, ps_copy_budget sets the step's budget and
+    ps_step_ruled consumes it under the partial-copy rule while the resident set decodes.  A backend makes
+    every call on the library and on the checkers and compares decisions, codes, states and plans; bytes of
+    two sampled layers and attention on sampled rows are compared as in the other full-size tests."""
+    _need_memory(130)
+    w = wl.churn()
+    sh = w.shape
+    params = el.config4_params()
+    try:
+        p = FullSizePair(w, [0, sh.num_layers - 1], max_batch=params.max_batch, max_blocks_per_req=1040,
+                         host_pool_bytes=30 * wl.GiB)
+    except B.PsError as e:
+        pytest.skip(str(e))
+    be = PairedBackend(p.lib, p.book, p.data)
+    stub = el.SchedulerStub(be, w.ctx_lens, w.priority, sh.block_size, sh.block_bytes, sh.num_gpu_blocks, params,
+                            seed=w.seed)
+    placed = stub.fill()
+    assert len(placed) > 30
+    q, out = _queries(sh, params.max_batch, 19)
+    checked = []
+
+    def on_step(batch, mask, qv, ov):
+        if stub.rounds % 12 == 0 or stub.rounds >= 58:
+            torch.cuda.synchronize()
+            rows = [k for k, m in enumerate(mask) if m]
+            gated_rows = [k for k in rows if batch[k] in {r for r, _, _ in be.plans}]
+            p.check_attention(ov, qv, batch, mask, (rows[:2] + rows[-1:] + gated_rows[:2]))
+            checked.append(len(rows))
+
+    tot = dict(evicted=0, readmitted=0, admitted=0, finished=0, copied=0, decoded=0)
+    for _ in range(60):
+        rep = stub.round(q, out, on_step)
+        tot["evicted"] += len(rep.evicted)
+        tot["readmitted"] += len(rep.readmitted)
+        tot["admitted"] += len(rep.admitted)
+        tot["finished"] += len(rep.finished)
+        tot["copied"] += rep.stats["blocks_copied"]
+        tot["decoded"] += sum(rep.mask)
+        if stub.rounds % 20 == 0:
+            p.book.check_invariants()
+    p.sync()
+    p.assert_tables_equal(sorted(p.book.reqs))
+    p.assert_sampled_pools_equal()
+    for r, rq in p.data.reqs.items():             # every image still on host equals the checker's
+        if rq.state == 3:
+            p.assert_image_matches(r)
+    assert tot["evicted"] >= 3 and tot["readmitted"] >= 2 and tot["copied"] > 500 and tot["decoded"] > 1500, tot
+    assert be.counts["victims"] >= 1 and be.counts["budget"] == 60 and len(checked) >= 5
     p.destroy()
