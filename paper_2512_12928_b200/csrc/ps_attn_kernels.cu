@@ -501,7 +501,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                        const __nv_bfloat16* __restrict__ q, __nv_bfloat16* __restrict__ out, float* __restrict__ lse,
                        AttnBatch batch, int32_t sched_lane, int32_t block_size, int32_t block_shift,
                        int32_t num_blocks, float* __restrict__ partials, int32_t* __restrict__ sched,
-                       int32_t* __restrict__ row_done, float scale_log2e, int32_t* status) {
+                       int32_t* __restrict__ row_done, float scale_log2e, int32_t* status, int32_t wait_first) {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     static_assert(HKV == kMmaHkv || kTma, "fewer than 8 KV heads need the tensor-map mode");
     constexpr int Hq = HKV * G;
@@ -557,6 +557,11 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy zeroes before async-proxy writes
     }
     __syncthreads();
+    // A launch whose inputs (queries, KV, batch metadata) may come from the kernel before it on the stream is
+    // still made programmatically dependent on that kernel: block scheduling, the shared-memory set-up and the
+    // barrier initialisation above then run under the predecessor's tail, and every thread waits here, before
+    // the first read of anything the predecessor may have written.
+    if (wait_first) dep_wait();
 
     const int32_t* cta_begin = batch.cta_begin[sched_lane];
     const int item0 = cta_begin[blockIdx.x];
@@ -883,7 +888,7 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
 template <int G, int HKV>
 cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool, const AttnTensorMaps* maps, const void* q,
                        void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials, int32_t* sched,
-                       int32_t* row_done, int32_t* d_status, bool after_own_launch, cudaStream_t stream) {
+                       int32_t* row_done, int32_t* d_status, int dep_mode, cudaStream_t stream) {
     const float scale_log2e = 1.4426950408889634f / sqrtf((float)kMmaD);
     static_assert(sizeof(CUtensorMap) == sizeof(maps->k), "AttnTensorMaps must hold driver tensor maps");
     if (HKV != kMmaHkv && maps == nullptr) return cudaErrorNotSupported;
@@ -896,7 +901,8 @@ cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = after_own_launch ? 1 : 0;
+    cfg.numAttrs = dep_mode != 0 ? 1 : 0;
+    const int32_t wait_first = dep_mode == 2 ? 1 : 0;
     CUtensorMap km, vm;
     if (maps != nullptr) {
         memcpy(&km, maps->k, sizeof km);
@@ -912,23 +918,23 @@ cudaError_t launch_mma(const AttnShape& sh, const void* kpool, const void* vpool
     const int32_t shift = shift_of(sh.block_size);
     if (maps != nullptr)
         return cudaLaunchKernelEx(&cfg, decode_attn_mma_kernel<G, HKV, true>, kp, vp, km, vm, qp, op, lse, batch, lane,
-                                  sh.block_size, shift, sh.num_blocks, partials, sched, row_done, scale_log2e, d_status);
+                                  sh.block_size, shift, sh.num_blocks, partials, sched, row_done, scale_log2e, d_status, wait_first);
     if constexpr (HKV == kMmaHkv)
         return cudaLaunchKernelEx(&cfg, decode_attn_mma_kernel<G, HKV, false>, kp, vp, km, vm, qp, op, lse, batch, lane,
-                                  sh.block_size, shift, sh.num_blocks, partials, sched, row_done, scale_log2e, d_status);
+                                  sh.block_size, shift, sh.num_blocks, partials, sched, row_done, scale_log2e, d_status, wait_first);
     return cudaErrorNotSupported;
 }
 
 template <int G>
 cudaError_t launch_mma_hkv(const AttnShape& sh, const void* kpool, const void* vpool, const AttnTensorMaps* maps,
                            const void* q, void* out, float* lse, const AttnBatch& batch, int32_t lane, float* partials,
-                           int32_t* sched, int32_t* row_done, int32_t* d_status, bool after_own_launch,
+                           int32_t* sched, int32_t* row_done, int32_t* d_status, int dep_mode,
                            cudaStream_t stream) {
     switch (sh.num_kv_heads) {
 #define PS_HKV_CASE(HH)                                                                                              \
     case HH:                                                                                                         \
         return launch_mma<G, HH>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status, \
-                                 after_own_launch, stream);
+                                 dep_mode, stream);
         PS_HKV_CASE(1) PS_HKV_CASE(2) PS_HKV_CASE(4) PS_HKV_CASE(8)
 #undef PS_HKV_CASE
     }
@@ -1003,7 +1009,7 @@ cudaError_t attn_make_tensor_maps(const AttnShape& sh, const void* kpool, const 
 cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool,
                                const AttnTensorMaps* maps, const void* q, void* out, float* lse, const AttnBatch& batch,
                                int32_t lane, float* partials, int32_t* sched, int32_t* row_done, int32_t* d_status,
-                               bool after_own_launch, cudaStream_t stream) {
+                               int dep_mode, cudaStream_t stream) {
     if (lane < 0 || lane > 1) return cudaErrorInvalidValue;
     const int item_begin = batch.lane_items[lane];
     const int n_items = batch.lane_items[lane + 1] - item_begin;
@@ -1014,21 +1020,21 @@ cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpoo
             return cudaErrorNotSupported;
         switch (G) {
             case 1: return launch_mma_hkv<1>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       after_own_launch, stream);
+                                       dep_mode, stream);
             case 2: return launch_mma_hkv<2>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       after_own_launch, stream);
+                                       dep_mode, stream);
             case 3: return launch_mma_hkv<3>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       after_own_launch, stream);
+                                       dep_mode, stream);
             case 4: return launch_mma_hkv<4>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       after_own_launch, stream);
+                                       dep_mode, stream);
             case 5: return launch_mma_hkv<5>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       after_own_launch, stream);
+                                       dep_mode, stream);
             case 6: return launch_mma_hkv<6>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       after_own_launch, stream);
+                                       dep_mode, stream);
             case 7: return launch_mma_hkv<7>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       after_own_launch, stream);
+                                       dep_mode, stream);
             case 8: return launch_mma_hkv<8>(sh, kpool, vpool, maps, q, out, lse, batch, lane, partials, sched, row_done, d_status,
-                                       after_own_launch, stream);
+                                       dep_mode, stream);
         }
         return cudaErrorNotSupported;
     }

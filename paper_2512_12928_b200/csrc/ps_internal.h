@@ -84,8 +84,11 @@ cudaError_t attn_make_tensor_maps(const AttnShape& sh, const void* kpool, const 
 cudaError_t launch_decode_attn(int kernel, const AttnShape& sh, const void* kpool, const void* vpool,
                                const AttnTensorMaps* maps, const void* q, void* out, float* lse, const AttnBatch& batch,
                                int32_t lane, float* partials, int32_t* sched, int32_t* row_done, int32_t* d_status,
-                               bool after_own_launch, cudaStream_t stream);
-// after_own_launch (tensor-core kernel only): the previous kernel on `stream` is a launch of the same kernel
+                               int dep_mode, cudaStream_t stream);
+// dep_mode (tensor-core kernel only): 0 = an ordinary launch.  2 = programmatically dependent on whatever kernel
+// precedes it on `stream`, the kernel waiting for that kernel's completion right after its own set-up and before
+// it reads any input (safe after any predecessor; gains the launch latency and the set-up when the predecessor
+// lets dependents start early, as this kernel does).  1 = the previous kernel on `stream` is a launch of the same kernel
 // whose inputs and outputs are independent of this one's; the launch is then made programmatically
 // dependent on it, so its CTAs start as that launch's CTAs retire.  The kernel waits for its predecessor's
 // completion before it first touches partials / sched / row_done, so consecutive launches may even share

@@ -309,6 +309,9 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
     if (wait_event && !lanes) CK(cudaStreamWaitEvent(ctx->compute, wait_event, 0));
     if (m.n_ungated_items > 0) {
         const bool overlap = follows_own && mma && !ctx->profile && m.dev.n_cta[0] == ctx->num_sms;
+        // one layer per call: the caller's kernels sit between the launches, so only the set-up may run early
+        const bool early_setup = !follows_own && mma && !ctx->profile && wait_event == nullptr &&
+                                 (ctx->cfg.flags & PS_FLAG_ATTN_EARLY_SETUP) != 0;
         const int set = ctx->scratch_set;
         ctx->scratch_set ^= 1;
         const int64_t bytes = m.kv_bytes_per_layer * m.n_ungated_items / m.n_items;
@@ -316,7 +319,7 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
             ProfScope prof(ctx, kProfAttn, ctx->compute, bytes, wait_event && !lanes ? 1000 + layer : layer);
             CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], maps, q, out, lse, m.dev,
                                       0, ctx->partials[set], ctx->d_sched[set], ctx->d_row_done[set], ctx->d_status,
-                                      overlap, ctx->compute));
+                                      overlap ? 1 : early_setup ? 2 : 0, ctx->compute));
             ctx->launches++;
             ++*n_launched;
         }
@@ -333,7 +336,7 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
         const int64_t bytes = m.kv_bytes_per_layer * (m.n_items - m.n_ungated_items) / m.n_items;
         ProfScope prof(ctx, kProfAttn, ctx->s_lane, bytes, 1000 + layer);
         CK(ps::launch_decode_attn(ctx->attn_kernel, sh, ctx->kpools[layer], ctx->vpools[layer], maps, q, out, lse, m.dev, 1,
-                                  ctx->partials[2], ctx->d_sched[2], ctx->d_row_done[2], ctx->d_status, false, ctx->s_lane));
+                                  ctx->partials[2], ctx->d_sched[2], ctx->d_row_done[2], ctx->d_status, 0, ctx->s_lane));
         ctx->launches++;
         ++*n_launched;
     }

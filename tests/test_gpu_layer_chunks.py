@@ -218,3 +218,41 @@ def test_attention_recovers_after_a_kernel_side_timeout_report():
     for l in range(2):
         check_attn(out[l], want[l])
     assert p.lib.sync() == B.PS_OK
+
+
+def test_attention_with_early_set_up_matches_after_any_predecessor():
+    """PS_FLAG_ATTN_EARLY_SETUP: one-layer-per-call launches are programmatically dependent on the kernel before
+    them and wait for it before reading any input.  Back to back (the predecessor is the same kernel, which lets
+    dependents start early), after another library's kernel that produces the queries, and after a table
+    change (the predecessor is the metadata upload): results equal the checker's every time."""
+    sh, rng, p = build_pair(4, 420, 59, Hkv=8, Hq=32, D=128, max_batch=8, max_blocks_per_req=64,
+                            attn_kernel=B.PS_ATTN_MMA, flags=B.PS_FLAG_ATTN_EARLY_SETUP)
+    tokens = [700, 33, 720, 512, 1, 705]
+    reqs = list(range(len(tokens)))
+    for r, n in enumerate(tokens):
+        assert p.both("kv_alloc", r, n) == B.PS_OK
+    q = wl.randn_bf16_bits(rng, (4, len(reqs), sh.num_q_heads, sh.head_dim))
+    qd = bits_to_dev(q)
+    out = torch.zeros_like(qd)
+    for rounds in range(3):
+        for l in range(4):                                   # back to back: every launch follows the same kernel
+            assert p.lib.decode_attn(l, qd[l], out[l], reqs) == B.PS_OK
+    torch.cuda.synchronize()
+    for l in range(4):
+        check_attn(out[l], p.orc.decode_attn(l, q[l], reqs)[0])
+    # the queries are produced on the stream right before the launch that reads them
+    q2 = wl.randn_bf16_bits(rng, (4, len(reqs), sh.num_q_heads, sh.head_dim))
+    src = bits_to_dev(q2)
+    big = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")
+    for l in range(4):
+        big.fill_(l)                                         # some work in front, so the copy below is not instant
+        qd[l].copy_(src[l])
+        assert p.lib.decode_attn(l, qd[l], out[l], reqs) == B.PS_OK
+    torch.cuda.synchronize()
+    for l in range(4):
+        check_attn(out[l], p.orc.decode_attn(l, q2[l], reqs)[0])
+    # a table change: the batch metadata is uploaded by a kernel right before the attention launch
+    assert p.both("kv_alloc", 1, 400) == B.PS_OK
+    assert p.lib.decode_attn(2, qd[2], out[2], reqs) == B.PS_OK
+    torch.cuda.synchronize()
+    check_attn(out[2], p.orc.decode_attn(2, q2[2], reqs)[0])
