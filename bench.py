@@ -315,7 +315,7 @@ def swap_workload_step(torch, B, lib, w, q, out, q_res, out_res, budget, e2e_buf
         decode(residents, q_res, out_res, 0)
         steps_a += 1
         lib.poll()
-        if all(lib.block_table(r)[1] == B.PS_REQ_HOST for r in w.victims):
+        if lib.req_state(w.victims[-1]) == B.PS_REQ_HOST:      # offloads complete in issue order
             break
     ev[1].record()
     for r in w.victims:
@@ -565,7 +565,7 @@ def offload_rates(torch, B, lib, w, batch, q_b, out_b, nbytes):
         stream.synchronize()
         steps += 1
         lib.poll()
-        if all(lib.block_table(r)[1] == B.PS_REQ_HOST for r in w.victims):
+        if lib.req_state(w.victims[-1]) == B.PS_REQ_HOST:      # offloads complete in issue order
             break
     e1.record(); e1.synchronize()
     under_ms = e0.elapsed_time(e1)
@@ -1005,7 +1005,7 @@ def run_gpu(args):
 
     def fresh_ctx(flags):
         lib = make_ctx(B, w, K, V, sh.num_gpu_blocks, max_batch=nreq, host_pool_bytes=victim_bytes + (256 << 20),
-                       flags=flags)
+                       flags=flags, staging_bytes=args.staging_mib * wl.MiB)
         for r, n in wl.build_order_round_robin(w):
             assert lib.kv_alloc(r, n) == 0, lib.last_error()
         return lib
@@ -1218,6 +1218,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--budget-mib", type=int, default=-1, help="copy budget per step in MiB for phase B (-1 = unlimited)")
+    ap.add_argument("--staging-mib", type=int, default=0, help="device staging per direction in MiB (0 = library default)")
     ap.add_argument("--no-overlap", action="store_true", help="skip the overlap budget sweep")
     ap.add_argument("--no-extra", action="store_true", help="skip the compact long-context and churn legs")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
