@@ -381,6 +381,13 @@ int32_t ps_step_ruled(ps_ctx* ctx, const void* q_all_layers, void* out_all_layer
                       int32_t batch, int64_t copy_budget_bytes, const ps_copy_rule* rule, int32_t* decoded_mask,
                       ps_step_stats* stats);
 
+/* Reload bytes that ps_step calls have issued and whose copies have not been seen complete yet (a non-blocking
+ * look at the copy streams).  The budget rule of Section 4.3 assumes that a step's transfer ends within the step;
+ * when the link runs below the profiled t_block the queue of copies grows from step to step and the step that
+ * completes a request then waits for all of it.  A scheduler can subtract this figure from the budget it passes
+ * to the next ps_step.  Timing-dependent by nature: 0 on a context without a device. */
+int32_t ps_reload_backlog(ps_ctx* ctx, int64_t* bytes_in_flight);
+
 /* ps_step for callers whose queries and outputs live in HOST memory: copies q_host to a device buffer of the
  * context on the compute stream, runs the step, and copies the outputs back, all asynchronously on the compute
  * stream (synchronise that stream, or call ps_sync, before reading out_host).

@@ -32,7 +32,7 @@ EXPORTS = [
     "ps_launch_count", "ps_get_profile", "ps_link_probe", "ps_copy_blocks", "ps_trace", "ps_trace_read",
     "ps_decode_attn_static", "ps_copy_budget", "ps_offload_progress", "ps_host_blocks", "ps_host_segment",
     "ps_select_victims", "ps_copy_condition", "ps_order_queue", "ps_estimate_batch", "ps_resume_cost",
-    "ps_reload_fence", "ps_offload_sweep", "ps_step_ruled", "ps_step_host", "ps_inject_status", "ps_hbm_probe",
+    "ps_reload_fence", "ps_offload_sweep", "ps_step_ruled", "ps_step_host", "ps_inject_status", "ps_hbm_probe", "ps_reload_backlog",
 ]
 
 
@@ -144,6 +144,7 @@ def load() -> C.CDLL:
         "ps_hbm_probe": (i32, [i64, i32, i32, C.POINTER(C.c_double)]),
         "ps_copy_blocks": (i32, [vp, i32, i32, p32, i32, vp, i32]),
         "ps_inject_status": (i32, [vp, i32]),
+        "ps_reload_backlog": (i32, [vp, p64]),
         "ps_step_ruled": (i32, [vp, vp, vp, p64, i32, i64, C.POINTER(PsCopyRule), p32, C.POINTER(PsStepStats)]),
         "ps_step_host": (i32, [vp, vp, vp, p64, i32, i64, p32, C.POINTER(PsStepStats)]),
         "ps_trace": (i32, [vp, i32]),
@@ -445,6 +446,12 @@ class KVSwap:
         rc = self.lib.ps_step_host(self.h, C.c_void_p(q_host.data_ptr()), C.c_void_p(out_host.data_ptr()), arr,
                                    len(reqs), copy_budget_bytes, mask, C.byref(st))
         return rc, list(mask[: len(reqs)]), st.as_dict()
+
+    def reload_backlog(self) -> int:
+        """Reload bytes issued by earlier steps whose copies have not been seen complete."""
+        out = C.c_int64()
+        self._ck(self.lib.ps_reload_backlog(self.h, C.byref(out)), "ps_reload_backlog")
+        return out.value
 
     def inject_status(self, value: int) -> int:
         return self.lib.ps_inject_status(self.h, value)

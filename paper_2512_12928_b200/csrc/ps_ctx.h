@@ -180,6 +180,7 @@ struct ps_ctx {
     std::vector<cudaEvent_t> ev_pool, ev_pool_timing;
     std::deque<std::pair<uint64_t, std::pair<int64_t, int64_t>>> img_release;  // in_ticket -> (off, bytes)
     std::deque<std::pair<uint64_t, std::pair<int64_t, int64_t>>> host_release;  // t_d2h ticket -> (off, bytes)
+    std::deque<std::pair<uint64_t, int64_t>> reload_inflight;  // s_scatter ticket -> reload bytes issued before it
     std::vector<int64_t> gated_reqs;
     // split-KV scratch: sets 0 and 1 are used alternately by the launches on the compute stream (consecutive
     // launches of a step may overlap), set 2 by the launches on the reload lane

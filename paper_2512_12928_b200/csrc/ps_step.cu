@@ -494,6 +494,13 @@ static int32_t step_impl(ps_ctx* ctx, const void* q_all_layers, void* out_all_la
         }
     }
 
+    if (!plan.empty() && !ctx->bk) {  // what ps_reload_backlog reports until these copies have been seen complete
+        uint64_t ticket = 0;
+        rc = tracker_mark(ctx, ctx->t_scatter, &ticket);
+        if (rc != PS_OK) return rc;
+        ctx->reload_inflight.push_back({ticket, st.h2d_bytes});
+    }
+
     // 5. request states follow what was issued
     for (size_t i = 0; i < plan.size(); ++i) {
         Req& r = ctx->reqs[plan[i].req];
@@ -528,6 +535,18 @@ int32_t ps_step_ruled(ps_ctx* ctx, const void* q_all_layers, void* out_all_layer
                       int64_t copy_budget_bytes, const ps_copy_rule* rule, int32_t* decoded_mask, ps_step_stats* stats) {
     if (!ctx) return PS_ERR_INVALID;
     return step_impl(ctx, q_all_layers, out_all_layers, reqs, batch, copy_budget_bytes, rule, decoded_mask, stats);
+}
+
+int32_t ps_reload_backlog(ps_ctx* ctx, int64_t* bytes_in_flight) {
+    if (!ctx || !bytes_in_flight) return PS_ERR_INVALID;
+    *bytes_in_flight = 0;
+    if (ctx->bk) return PS_OK;
+    int32_t rc = tracker_poll(ctx, ctx->t_scatter);
+    if (rc != PS_OK) return rc;
+    while (!ctx->reload_inflight.empty() && ctx->reload_inflight.front().first <= ctx->t_scatter.done)
+        ctx->reload_inflight.pop_front();
+    for (const auto& e : ctx->reload_inflight) *bytes_in_flight += e.second;
+    return PS_OK;
 }
 
 int32_t ps_step_host(ps_ctx* ctx, const void* q_host, void* out_host, const int64_t* reqs, int32_t batch,

@@ -54,6 +54,7 @@ class LoopParams:
     fill_frac: float = 0.9           # device pool share filled before the first round
     host_budget_bytes: int = 12 << 30   # host images the stub plans with
     max_batch: int = 256
+    subtract_backlog: bool = True    # take reload copies still in flight off the next step's budget
 
 
 def config4_params(**over) -> LoopParams:
@@ -134,6 +135,9 @@ class LibBackend:
 
     def free_blocks(self) -> int:
         return self.lib.num_free_blocks()
+
+    def reload_backlog(self) -> int:
+        return self.lib.reload_backlog()
 
 
 @dataclass
@@ -292,6 +296,12 @@ class SchedulerStub:
             holders += 1
         # GetCopyBudget, then the step: ConsumeCopyBudget under SatisfyCopyCondition, reload, attention
         blocks, nbytes, case = be.copy_budget(queue, p, t_budget)
+        if p.subtract_backlog:
+            # GetCopyBudget assumes the previous steps' transfers have ended; what is still in flight (the link ran
+            # below the profiled t_block) comes off this step's budget, so the copy queue cannot grow without bound
+            backlog_blocks = -(-be.reload_backlog() // self.block_bytes)
+            blocks = max(0, blocks - backlog_blocks)
+            nbytes = blocks * self.block_bytes
         batch = [r for r in queue if states[r] in (B.PS_REQ_RESIDENT, B.PS_REQ_SWAPPING_IN)][: p.max_batch]
         rule = {}
         for rid in batch:

@@ -104,6 +104,9 @@ class PairedBackend:
         assert a == self.book.missing_blocks(rid)
         return a
 
+    def reload_backlog(self):
+        return self.lib.reload_backlog()                  # timing information: an input to both sides, not compared
+
     def free_blocks(self):
         a = self.lib.num_free_blocks()
         assert a == self.book.num_free_blocks()
