@@ -124,7 +124,8 @@ struct BatchMeta {  // cached device metadata of the last prepared decode batch
     int32_t n_items = 0, n_ungated_items = 0, n_parts = 0;
     int32_t n_gated_rows = 0;
     bool any_multi = false, lane_multi[2] = {false, false};
-    bool two_lanes = false, contended = false;
+    bool two_lanes = false;
+    int tail_mode = 0;
     int64_t kv_bytes_per_layer = 0;
 };
 
@@ -284,7 +285,7 @@ int32_t missing_of(const Req& r);
 // copy-budget consumption and the attention batch (ps_step.cu)
 std::vector<PlanEntry> make_plan(ps_ctx* ctx, int64_t copy_budget_bytes, const ps_copy_rule* rule);
 int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::vector<char>& active,
-                      const std::vector<char>& gated, bool want_lanes, bool contended);
+                      const std::vector<char>& gated, bool want_lanes, int tail_mode);
 int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, float* lse, cudaEvent_t wait_event,
                           bool follows_own, int32_t* n_launched);
 

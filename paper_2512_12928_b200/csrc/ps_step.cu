@@ -69,14 +69,14 @@ int32_t choose_split(const ps_ctx* ctx, int64_t total_tokens) {
 // the layer's reload event.  With want_lanes they get a work list of their own (lane 1), launched on
 // the reload-lane stream behind the event, so that the launches of the other rows never wait.
 int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::vector<char>& active,
-                      const std::vector<char>& gated, bool want_lanes, bool contended) {
+                      const std::vector<char>& gated, bool want_lanes, int tail_mode) {
     BatchMeta& m = ctx->meta;
     // two work lists (lanes) only for the tensor-core kernel and only when some row is gated
     bool two_lanes = false;
     if (want_lanes && ctx->attn_kernel == PS_ATTN_MMA)
         for (int32_t b = 0; b < B; ++b) two_lanes |= active[b] && gated[b];
     if (m.valid && m.epoch == ctx->table_epoch && (int32_t)m.reqs.size() == B && m.two_lanes == two_lanes &&
-        m.contended == contended &&
+        m.tail_mode == tail_mode &&
         std::equal(m.reqs.begin(), m.reqs.end(), reqs) && m.gated == gated && m.active == active)
         return PS_OK;
 
@@ -122,11 +122,14 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
         } else {
             // Tensor-core kernel: the lane's 16-token tiles form one sequence, cut into equal static shares,
             // one per CTA: every CTA streams the same number of bytes whatever the context-length mix, and
-            // only the rows cut by share borders need combining.  When reload traffic runs beside the step
-            // (scatter kernels and the reload lane take SM time unevenly) the last 5 % of the tiles become
-            // chunks that the CTAs take dynamically; without contention such a tail only costs (more parts
-            // to combine, a last round of chunks that does not fill the machine): 172 against 189 us per
-            // 1 GiB launch.  An item is the part of a row that falls into one share or chunk.
+            // only the rows cut by share borders need combining.  With tail_mode 1 (reload traffic beside the
+            // step: scatter kernels and the reload lane take SM time unevenly) the last 5 % of the sequence
+            // become chunks that the CTAs take dynamically through an atomic counter.  Without contention a
+            // dynamic part only costs: every chunk is one more partial result to write and combine (172
+            // against 189 us per 1 GiB launch for a 5 % tail; handing out the last 3 % of every share instead,
+            // 148 small chunks at share borders, took an isolated 537 MB launch from 89 to 93 us), so launches
+            // on their own keep equal static shares.  An item is the part of a row that falls into one share
+            // or chunk.
             const ps::AttnShape shape{ctx->cfg.num_kv_heads, ctx->cfg.num_q_heads, ctx->cfg.head_dim, ctx->cfg.block_size,
                                       ctx->cfg.num_gpu_blocks};
             const int kTile = ps::attn_mma_tile_tokens(shape);
@@ -145,62 +148,57 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
                 n_cta = std::min<int64_t>(std::max<int64_t>((total_tiles + kMinTilesPerCta - 1) / kMinTilesPerCta, 1),
                                           ctx->num_sms);
             int64_t dyn_tiles = 0, chunk = 0;
-            if (contended && n_cta > 0 && total_tiles >= 32 * n_cta) {
+            if (tail_mode == 1 && n_cta > 0 && total_tiles >= 32 * n_cta) {
                 dyn_tiles = total_tiles * 5 / 100;
                 chunk = std::max<int64_t>(kDynMinChunk, (dyn_tiles + kDynChunksPerCta * n_cta - 1) / (kDynChunksPerCta * n_cta));
             }
             const int64_t static_tiles = total_tiles - dyn_tiles;
             const int64_t per = n_cta > 0 ? std::max<int64_t>((static_tiles + n_cta - 1) / n_cta, 1) : 1;
-            // walk the rows; `pos` is the position in the lane's tile sequence
-            int64_t pos = 0, filled = 0;       // filled: tiles in the current share or chunk
-            bool in_dyn = false;
-            if (n_cta > 0) cta_begin[pass].push_back((int32_t)items.size());
-            auto close_static = [&]() {        // pad the share list and mark where the dynamic chunks start
-                while ((int64_t)cta_begin[pass].size() < n_cta + 1) cta_begin[pass].push_back((int32_t)items.size());
-                in_dyn = true;
-                filled = 0;
+            // Owner of sequence position pos: a CTA (its static share) or -1 (dynamic); *bound = where that ends.
+            auto owner_at = [&](int64_t pos, int64_t* bound) -> int64_t {
+                if (pos >= static_tiles) {  // tail_mode 1: chunks of the sequence's end
+                    const int64_t k = (pos - static_tiles) / chunk;
+                    *bound = std::min(total_tiles, static_tiles + (k + 1) * chunk);
+                    return -1;
+                }
+                const int64_t c = std::min(pos / per, n_cta - 1);
+                *bound = std::min((c + 1) * per, static_tiles);
+                return c;
             };
+            struct Piece {
+                ps::AttnItem it;
+                int64_t owner;
+            };
+            std::vector<Piece> pieces;  // in sequence order
+            int64_t pos = 0;
             for (int32_t b = 0; b < B; ++b) {
                 if (!active[b] || (two_lanes && (gated[b] ? 1 : 0) != pass)) continue;
                 const Req& r = ctx->reqs[reqs[b]];
                 const int64_t tiles_b = (r.n_tokens + kTile - 1) / kTile;
-                const size_t first_item = items.size();
+                const size_t first_piece = pieces.size();
                 ctx_len[b] = r.n_tokens;
                 row_first[b] = parts;
                 if (tiles_b == 0) {  // empty context: one item without tiles writes the zero row
                     ps::AttnItem it{};
                     it.b = b;
-                    items.push_back(it);
+                    pieces.push_back({it, std::min(pos / per, n_cta - 1)});
                 }
                 for (int64_t lo = 0; lo < tiles_b;) {
-                    if (!in_dyn && pos >= static_tiles) close_static();
-                    int64_t room;
-                    if (!in_dyn) {
-                        if (filled == per && (int64_t)cta_begin[pass].size() < n_cta) {
-                            cta_begin[pass].push_back((int32_t)items.size());
-                            filled = 0;
-                        }
-                        room = std::min(per - filled, static_tiles - pos);
-                    } else {
-                        if (filled == chunk) filled = 0;
-                        room = chunk - filled;
-                    }
-                    const int64_t take = std::min(tiles_b - lo, std::max<int64_t>(room, 1));
+                    int64_t bound = 0;
+                    const int64_t owner = owner_at(pos, &bound);
+                    const int64_t take = std::min(tiles_b - lo, std::max<int64_t>(bound - pos, 1));
                     ps::AttnItem it{};
                     it.b = b;
                     it.t_begin = (int32_t)(lo * kTile);
                     it.t_end = (int32_t)std::min<int64_t>(r.n_tokens, (lo + take) * kTile);
-                    items.push_back(it);
+                    pieces.push_back({it, owner});
                     lo += take;
                     pos += take;
-                    // a dynamic chunk never spans two rows: every item of the tail is its own chunk
-                    filled = in_dyn ? chunk : filled + take;
-                    if (in_dyn && take < chunk && lo < tiles_b) filled = chunk;
                 }
-                const int32_t n = (int32_t)(items.size() - first_item);
-                for (size_t k = first_item; k < items.size(); ++k) {
-                    items[k].part = parts + (int32_t)(k - first_item);
-                    items[k].n_parts = n;
+                const int32_t n = (int32_t)(pieces.size() - first_piece);
+                for (size_t k = first_piece; k < pieces.size(); ++k) {
+                    pieces[k].it.part = parts + (int32_t)(k - first_piece);
+                    pieces[k].it.n_parts = n;
                 }
                 row_parts[b] = n;
                 parts += n;
@@ -208,7 +206,25 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
                 lane_multi[pass] |= n > 1;
                 if (gated[b]) ++n_gated_rows;
             }
-            if (n_cta > 0 && !in_dyn) close_static();
+            // the lane's item list: the static items CTA by CTA (their owners never decrease along the sequence),
+            // then the dynamic ones in sequence order
+            if (n_cta > 0) {
+                int64_t next_cta = 0;
+                for (const Piece& pc : pieces) {
+                    if (pc.owner < 0) continue;
+                    while (next_cta <= pc.owner) {
+                        cta_begin[pass].push_back((int32_t)items.size());
+                        ++next_cta;
+                    }
+                    items.push_back(pc.it);
+                }
+                while (next_cta <= n_cta) {  // CTAs without items, and entry n_cta: where the dynamic items start
+                    cta_begin[pass].push_back((int32_t)items.size());
+                    ++next_cta;
+                }
+                for (const Piece& pc : pieces)
+                    if (pc.owner < 0) items.push_back(pc.it);
+            }
         }
         if (pass == 0) n_ungated = (int32_t)items.size();
     }
@@ -258,7 +274,7 @@ int32_t prepare_batch(ps_ctx* ctx, const int64_t* reqs, int32_t B, const std::ve
     m.gated = gated;
     m.active = active;
     m.two_lanes = two_lanes;
-    m.contended = contended;
+    m.tail_mode = tail_mode;
     m.epoch = ctx->table_epoch;
     m.valid = true;
     m.dev.block_tables = (const int32_t*)d;
@@ -368,7 +384,7 @@ int32_t ps_decode_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, flo
     }
     std::vector<char> active((size_t)batch, 1), gated((size_t)batch, 0);
     for (int32_t b = 0; b < batch; ++b) gated[(size_t)b] = ctx->reqs[reqs[b]].gated ? 1 : 0;
-    int32_t rc = prepare_batch(ctx, reqs, batch, active, gated, /*want_lanes=*/false, /*contended=*/false);
+    int32_t rc = prepare_batch(ctx, reqs, batch, active, gated, /*want_lanes=*/false, /*tail_mode=*/0);
     if (rc != PS_OK) return rc;
     int32_t launched = 0;
     return launch_layer_attn(ctx, layer, q, out, lse,
@@ -430,7 +446,7 @@ static int32_t step_impl(ps_ctx* ctx, const void* q_all_layers, void* out_all_la
         // a reload of 32 MiB or more per step slows SMs unevenly enough for a dynamic tail to pay off
         const bool pipelined = (ctx->cfg.flags & PS_FLAG_SYNC_RELOAD) == 0;
         rc = prepare_batch(ctx, reqs, batch, active, gated, pipelined,
-                           /*contended=*/pipelined && st.h2d_bytes >= (32LL << 20));
+                           /*tail_mode=*/pipelined && st.h2d_bytes >= (32LL << 20) ? 1 : 0);
         if (rc != PS_OK) return rc;
         st.gated = ctx->meta.n_gated_rows;
     }
