@@ -1063,6 +1063,7 @@ def run_gpu(args):
            "h2d_bytes_per_step": int(victim_bytes + io_bytes), "d2h_bytes_per_step": int(victim_bytes + io_bytes),
            "api": "ps_step_host: queries from and outputs to pinned host memory through the C ABI, every decode step",
            "decode_steps_per_pass": sum(r["steps_out"] + r["steps_in"] for r in e2e_recs) / len(e2e_recs),
+           "decode_step_us_during_swap_out": sum(r["out_ms"] for r in e2e_recs) / sum(r["steps_out"] for r in e2e_recs) * 1e3,
            "note": "bytes per step = the swapped KV each way (host images live in pinned host memory by "
                    "definition) + the queries (up) / outputs (down) of every decode step: 48 rows while the "
                    "offload drains, 64 rows in the reload step"}

@@ -392,7 +392,9 @@ int32_t ps_reload_backlog(ps_ctx* ctx, int64_t* bytes_in_flight);
  * context on the compute stream, runs the step, and copies the outputs back, all asynchronously on the compute
  * stream (synchronise that stream, or call ps_sync, before reading out_host).
  *   q_host, out_host : host, bf16 [num_layers][batch][num_q_heads][head_dim]; pinned memory keeps the copies
- *                      asynchronous.  Rows of out_host whose request did not decode are zero.
+ *                      asynchronous.  Rows of out_host whose request did not decode are zero.  Into pinned
+ *                      memory the outputs are stored by a kernel, not by a copy engine, so that a step never
+ *                      waits behind the device-to-host copies of an offload in flight.
  * The context's two device buffers ([num_layers][max_batch][num_q_heads][head_dim] each) are allocated by the
  * first call.  Errors: those of ps_step; PS_ERR_INVALID (batch 0, null buffers, bookkeeping-only context). */
 int32_t ps_step_host(ps_ctx* ctx, const void* q_host, void* out_host, const int64_t* reqs, int32_t batch,

@@ -20,9 +20,9 @@ cudaError_t launch_image_copy(bool scatter, void* const* d_kpools, void* const* 
                               int32_t n, int32_t layer0, int64_t slab_begin, int64_t slab_count, void* staging,
                               int32_t slab_vec, int32_t num_blocks, int32_t* d_status, cudaStream_t stream);
 
-// Copies `bytes` (a multiple of 16) from mapped pinned host memory (device view src) to device
-// memory with a small kernel, so that descriptor uploads never queue behind bulk transfers in a
-// copy engine.
+// Copies `bytes` (a multiple of 16) between device-addressable ranges with a small kernel: from mapped
+// pinned host memory (device view src) to device memory, so that descriptor uploads never queue behind
+// bulk transfers in a copy engine, or from device memory into pinned host memory (results of a step).
 cudaError_t launch_upload(void* dst, const void* src_mapped, size_t bytes, cudaStream_t stream);
 
 // Streams `bytes` (a multiple of 16) of src with `ctas` CTAs of 256 threads: read-only (every thread folds what

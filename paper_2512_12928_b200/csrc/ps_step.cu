@@ -587,7 +587,18 @@ int32_t ps_step_host(ps_ctx* ctx, const void* q_host, void* out_host, const int6
     CK(cudaMemsetAsync(ctx->io_out, 0, bytes, ctx->compute));
     int32_t rc = step_impl(ctx, ctx->io_q, ctx->io_out, reqs, batch, copy_budget_bytes, nullptr, decoded_mask, stats);
     if (rc != PS_OK) return rc;
-    CK(cudaMemcpyAsync(out_host, ctx->io_out, bytes, cudaMemcpyDeviceToHost, ctx->compute));
+    // The outputs go back through a small kernel that stores into the pinned buffer (16-byte coalesced stores
+    // over the host link) when the device can address it: a copy-engine transfer would queue behind every
+    // device-to-host copy already submitted, i.e. behind a whole offload in flight, and hold the step for
+    // its duration.  Pageable memory takes the copy engine.
+    void* out_dev = nullptr;
+    if (bytes % 16 == 0 && cudaHostGetDevicePointer(&out_dev, out_host, 0) == cudaSuccess && out_dev != nullptr) {
+        CK(ps::launch_upload(out_dev, ctx->io_out, bytes, ctx->compute));
+        ctx->launches++;
+    } else {
+        cudaGetLastError();
+        CK(cudaMemcpyAsync(out_host, ctx->io_out, bytes, cudaMemcpyDeviceToHost, ctx->compute));
+    }
     return PS_OK;
 }
 
