@@ -21,7 +21,7 @@
  *     partially applied (allocation is all-or-nothing).  No function throws or aborts.
  *   - "device pointer" = address in the memory of the CUDA device that was current when
  *     ps_create was called; "host pointer" = ordinary process memory unless it says pinned.
- *   - One caller thread per context.  All GPU work is asynchronous with respect to the host
+ *   - One caller thread per context (the context runs one worker thread of its own, for offloads).  All GPU work is asynchronous with respect to the host
  *     unless a function says it waits.  Asynchronous CUDA failures surface as PS_ERR_CUDA (and
  *     kernel-side id checks as PS_ERR_BOUNDS, a kernel-side wait that ran out as PS_ERR_TIMEOUT) from the
  *     next ps_poll / ps_sync / ps_step.
@@ -199,6 +199,11 @@ int32_t ps_num_free_blocks(ps_ctx* ctx, int32_t* out);
  * its blocks.  When a later ps_poll / ps_step / ps_sync finds the transfer complete (offloads
  * complete in issue order) the blocks are pushed back to the pool and the state becomes HOST.
  * Blocks already covered by ps_offload_progress are not copied again.
+ * The copies are handed to the copy engine by a worker thread of the context, two staging slots at a time
+ * (Section 4.3: a separate thread copies the accumulated blocks).  The engine serves device-to-host copies in
+ * submission order whatever their stream, so an offload submitted whole would hold every later copy of the
+ * process -- a step's results, sampled tokens -- for its full duration; paced, such a copy waits behind at most
+ * two slots.  A failure inside the worker surfaces as PS_ERR_CUDA from the next ps_poll / ps_step / ps_sync.
  * Errors: PS_ERR_STATE, PS_ERR_HOST_NOMEM, PS_ERR_INVALID, PS_ERR_CUDA. */
 int32_t ps_swap_out(ps_ctx* ctx, int64_t req);
 

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <algorithm>
+#include <atomic>
 #include <chrono>
 #include <cmath>
 #include <cstdio>
@@ -9,6 +10,8 @@
 #include <cstring>
 #include <deque>
 #include <map>
+#include <mutex>
+#include <condition_variable>
 #include <string>
 #include <thread>
 #include <unordered_map>
@@ -50,6 +53,21 @@ struct Tracker {  // completion tickets on one stream
     cudaStream_t s = nullptr;
     std::deque<std::pair<uint64_t, cudaEvent_t>> pending;
     uint64_t next = 1, done = 0;
+    // via_worker: tickets are numbered by the caller but their events are recorded by the offload worker when it
+    // reaches them in its queue; `pending` is then shared between the two threads (under mu), `next` and `done`
+    // stay with the caller's thread
+    bool via_worker = false;
+    std::mutex mu;
+};
+
+// One unit of offload work handed to the worker: a staging slot's worth of an image (gather + copy), and / or
+// a completion ticket to record on the D2H stream behind everything issued before it.
+struct OutChunk {
+    const int32_t* d_table = nullptr;
+    int32_t n_blk = 0;
+    int64_t s0 = 0, cnt = 0;     // slabs [s0, s0 + cnt) of the segment's image; cnt = 0: ticket only
+    char* host_dst = nullptr;
+    uint64_t ticket = 0;         // != 0: record this ticket's event after the chunk's copy
 };
 
 struct Arena {  // pinned (mapped) + device ring of chunks for descriptor uploads on ONE stream
@@ -197,8 +215,21 @@ struct ps_ctx {
     char* io_q = nullptr;    // ps_step_host: device copies of the queries and of the outputs (allocated on first use)
     char* io_out = nullptr;
 
+    // offload worker (Section 4.3 "Asynchronous Offloading": a separate thread copies the blocks): hands the
+    // copy engine at most kOutInflight staging slots at a time, so that other device-to-host copies of the
+    // process queue behind that much and not behind a whole offload
+    bool out_paced = false;
+    int device = 0;
+    std::thread out_thread;
+    std::mutex out_mu;
+    std::condition_variable out_cv;
+    std::deque<OutChunk> out_pending;
+    bool out_stop = false;
+    std::atomic<bool> out_failed{false};
+    std::string out_error;
+
     // measurement
-    int64_t launches = 0;
+    std::atomic<int64_t> launches{0};
     std::vector<ProfSpan> spans;
     double prof_ms[kProfKinds]{};
     int64_t prof_n[kProfKinds]{};
@@ -246,7 +277,9 @@ struct ProfScope {
     cudaEvent_t e0 = nullptr;
     bool on = false;
     int tag;
-    ProfScope(ps_ctx* c, int k, cudaStream_t st, int64_t bytes, int tg = -1) : ctx(c), kind(k), s(st), tag(tg) {
+    ProfScope(ps_ctx* c, int k, cudaStream_t st, int64_t bytes, int tg = -1, bool enabled = true)
+        : ctx(c), kind(k), s(st), tag(tg) {
+        if (!enabled) return;  // the offload worker's thread keeps out of the profiling state
         ctx->prof_bytes[kind] += bytes;
         ctx->prof_n[kind] += 1;
         if (ctx->profile && !ctx->bk && get_event(ctx, true, &e0) == cudaSuccess) {
@@ -273,6 +306,11 @@ int32_t check_status_word(ps_ctx* ctx);
 // finished offloads give their blocks back in ps_poll / ps_step / ps_sync alone, which report how many, so a
 // caller can follow the free-block count exactly.
 int32_t do_poll(ps_ctx* ctx, int32_t* n_reaped, bool reap_offloads = true);
+
+// offload worker (ps_swap.cu)
+constexpr int kOutInflight = 2;
+void out_worker_main(ps_ctx* ctx);
+cudaError_t issue_out_chunk(ps_ctx* ctx, const OutChunk& c, int slot, bool profiled);
 
 // swap-out and swap-in issue (ps_swap.cu)
 int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi);

@@ -40,6 +40,16 @@ int32_t tracker_mark(ps_ctx* ctx, Tracker& t, uint64_t* ticket) {
         t.done = *ticket;
         return PS_OK;
     }
+    if (t.via_worker) {  // the worker records the event when it reaches this point of its queue
+        OutChunk c;
+        c.ticket = *ticket;
+        {
+            std::lock_guard<std::mutex> lk(ctx->out_mu);
+            ctx->out_pending.push_back(c);
+        }
+        ctx->out_cv.notify_one();
+        return PS_OK;
+    }
     cudaEvent_t ev;
     CK(get_event(ctx, false, &ev));
     CK(cudaEventRecord(ev, t.s));
@@ -48,6 +58,8 @@ int32_t tracker_mark(ps_ctx* ctx, Tracker& t, uint64_t* ticket) {
 }
 
 int32_t tracker_poll(ps_ctx* ctx, Tracker& t) {
+    std::unique_lock<std::mutex> lk(t.mu, std::defer_lock);
+    if (t.via_worker) lk.lock();
     while (!t.pending.empty()) {
         cudaError_t e = cudaEventQuery(t.pending.front().second);
         if (e == cudaErrorNotReady) break;
@@ -59,15 +71,23 @@ int32_t tracker_poll(ps_ctx* ctx, Tracker& t) {
     return PS_OK;
 }
 
-// Waits until every ticket of the tracker is complete or the deadline passes.
+// Waits until every ticket handed out so far is complete or the deadline passes.
 int32_t tracker_drain(ps_ctx* ctx, Tracker& t, bool bounded, std::chrono::steady_clock::time_point deadline) {
-    while (!t.pending.empty()) {
-        if (!bounded) {
-            CK(cudaEventSynchronize(t.pending.back().second));
+    while (t.done + 1 < t.next) {
+        cudaEvent_t last = nullptr;
+        {
+            std::unique_lock<std::mutex> lk(t.mu, std::defer_lock);
+            if (t.via_worker) lk.lock();
+            if (!t.pending.empty()) last = t.pending.back().second;
         }
+        if (!bounded && last != nullptr) CK(cudaEventSynchronize(last));
         int32_t rc = tracker_poll(ctx, t);
         if (rc != PS_OK) return rc;
-        if (t.pending.empty()) break;
+        if (t.done + 1 >= t.next) break;
+        if (t.via_worker && ctx->out_failed.load()) {
+            std::lock_guard<std::mutex> lk(ctx->out_mu);
+            return ctx->fail(PS_ERR_CUDA, "offload worker: " + ctx->out_error);
+        }
         if (bounded && std::chrono::steady_clock::now() > deadline) return ctx->fail(PS_ERR_TIMEOUT, "ps_sync timed out");
         std::this_thread::sleep_for(std::chrono::microseconds(50));
     }
@@ -220,10 +240,22 @@ int32_t do_poll(ps_ctx* ctx, int32_t* n_reaped, bool reap_offloads) {
     rc = tracker_poll(ctx, ctx->t_compute);
     if (rc != PS_OK) return rc;
     if (n_reaped) *n_reaped = reaped;
+    if (ctx->out_failed.load()) {
+        std::lock_guard<std::mutex> lk(ctx->out_mu);
+        return ctx->fail(PS_ERR_CUDA, "offload worker: " + ctx->out_error);
+    }
     return check_status_word(ctx);
 }
 
 void destroy_ctx(ps_ctx* ctx) {
+    if (ctx->out_thread.joinable()) {
+        {
+            std::lock_guard<std::mutex> lk(ctx->out_mu);
+            ctx->out_stop = true;
+        }
+        ctx->out_cv.notify_all();
+        ctx->out_thread.join();
+    }
     if (!ctx->bk) {
         for (cudaStream_t s : {ctx->s_gather, ctx->s_d2h, ctx->s_h2d, ctx->s_scatter, ctx->s_lane})
             if (s) cudaStreamDestroy(s);
@@ -389,6 +421,7 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     // the reload lane: attention of the requests whose reload lands in this step, behind the per-layer events;
     // its few CTAs should get an SM as soon as one frees up
     CKC(cudaStreamCreateWithPriority(&ctx->s_lane, cudaStreamNonBlocking, prio_hi));
+    CKC(cudaGetDevice(&ctx->device));
     ctx->t_d2h.s = ctx->s_d2h;
     ctx->t_scatter.s = ctx->s_scatter;
     ctx->t_compute.s = ctx->compute;
@@ -489,6 +522,12 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
     }
 #undef CKC
 #undef CKR
+    // the offload worker; contexts that time every launch issue their offloads on the caller's thread instead
+    if (!ctx->profile) {
+        ctx->out_paced = true;
+        ctx->t_d2h.via_worker = true;
+        ctx->out_thread = std::thread(out_worker_main, ctx);
+    }
     *out = ctx;
     return PS_OK;
 }
@@ -600,7 +639,7 @@ int32_t ps_sync(ps_ctx* ctx, int32_t timeout_ms) {
 
 int32_t ps_launch_count(ps_ctx* ctx, int64_t* out) {
     if (!ctx || !out) return PS_ERR_INVALID;
-    *out = ctx->launches;
+    *out = ctx->launches.load();
     return PS_OK;
 }
 

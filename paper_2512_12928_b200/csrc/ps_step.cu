@@ -421,7 +421,7 @@ static int32_t step_impl(ps_ctx* ctx, const void* q_all_layers, void* out_all_la
     }
     st.h2d_bytes = st.blocks_copied * ctx->block_bytes;
     const int L = ctx->cfg.num_layers;
-    const int64_t launches_before = ctx->launches;
+    const int64_t launches_before = ctx->launches.load();
 
     // 2. the decode set: resident now, or made complete by this step's reload (those wait on events)
     std::vector<char> active((size_t)batch, 0), gated((size_t)batch, 0);
@@ -536,7 +536,7 @@ static int32_t step_impl(ps_ctx* ctx, const void* q_all_layers, void* out_all_la
                 if (it != ctx->reqs.end()) it->second.gated = false;
             }
     }
-    st.kernel_launches = (int32_t)(ctx->launches - launches_before);
+    st.kernel_launches = (int32_t)(ctx->launches.load() - launches_before);
     if (stats) *stats = st;
     return PS_OK;
 }

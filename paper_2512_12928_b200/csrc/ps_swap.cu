@@ -174,6 +174,82 @@ int32_t missing_of(const Req& r) {
     return (int32_t)r.table.size() - mn;
 }
 
+// Gathers one staging slot's worth of an image and copies it to the host (slot -> host on the D2H stream).
+cudaError_t issue_out_chunk(ps_ctx* ctx, const OutChunk& c, int slot, bool profiled) {
+    char* sp = ctx->stage_out + (int64_t)slot * ctx->slot_bytes;
+    cudaError_t e = cudaSuccess;
+    if (ctx->out_used[slot]) e = cudaStreamWaitEvent(ctx->s_gather, ctx->e_drained[slot], 0);
+    if (e != cudaSuccess) return e;
+    const int64_t bytes = c.cnt * ctx->slab_bytes;
+    {
+        ProfScope prof(ctx, kProfGather, ctx->s_gather, profiled ? bytes : 0, -1, profiled);
+        e = ps::launch_image_copy(/*scatter=*/false, ctx->d_kpools, ctx->d_vpools, c.d_table, c.n_blk, 0, c.s0, c.cnt, sp,
+                                  ctx->slab_vec, ctx->cfg.num_gpu_blocks, ctx->d_status, ctx->s_gather);
+        ctx->launches++;
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->e_gathered[slot], ctx->s_gather);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_d2h, ctx->e_gathered[slot], 0);
+    if (e != cudaSuccess) return e;
+    {
+        ProfScope prof(ctx, kProfD2H, ctx->s_d2h, profiled ? bytes : 0, -1, profiled);
+        e = cudaMemcpyAsync(c.host_dst, sp, (size_t)bytes, cudaMemcpyDeviceToHost, ctx->s_d2h);
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(ctx->e_drained[slot], ctx->s_d2h);
+    if (e == cudaSuccess) ctx->out_used[slot] = true;
+    return e;
+}
+
+// The offload worker: takes chunks in issue order and keeps at most kOutInflight of them with the copy engine.
+// The copy engine serves device-to-host copies in the order they were submitted, whatever their stream, so an
+// offload submitted whole would hold every later copy of the process (a step's results, sampled tokens) for its
+// full duration.  Completion tickets are recorded here too, behind the chunks queued before them.
+void out_worker_main(ps_ctx* ctx) {
+    cudaSetDevice(ctx->device);
+    std::deque<int> inflight;  // slots whose copy has been submitted, oldest first
+    for (;;) {
+        OutChunk c;
+        {
+            std::unique_lock<std::mutex> lk(ctx->out_mu);
+            ctx->out_cv.wait(lk, [&] { return ctx->out_stop || !ctx->out_pending.empty(); });
+            if (ctx->out_stop) return;
+            c = ctx->out_pending.front();
+            ctx->out_pending.pop_front();
+        }
+        cudaError_t e = cudaSuccess;
+        const char* what = "";
+        if (c.cnt > 0 && !ctx->out_failed.load()) {
+            if ((int)inflight.size() >= kOutInflight) {
+                e = cudaEventSynchronize(ctx->e_drained[inflight.front()]);
+                what = "waiting for a staging slot to drain";
+                inflight.pop_front();
+            }
+            if (e == cudaSuccess) {
+                const int slot = (int)(ctx->out_next++ % kSlots);
+                e = issue_out_chunk(ctx, c, slot, /*profiled=*/false);
+                what = "offload chunk (gather + device-to-host copy)";
+                inflight.push_back(slot);
+            }
+        }
+        if (c.ticket != 0) {  // recorded even after a failure, so that waits on the ticket end
+            cudaEvent_t ev = nullptr;
+            cudaError_t e2 = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+            if (e2 == cudaSuccess) e2 = cudaEventRecord(ev, ctx->s_d2h);
+            if (e2 == cudaSuccess) {
+                std::lock_guard<std::mutex> lk(ctx->t_d2h.mu);
+                ctx->t_d2h.pending.emplace_back(c.ticket, ev);
+            } else if (e == cudaSuccess) {
+                e = e2;
+                what = "recording an offload's completion event";
+            }
+        }
+        if (e != cudaSuccess && !ctx->out_failed.load()) {
+            std::lock_guard<std::mutex> lk(ctx->out_mu);
+            ctx->out_error = std::string(what) + ": " + cudaGetErrorString(e);
+            ctx->out_failed.store(true);
+        }
+    }
+}
+
 // Starts the offload of logical blocks [lo, hi) of a request as a new image segment: gather through the
 // table into staging slots, slot by slot to the host.  Ordered after everything already enqueued on the
 // compute stream (and after the scatters of a reload that is still landing).
@@ -187,7 +263,13 @@ int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi) {
         off = ctx->hpool.alloc(bytes);
     }
     if (off < 0) return ctx->fail(PS_ERR_HOST_NOMEM, "host pool cannot hold the image");
+    if (ctx->out_failed.load()) {
+        ctx->hpool.release(off, bytes);
+        std::lock_guard<std::mutex> lk(ctx->out_mu);
+        return ctx->fail(PS_ERR_CUDA, "an earlier offload failed: " + ctx->out_error);
+    }
 
+    std::vector<OutChunk> chunks;
     if (!ctx->bk && n_blk > 0) {
         cudaError_t e = cudaEventRecord(ctx->e_mark2, ctx->compute);
         if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_gather, ctx->e_mark2, 0);
@@ -203,59 +285,65 @@ int32_t offload_segment(ps_ctx* ctx, Req& r, int32_t lo, int32_t hi) {
             return rc;
         }
         memcpy(ctx->a_gather.h + toff, r.table.data() + lo, (size_t)n_blk * 4);
-        // On a failure after the first copy into the range was enqueued, the range must not be handed out
-        // again before those copies have ended: it is parked behind a ticket of the D2H stream.
-        bool copies_enqueued = false;
-        auto bail = [&](cudaError_t ce, const char* what) {
-            uint64_t ticket = 0;
-            if (!copies_enqueued)
-                ctx->hpool.release(off, bytes);
-            else if (tracker_mark(ctx, ctx->t_d2h, &ticket) == PS_OK)
-                ctx->host_release.push_back({ticket, {off, bytes}});
-            // (if not even the ticket could be recorded the range stays reserved: a leak, never a reuse)
-            return ctx->fail_cuda(ce, what);
-        };
         e = ps::launch_upload(ctx->a_gather.d + toff, ctx->a_gather.hd + toff, (size_t)round_up(n_blk * 4, 16),
                               ctx->s_gather);
         ctx->launches++;
-        if (e != cudaSuccess) return bail(e, "table upload");
+        if (e != cudaSuccess) {
+            ctx->hpool.release(off, bytes);
+            return ctx->fail_cuda(e, "table upload");
+        }
         const int64_t total_slabs = 2 * n_blk * ctx->cfg.num_layers;
         const int64_t slot_slabs = ctx->slot_bytes / ctx->slab_bytes;
         for (int64_t s0 = 0; s0 < total_slabs; s0 += slot_slabs) {
-            const int64_t cnt = std::min(slot_slabs, total_slabs - s0);
-            const int slot = (int)(ctx->out_next++ % kSlots);
-            char* sp = ctx->stage_out + (int64_t)slot * ctx->slot_bytes;
-            if (ctx->out_used[slot]) {
-                e = cudaStreamWaitEvent(ctx->s_gather, ctx->e_drained[slot], 0);
-                if (e != cudaSuccess) return bail(e, "slot wait");
-            }
-            {
-                ProfScope prof(ctx, kProfGather, ctx->s_gather, cnt * ctx->slab_bytes);
-                e = ps::launch_image_copy(/*scatter=*/false, ctx->d_kpools, ctx->d_vpools,
-                                          (const int32_t*)(ctx->a_gather.d + toff), (int32_t)n_blk, 0, s0, cnt, sp,
-                                          ctx->slab_vec, ctx->cfg.num_gpu_blocks, ctx->d_status, ctx->s_gather);
-                ctx->launches++;
-            }
-            if (e == cudaSuccess) e = cudaEventRecord(ctx->e_gathered[slot], ctx->s_gather);
-            if (e == cudaSuccess) e = cudaStreamWaitEvent(ctx->s_d2h, ctx->e_gathered[slot], 0);
-            if (e != cudaSuccess) return bail(e, "gather launch");
-            {
-                ProfScope prof(ctx, kProfD2H, ctx->s_d2h, cnt * ctx->slab_bytes);
-                e = cudaMemcpyAsync(ctx->host_pool + off + s0 * ctx->slab_bytes, sp, (size_t)(cnt * ctx->slab_bytes),
-                                    cudaMemcpyDeviceToHost, ctx->s_d2h);
-                copies_enqueued |= e == cudaSuccess;
-            }
-            if (e == cudaSuccess) e = cudaEventRecord(ctx->e_drained[slot], ctx->s_d2h);
-            if (e != cudaSuccess) return bail(e, "device-to-host copy");
-            ctx->out_used[slot] = true;
+            OutChunk c;
+            c.d_table = (const int32_t*)(ctx->a_gather.d + toff);
+            c.n_blk = (int32_t)n_blk;
+            c.s0 = s0;
+            c.cnt = std::min(slot_slabs, total_slabs - s0);
+            c.host_dst = ctx->host_pool + off + s0 * ctx->slab_bytes;
+            chunks.push_back(c);
         }
     }
     Req::Seg sg{lo, hi, off, bytes, 0};
-    int32_t rc = tracker_mark(ctx, ctx->t_d2h, &sg.ticket);
-    if (rc != PS_OK) {
-        // copies into the range may be in flight and there is no ticket to wait for: the range stays
-        // reserved until ps_destroy rather than being reused under them
-        return rc;
+    if (ctx->out_paced) {
+        // The block tables of queued chunks live in the descriptor ring, whose chunks are reused after a few MiB
+        // of newer tables: tables of pending chunks add up to less than the pool's ids plus 256 bytes per
+        // segment, so bounding the queue keeps them far from reuse.
+        for (;;) {
+            {
+                std::lock_guard<std::mutex> lk(ctx->out_mu);
+                if (ctx->out_pending.size() < 4096 || ctx->out_failed.load()) break;
+            }
+            std::this_thread::sleep_for(std::chrono::microseconds(100));
+        }
+        // the worker issues the chunks; the segment's ticket rides on the last one (or on an empty chunk)
+        sg.ticket = ctx->t_d2h.next++;
+        if (chunks.empty()) chunks.emplace_back();
+        chunks.back().ticket = sg.ticket;
+        {
+            std::lock_guard<std::mutex> lk(ctx->out_mu);
+            for (const OutChunk& c : chunks) ctx->out_pending.push_back(c);
+        }
+        ctx->out_cv.notify_one();
+    } else {
+        // issued here, slot after slot (contexts that time every launch, or hold no device)
+        bool copies_enqueued = false;
+        for (const OutChunk& c : chunks) {
+            const int slot = (int)(ctx->out_next++ % kSlots);
+            cudaError_t e = issue_out_chunk(ctx, c, slot, /*profiled=*/true);
+            if (e != cudaSuccess) {
+                // a range that copies already in flight write into is parked behind a ticket, never reused early
+                uint64_t ticket = 0;
+                if (!copies_enqueued)
+                    ctx->hpool.release(off, bytes);
+                else if (tracker_mark(ctx, ctx->t_d2h, &ticket) == PS_OK)
+                    ctx->host_release.push_back({ticket, {off, bytes}});
+                return ctx->fail_cuda(e, "offload chunk (gather + device-to-host copy)");
+            }
+            copies_enqueued = true;
+        }
+        int32_t rc = tracker_mark(ctx, ctx->t_d2h, &sg.ticket);
+        if (rc != PS_OK) return rc;  // the range stays reserved: copies may be in flight and nothing tells when they end
     }
     r.segs.push_back(sg);
     r.host_issued = hi;

@@ -256,3 +256,42 @@ def test_attention_with_early_set_up_matches_after_any_predecessor():
     assert p.lib.decode_attn(2, qd[2], out[2], reqs) == B.PS_OK
     torch.cuda.synchronize()
     check_attn(out[2], p.orc.decode_attn(2, q2[2], reqs)[0])
+
+
+def test_small_device_to_host_copies_do_not_wait_for_a_whole_offload():
+    """The copy engine serves device-to-host copies in submission order, whatever their stream.  The library's
+    offload worker therefore hands it two staging slots at a time: a small copy the caller makes right after
+    ps_swap_out (a step's result, sampled tokens) completes after those, not after the whole image.  The image
+    itself is byte-exact as ever."""
+    import time
+    L, nb = 16, 2200                                       # 16 layers x 64 KiB: 1 MiB per block
+    sh = wl.KVShape(L, 8, 8, 128, 16, nb)
+    g = torch.Generator(device="cuda"); g.manual_seed(5)
+    K = torch.empty((L, nb, 16, 8, 128), dtype=torch.bfloat16, device="cuda").normal_(generator=g)
+    V = torch.empty_like(K).normal_(generator=g)
+    lib = B.KVSwap(num_layers=L, num_kv_heads=8, num_q_heads=8, head_dim=128, block_size=16, num_gpu_blocks=nb,
+                   max_blocks_per_req=2100, max_batch=1, host_pool_bytes=(2048 + 64) << 20,
+                   k_pools=[K[l] for l in range(L)], v_pools=[V[l] for l in range(L)])
+    assert lib.kv_alloc(7, 2048 * 16) == B.PS_OK           # 2048 blocks = 2 GiB of KV: about 36 ms of host link
+    table = torch.tensor(lib.block_table(7)[0], device="cuda", dtype=torch.long)
+    small = torch.arange(4096, device="cuda", dtype=torch.int32)
+    host = torch.empty(4096, dtype=torch.int32).pin_memory()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    assert lib.swap_out(7) == B.PS_OK
+    host.copy_(small, non_blocking=True)
+    torch.cuda.current_stream().synchronize()
+    t_small = time.perf_counter() - t0
+    assert lib.sync() == B.PS_OK
+    t_all = time.perf_counter() - t0
+    assert torch.equal(host, small.cpu())
+    assert t_all > 0.025, t_all                            # the offload really took its tens of milliseconds
+    assert t_small < 0.5 * t_all, (t_small, t_all)         # and the small copy did not wait for it
+    # the image: layer-major, block by block through the table
+    ptr, nbytes = lib.host_image(7)
+    import ctypes as C
+    img = np.ctypeslib.as_array((C.c_uint16 * (nbytes // 2)).from_address(ptr)).reshape(L, 2048, 2, -1)
+    for l in (0, 7, L - 1):
+        assert np.array_equal(img[l][:, 0], dev_to_bits(K[l][table]).reshape(2048, -1))
+        assert np.array_equal(img[l][:, 1], dev_to_bits(V[l][table]).reshape(2048, -1))
+    lib.destroy()
