@@ -1,10 +1,11 @@
 """A seeded random mix of every state-changing call on the GPU (tensor-core attention shape), driven side by
 side with the CPU checker over identical pools: allocation and growth with fresh KV written on the compute
-stream, proactive and on-demand offloading, budgeted and unbudgeted reloads that interleave with decode
-steps, frees and cancels.  No host synchronisation is placed between dependent calls except where the
-checker needs the transfers' completion order (reaping offloads), so that any missing stream ordering in the
-library (a block reused while a kernel still reads it, a gather racing a write) shows up as a byte or
-attention mismatch."""
+stream, proactive and on-demand offloading, budgeted and unbudgeted reloads (with and without the
+partial-copy rule, in layer chunks of several sizes) that interleave with decode steps, frees and cancels.
+No host synchronisation is placed between dependent calls: offloads are still in flight when steps run, and
+the checker is told how many of them each step reaped (the library reports it), so that any missing stream
+ordering in the library (a block reused while a kernel still reads it, a gather racing a write) shows up as a
+byte or attention mismatch."""
 import numpy as np
 import pytest
 import torch
@@ -26,9 +27,10 @@ def test_random_script_with_data(seed, Hkv, Hq, S):
     rng = np.random.default_rng([2512, seed])
     K = wl.randn_bf16_bits(rng, (L, nb, S, Hkv, D))
     V = wl.randn_bf16_bits(rng, (L, nb, S, Hkv, D))
-    p = Pair(sh, rng.permutation(nb), K, V, max_batch=12, staging_bytes=2 << 20, max_blocks_per_req=64)
+    p = Pair(sh, rng.permutation(nb), K, V, max_batch=12, staging_bytes=2 << 20, max_blocks_per_req=64,
+             layer_chunk_bytes=[0, -1, 96 * 1024, 1 << 30][seed % 4])
     live, next_id = [], 0
-    decoded_steps = reloaded = 0
+    decoded_steps = reloaded = ruled_steps = reaped_by_steps = 0
 
     def write_fresh_kv(r, old_blocks):
         """New tokens of a growing request: random KV into its new blocks, enqueued on the compute stream."""
@@ -82,11 +84,21 @@ def test_random_script_with_data(seed, Hkv, Hq, S):
             q = wl.randn_bf16_bits(rng, (L, len(live), Hq, D))
             qd = bits_to_dev(q)
             out = torch.full_like(qd, 3.0)
-            if p.orc.out_fifo:
-                p.sync()                                         # the step reaps finished offloads: make "finished" definite
-            rc, mask, st = p.lib.step(qd, out, live, budget)
+            rule, beta = None, None
+            if rng.random() < 0.5:                               # the partial-copy test for the queued reloads
+                beta = 1.5
+                rule = {r: [(0, 1), (1, 1), (40, 64), (200, 64)][int(rng.integers(0, 4))]
+                        for r in live if p.orc.reqs[r].state == 4}
+                rr = sorted(rule)
+                rc, mask, st = p.lib.step_ruled(qd, out, live, budget, beta, rr, [rule[r][0] for r in rr],
+                                                [rule[r][1] for r in rr])
+                ruled_steps += 1
+            else:
+                rc, mask, st = p.lib.step(qd, out, live, budget)
             assert rc == B.PS_OK, p.lib.last_error()
-            plan, omask, want = p.orc.step(budget, live, q)
+            p.orc.reap(st["swapouts_reaped"])                    # offloads the step found complete, in issue order
+            reaped_by_steps += st["swapouts_reaped"]
+            plan, omask, want = p.orc.step(budget, live, q, rule=rule, beta=beta)
             assert mask == omask, it
             assert st["blocks_copied"] == sum(hi - lo for _, lo, hi in plan)
             reloaded += st["reloads_completed"]
@@ -105,4 +117,4 @@ def test_random_script_with_data(seed, Hkv, Hq, S):
     p.sync()
     p.assert_pools_equal()
     p.assert_tables_equal(live)
-    assert decoded_steps > 10 and reloaded > 0
+    assert decoded_steps > 10 and reloaded > 0 and ruled_steps > 5
