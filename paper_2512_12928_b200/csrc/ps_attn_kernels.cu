@@ -329,6 +329,11 @@ struct StageDesc {  // published by the producer next to every ring stage
     int32_t flags;  // kFlagFirst | kFlagLast | kFlagEnd
 };
 
+// Release / acquire fence at device scope: what publishing a partial result before announcing it, and reading
+// the other parts after finding them all announced, need.  (__threadfence() is the sequentially consistent
+// fence, which costs more and orders nothing more that this kernel relies on.)
+__device__ __forceinline__ void fence_acq_rel_gpu() { asm volatile("fence.acq_rel.gpu;" ::: "memory"); }
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -421,26 +426,20 @@ __device__ __forceinline__ void merge_row(int b, int h, int lane, const AttnBatc
                                           const float* __restrict__ partials, __nv_bfloat16* __restrict__ out,
                                           float* __restrict__ lse, int32_t* __restrict__ row_done) {
     constexpr int Hq = HKV * G;
-    __threadfence();
+    fence_acq_rel_gpu();
     const int n = batch.row_parts[b];
     const float* base = partials + ((int64_t)batch.row_first_part[b] * Hq + h * G) * kMmaPartStride;
     const int64_t stride = (int64_t)Hq * kMmaPartStride;   // floats between parts
-    // pass 1: per head the maximum over the parts (lanes stride over the parts)
+    // One pass over the parts, two at a time, with a running maximum per head (sums and accumulators are
+    // rescaled when it grows): every part is loaded once, the loads of a pair are issued together, and the
+    // chain of dependent round trips to L2 is half as long as with a separate pass for the maximum.  Lane owns
+    // dims [4 lane, 4 lane + 4) of every head.
     float M[G];
-#pragma unroll
-    for (int gg = 0; gg < G; ++gg) M[gg] = kNegBig;
-    for (int i = lane; i < n; i += 32)
-#pragma unroll
-        for (int gg = 0; gg < G; ++gg) M[gg] = fmaxf(M[gg], __ldcg(base + i * stride + gg * kMmaPartStride + kMmaD));
-#pragma unroll
-    for (int gg = 0; gg < G; ++gg)
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) M[gg] = fmaxf(M[gg], __shfl_xor_sync(0xffffffffu, M[gg], off));
-    // pass 2: lane owns dims [4 lane, 4 lane + 4) of every head
     float4 acc[G];
     float Ls[G];
 #pragma unroll
     for (int gg = 0; gg < G; ++gg) {
+        M[gg] = kNegBig;
         acc[gg] = make_float4(0.f, 0.f, 0.f, 0.f);
         Ls[gg] = 0.f;
     }
@@ -465,18 +464,16 @@ __device__ __forceinline__ void merge_row(int b, int h, int lane, const AttnBatc
         }
 #pragma unroll
         for (int gg = 0; gg < G; ++gg) {
-            const float wa = exp2f(ma[gg] - M[gg]);
-            const float wb = two ? exp2f(mb[gg] - M[gg]) : 0.f;
-            Ls[gg] = fmaf(la[gg], wa, Ls[gg]);
-            acc[gg].x = fmaf(va[gg].x, wa, acc[gg].x);
-            acc[gg].y = fmaf(va[gg].y, wa, acc[gg].y);
-            acc[gg].z = fmaf(va[gg].z, wa, acc[gg].z);
-            acc[gg].w = fmaf(va[gg].w, wa, acc[gg].w);
-            Ls[gg] = fmaf(lb[gg], wb, Ls[gg]);
-            acc[gg].x = fmaf(vb[gg].x, wb, acc[gg].x);
-            acc[gg].y = fmaf(vb[gg].y, wb, acc[gg].y);
-            acc[gg].z = fmaf(vb[gg].z, wb, acc[gg].z);
-            acc[gg].w = fmaf(vb[gg].w, wb, acc[gg].w);
+            const float m_new = fmaxf(M[gg], fmaxf(ma[gg], mb[gg]));
+            const float sc = exp2f(M[gg] - m_new);
+            const float wa = exp2f(ma[gg] - m_new);
+            const float wb = two ? exp2f(mb[gg] - m_new) : 0.f;
+            M[gg] = m_new;
+            Ls[gg] = fmaf(lb[gg], wb, fmaf(la[gg], wa, Ls[gg] * sc));
+            acc[gg].x = fmaf(vb[gg].x, wb, fmaf(va[gg].x, wa, acc[gg].x * sc));
+            acc[gg].y = fmaf(vb[gg].y, wb, fmaf(va[gg].y, wa, acc[gg].y * sc));
+            acc[gg].z = fmaf(vb[gg].z, wb, fmaf(va[gg].z, wa, acc[gg].z * sc));
+            acc[gg].w = fmaf(vb[gg].w, wb, fmaf(va[gg].w, wa, acc[gg].w * sc));
         }
     }
 #pragma unroll
@@ -577,6 +574,8 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
         int32_t* counter = sched + 2 * sched_lane;
         int it = item0;
         bool dynamic = false;
+        AttnItem pre_item{};   // descriptor and id windows of the CTA's next static item, fetched ahead
+        int pre_it = -1, pre_ids = 0, pre_ids_next = 0;
         while (ok) {
             if (!dynamic && it >= item1) dynamic = true;
             if (dynamic) {
@@ -587,15 +586,22 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                 it = dyn_begin + c;
                 if (it >= dyn_end) break;
             }
-            const AttnItem item = batch.items[it];
+            // A static item's descriptor and first block-id windows were fetched while the item before it was
+            // being streamed (below); otherwise they are fetched now, three dependent loads during which no
+            // copy is issued.
+            const bool primed = pre_it == it;
+            const AttnItem item = primed ? pre_item : batch.items[it];
             const int32_t* table = batch.block_tables + (int64_t)item.b * batch.table_stride;
             const int ntiles = max(1, (item.t_end - item.t_begin + kStageTokens - 1) / kStageTokens);
             // Block ids are read 32 at a time, one per lane, a window ahead of their use: the table read
             // never sits between a freed stage and the copies that refill it.
             const int last_blk = (max(item.t_end, 1) - 1) / block_size;
             int win = block_shift >= 0 ? (item.t_begin >> block_shift) : (item.t_begin / block_size);
-            int ids = win + lane <= last_blk ? __ldg(table + win + lane) : 0;
-            int ids_next = win + 32 + lane <= last_blk ? __ldg(table + win + 32 + lane) : 0;
+            int ids = primed ? pre_ids : (win + lane <= last_blk ? __ldg(table + win + lane) : 0);
+            int ids_next = primed ? pre_ids_next : (win + 32 + lane <= last_blk ? __ldg(table + win + 32 + lane) : 0);
+            pre_it = -1;
+            const bool prime_next = !dynamic && it + 1 < item1;
+            if (prime_next) pre_item = batch.items[it + 1];  // issued now, needed after this item's first copies
             for (int ti = 0; ti < ntiles; ++ti, ++n) {
                 const int s = n % kMmaStages;
                 const int t0 = item.t_begin + ti * kStageTokens;
@@ -652,6 +658,15 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                             bulk_g2s(dst, (lane < 16 ? kpool : vpool) + off, kMmaRowBytes, full, kv_policy);
                         }
                     }
+                }
+                if (prime_next && ti == min(1, ntiles - 1)) {
+                    // the next item's first two block-id windows, under the copies just issued
+                    const int32_t* ntable = batch.block_tables + (int64_t)pre_item.b * batch.table_stride;
+                    const int nlast = (max(pre_item.t_end, 1) - 1) / block_size;
+                    const int nwin = block_shift >= 0 ? (pre_item.t_begin >> block_shift) : (pre_item.t_begin / block_size);
+                    pre_ids = nwin + lane <= nlast ? __ldg(ntable + nwin + lane) : 0;
+                    pre_ids_next = nwin + 32 + lane <= nlast ? __ldg(ntable + nwin + 32 + lane) : 0;
+                    pre_it = it + 1;
                 }
             }
             if (!dynamic) ++it;
@@ -859,7 +874,10 @@ decode_attn_mma_kernel(const __nv_bfloat16* __restrict__ kpool, const __nv_bfloa
                     // Split-KV fix-up: the warp that delivers the last part of a (row, KV head) combines the
                     // parts.  Combining costs a few round trips to L2 during which this warp would hold up the
                     // CTA's ring, so the row is only noted here and combined after the CTA's last tile.
-                    __threadfence();
+                    // (Publishing and announcing the part right here costs two such round trips already, about
+                    // 3.5 us under full memory load; putting them off to the CTA's end as well was measured and is
+                    // worse: every row is then completed, and combined, in the launch's last microseconds.)
+                    fence_acq_rel_gpu();
                     __syncwarp();
                     int prev = 0;
                     if (lane == 0) prev = atomicAdd(row_done + item_b * HKV + h, 1);
