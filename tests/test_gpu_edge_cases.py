@@ -1,0 +1,142 @@
+"""GPU parity at the edges of the path: empty and maximal batches, budgets of zero and of less than one
+block, requests without blocks, a request at the table limit, a pool used to its last block."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2512_12928_b200 import binding as B
+from paper_2512_12928_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    from gpu_util import Pair, bits_to_dev, check_attn
+
+
+def make_pair(L, Hkv, Hq, D, S, nb, seed, **kw):
+    sh = wl.KVShape(L, Hkv, Hq, D, S, nb)
+    rng = np.random.default_rng(seed)
+    K = wl.randn_bf16_bits(rng, (L, nb, S, Hkv, D))
+    V = wl.randn_bf16_bits(rng, (L, nb, S, Hkv, D))
+    return sh, rng, Pair(sh, rng.permutation(nb), K, V, **kw)
+
+
+def test_empty_batch_and_budgets_below_one_block():
+    sh, rng, p = make_pair(3, 8, 32, 128, 16, 96, 11, max_batch=8)
+    for r, n in ((0, 40), (1, 16), (2, 100)):
+        assert p.both("kv_alloc", r, n) == B.PS_OK
+    assert p.both("swap_out", 2) == B.PS_OK
+    p.sync()
+    assert p.both("swap_in_begin", 2) == B.PS_OK
+    # an empty decode batch is legal: the step only moves the reload forward
+    q0 = torch.zeros((3, 0, 32, 128), dtype=torch.bfloat16, device="cuda")
+    assert p.lib.decode_attn(0, q0[0], q0[0], []) == B.PS_OK
+    for budget in (0, 1, sh.block_bytes - 1):            # floor(bytes / block bytes) = 0 blocks
+        rc, mask, st = p.lib.step(q0, q0, [], budget)
+        plan, omask, _ = p.orc.step(budget, [], None)
+        assert rc == B.PS_OK and mask == omask == [] and plan == [] and st["blocks_copied"] == 0
+    assert p.lib.missing_blocks(2) == p.orc.missing_blocks(2) == 7
+    # exactly one block per step, no decode rows: 7 steps bring the request back
+    for k in range(7):
+        rc, mask, st = p.lib.step(q0, q0, [], sh.block_bytes)
+        plan, _, _ = p.orc.step(sh.block_bytes, [], None)
+        assert rc == B.PS_OK and st["blocks_copied"] == 1 and plan == [(2, k, k + 1)]
+        assert st["reloads_completed"] == (1 if k == 6 else 0)
+    p.sync()
+    p.assert_pools_equal()
+    p.assert_tables_equal([0, 1, 2])
+    # a budget of zero with a decode batch: the queued request does not decode, the others do
+    assert p.both("swap_out", 1) == B.PS_OK
+    p.sync()
+    assert p.both("swap_in_begin", 1) == B.PS_OK
+    q = wl.randn_bf16_bits(rng, (3, 3, 32, 128))
+    qd = bits_to_dev(q)
+    out = torch.full_like(qd, 5.0)
+    rc, mask, st = p.lib.step(qd, out, [0, 1, 2], 0)
+    plan, omask, want = p.orc.step(0, [0, 1, 2], q)
+    assert rc == B.PS_OK and mask == omask == [1, 0, 1] and st["decoded"] == 2
+    p.sync()
+    check_attn(out[:, [0, 2]], want[:, [0, 2]])
+    assert (out[:, 1].float() == 5.0).all()
+    p.orc.check_invariants()
+
+
+def test_requests_without_blocks_go_out_and_come_back():
+    sh, rng, p = make_pair(2, 4, 8, 64, 16, 32, 12, max_batch=8)
+    assert p.both("kv_alloc", 0, 0) == B.PS_OK
+    assert p.both("kv_alloc", 1, 33) == B.PS_OK
+    assert p.both("swap_out", 0) == B.PS_OK              # nothing to copy
+    p.sync()
+    assert p.lib.block_table(0) == p.orc.block_table(0)
+    assert p.both("swap_in_begin", 0) == B.PS_OK         # nothing to restore: resident at once
+    assert p.lib.block_table(0) == p.orc.block_table(0)
+    assert p.lib.missing_blocks(0) == p.orc.missing_blocks(0) == 0
+    q = wl.randn_bf16_bits(rng, (2, 2, 8, 64))
+    qd = bits_to_dev(q)
+    out = torch.full_like(qd, 9.0)
+    rc, mask, st = p.lib.step(qd, out, [0, 1], -1)
+    plan, omask, want = p.orc.step(-1, [0, 1], q)
+    assert rc == B.PS_OK and mask == omask == [1, 1] and plan == []
+    p.sync()
+    check_attn(out, want)                                # the row without tokens is all zeros on both sides
+    assert (out[:, 0].float() == 0.0).all()
+    assert p.both("kv_free", 0) == B.PS_OK
+    p.orc.check_invariants()
+
+
+def test_request_at_the_table_limit_and_pool_used_to_the_last_block():
+    S, nb, cap = 16, 72, 40
+    sh, rng, p = make_pair(2, 8, 64, 128, S, nb, 13, max_batch=4, max_blocks_per_req=cap)
+    assert p.lib.kv_alloc(0, cap * S + 1) == B.PS_ERR_INVALID       # one token beyond the table limit
+    assert p.both("kv_alloc", 0, cap * S) == B.PS_OK                 # exactly at the limit
+    assert p.both("kv_alloc", 1, (nb - cap) * S) == B.PS_OK          # the pool's last block
+    assert p.lib.num_free_blocks() == p.orc.num_free_blocks() == 0
+    assert p.both("kv_alloc", 2, 1) == B.PS_ERR_NOMEM
+    q = wl.randn_bf16_bits(rng, (2, 2, 64, 128))
+    qd = bits_to_dev(q)
+    out = torch.zeros_like(qd)
+    rc, mask, _ = p.lib.step(qd, out, [0, 1], -1)
+    _, omask, want = p.orc.step(-1, [0, 1], q)
+    assert rc == B.PS_OK and mask == omask == [1, 1]
+    p.sync()
+    check_attn(out, want)
+    # with no free block a readmission is refused and changes nothing; after an eviction it goes through
+    assert p.both("swap_out", 0) == B.PS_OK
+    p.sync()
+    assert p.both("kv_alloc", 2, (cap - 1) * S) == B.PS_OK
+    assert p.both("swap_in_begin", 0) == B.PS_ERR_NOMEM
+    p.assert_tables_equal([0, 1, 2])
+    assert p.both("kv_free", 2) == B.PS_OK
+    assert p.both("swap_in_begin", 0) == B.PS_OK
+    out2 = torch.zeros_like(qd)
+    rc, mask, st = p.lib.step(qd, out2, [0, 1], -1)
+    _, omask, want2 = p.orc.step(-1, [0, 1], q)
+    assert rc == B.PS_OK and mask == omask == [1, 1] and st["blocks_copied"] == cap
+    p.sync()
+    p.assert_pools_equal()
+    check_attn(out2, want2)
+    assert torch.equal(out, out2)                                    # the same bytes in other blocks
+    p.orc.check_invariants()
+
+
+@pytest.mark.parametrize("Hkv,Hq,D,kernel", [(8, 32, 128, B.PS_ATTN_MMA), (4, 8, 64, B.PS_ATTN_SIMT)])
+def test_batch_of_the_maximum_size_with_one_token_rows(Hkv, Hq, D, kernel):
+    """256 rows (the largest batch a context takes), most of one token: more rows than work items per CTA."""
+    S, nbatch = 16, 256
+    sh, rng, p = make_pair(1, Hkv, Hq, D, S, 400, [14, Hkv], max_batch=nbatch, attn_kernel=kernel)
+    ctxs = [1] * nbatch
+    ctxs[7], ctxs[100], ctxs[255] = 5 * S + 3, 2 * S, 64 * S - 1
+    for r, c in enumerate(ctxs):
+        assert p.both("kv_alloc", r, c) == B.PS_OK
+    reqs = list(range(nbatch))
+    q = wl.randn_bf16_bits(rng, (1, nbatch, Hq, D))
+    qd = bits_to_dev(q)
+    out = torch.zeros_like(qd)
+    rc, mask, st = p.lib.step(qd, out, reqs, -1)
+    _, omask, want = p.orc.step(-1, reqs, q)
+    assert rc == B.PS_OK and mask == omask and st["decoded"] == nbatch
+    p.sync()
+    check_attn(out, want)
+    # one row more than the context was created for is refused before any launch
+    big = torch.zeros((1, nbatch + 1, Hq, D), dtype=torch.bfloat16, device="cuda")
+    assert p.lib.decode_attn(0, big[0], big[0], reqs + [0]) == B.PS_ERR_INVALID
