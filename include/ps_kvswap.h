@@ -164,7 +164,10 @@ typedef struct ps_trace_span {
 int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_pools, void* host_pool,
                   void* compute_stream, ps_ctx** out);
 
-/* Waits for the context's outstanding work (bounded), then frees everything it owns. */
+/* Waits up to 10 s for the context's outstanding work (as ps_sync does); if that runs out, waits for its
+ * streams and the compute stream without a limit, so that no staging slot or pinned range is freed under a
+ * copy still queued.  Frees everything the context owns either way; returns PS_ERR_TIMEOUT if the bounded
+ * wait ran out, else PS_OK.  The pools and the compute stream stay the caller's. */
 int32_t ps_destroy(ps_ctx* ctx);
 
 /* Text of the most recent error of this context (static storage inside the context; never NULL).

@@ -257,6 +257,17 @@ void destroy_ctx(ps_ctx* ctx) {
         ctx->out_thread.join();
     }
     if (!ctx->bk) {
+        // If the caller's bounded wait ran out, copies into the staging slots and the pinned pool may still be
+        // queued (the worker, joined above, issues none any more): nothing is freed under them.  What is left
+        // is finite (transfers, and kernels whose own waits are bounded), so the streams are waited for here
+        // without a limit; on an idle context this costs nothing.
+        bool any_stream = false;
+        for (cudaStream_t s : {ctx->s_gather, ctx->s_d2h, ctx->s_h2d, ctx->s_scatter, ctx->s_lane})
+            if (s) {
+                cudaStreamSynchronize(s);
+                any_stream = true;
+            }
+        if (any_stream) cudaStreamSynchronize(ctx->compute);
         for (cudaStream_t s : {ctx->s_gather, ctx->s_d2h, ctx->s_h2d, ctx->s_scatter, ctx->s_lane})
             if (s) cudaStreamDestroy(s);
         for (int i = 0; i < kSlots; ++i)
@@ -534,11 +545,12 @@ int32_t ps_create(const ps_config* cfg, void* const* k_pools, void* const* v_poo
 
 int32_t ps_destroy(ps_ctx* ctx) {
     if (!ctx) return PS_ERR_INVALID;
+    int32_t rc = PS_OK;
     if (!ctx->bk) {
-        ps_sync(ctx, 10000);
+        rc = ps_sync(ctx, 10000);
     }
     destroy_ctx(ctx);
-    return PS_OK;
+    return rc == PS_ERR_TIMEOUT ? PS_ERR_TIMEOUT : PS_OK;
 }
 
 int32_t ps_kv_alloc(ps_ctx* ctx, int64_t req, int32_t n_tokens_total) {
