@@ -140,3 +140,53 @@ def test_batch_of_the_maximum_size_with_one_token_rows(Hkv, Hq, D, kernel):
     # one row more than the context was created for is refused before any launch
     big = torch.zeros((1, nbatch + 1, Hq, D), dtype=torch.bfloat16, device="cuda")
     assert p.lib.decode_attn(0, big[0], big[0], reqs + [0]) == B.PS_ERR_INVALID
+
+
+def test_two_contexts_of_different_shapes_interleaved():
+    """Two live contexts (different shapes, kernels and staging sizes) driven in turn: nothing is shared."""
+    sh_a, rng_a, a = make_pair(3, 8, 32, 128, 16, 128, 21, max_batch=8, staging_bytes=1 << 20)
+    sh_b, rng_b, b = make_pair(2, 4, 8, 64, 16, 96, 22, max_batch=8)
+    ctx_a, ctx_b = [300, 77, 512, 16], [40, 200, 129]
+    for r, n in enumerate(ctx_a):
+        assert a.both("kv_alloc", r, n) == B.PS_OK
+    for r, n in enumerate(ctx_b):
+        assert b.both("kv_alloc", r, n) == B.PS_OK
+    qa = wl.randn_bf16_bits(rng_a, (3, 4, 32, 128))
+    qb = wl.randn_bf16_bits(rng_b, (2, 3, 8, 64))
+    qa_d, qb_d = bits_to_dev(qa), bits_to_dev(qb)
+    assert a.both("swap_out", 2) == B.PS_OK
+    assert b.both("swap_out", 1) == B.PS_OK
+    assert a.both("swap_out", 0) == B.PS_OK
+    a.sync()
+    b.sync()
+    for r in (2, 0):
+        assert a.both("swap_in_begin", r) == B.PS_OK
+    assert b.both("swap_in_begin", 1) == B.PS_OK
+    budget_a, budget_b = 9 * sh_a.block_bytes, 4 * sh_b.block_bytes
+    for _ in range(8):
+        oa = torch.full_like(qa_d, 2.0)
+        ob = torch.full_like(qb_d, 2.0)
+        rc_a, mask_a, _ = a.lib.step(qa_d, oa, [0, 1, 2, 3], budget_a)      # both steps in flight together
+        rc_b, mask_b, _ = b.lib.step(qb_d, ob, [0, 1, 2], budget_b)
+        assert rc_a == B.PS_OK and rc_b == B.PS_OK
+        _, want_mask_a, want_a = a.orc.step(budget_a, [0, 1, 2, 3], qa)
+        _, want_mask_b, want_b = b.orc.step(budget_b, [0, 1, 2], qb)
+        assert mask_a == want_mask_a and mask_b == want_mask_b
+        a.sync()
+        b.sync()
+        la = [i for i, m in enumerate(mask_a) if m]
+        lb = [i for i, m in enumerate(mask_b) if m]
+        check_attn(oa[:, la], want_a[:, la])
+        check_attn(ob[:, lb], want_b[:, lb])
+    assert mask_a == [1, 1, 1, 1] and mask_b == [1, 1, 1]
+    a.assert_pools_equal()
+    b.assert_pools_equal()
+    a.assert_tables_equal([0, 1, 2, 3])
+    b.assert_tables_equal([0, 1, 2])
+    a.lib.destroy()                                   # one context goes, the other keeps working
+    ob = torch.zeros_like(qb_d)
+    rc_b, mask_b, _ = b.lib.step(qb_d, ob, [0, 1, 2], 0)
+    _, _, want_b = b.orc.step(0, [0, 1, 2], qb)
+    assert rc_b == B.PS_OK
+    b.sync()
+    check_attn(ob, want_b)
