@@ -27,7 +27,10 @@ def test_random_script_with_data(seed, Hkv, Hq, S):
     rng = np.random.default_rng([2512, seed])
     K = wl.randn_bf16_bits(rng, (L, nb, S, Hkv, D))
     V = wl.randn_bf16_bits(rng, (L, nb, S, Hkv, D))
+    # host pool of twice what 8 live requests of 64 blocks can hold (proactive copies of residents included):
+    # the checker has no host limit, so the library's must never bind here
     p = Pair(sh, rng.permutation(nb), K, V, max_batch=12, staging_bytes=2 << 20, max_blocks_per_req=64,
+             host_pool_bytes=1024 * sh.block_bytes,
              layer_chunk_bytes=[0, -1, 96 * 1024, 1 << 30][seed % 4])
     live, next_id = [], 0
     decoded_steps = reloaded = ruled_steps = reaped_by_steps = 0
