@@ -1042,12 +1042,12 @@ def run_gpu(args):
     time_decode_steps(torch, lib, residents, q_res, out_res, 2)
     rf_res = decode_roofline(torch, lib, sh, w.ctx_lens, residents, q_res, out_res, steps=5)
     rf_single = single_launch_rate(torch, lib, sh, w.ctx_lens, all_reqs, q, out)
-    # the same with PS_FLAG_ATTN_EARLY_SETUP: each launch is scheduled and set up under its predecessor's tail
+    # the same with PS_FLAG_ATTN_PLAIN_LAUNCH: no set-up under the predecessor's tail (the default has it)
     elib = make_ctx(B, w, K, V, sh.num_gpu_blocks, max_batch=nreq, host_pool_bytes=64 << 20,
-                    flags=B.PS_FLAG_ATTN_EARLY_SETUP)
+                    flags=B.PS_FLAG_ATTN_PLAIN_LAUNCH)
     for r, n in wl.build_order_round_robin(w):
         assert elib.kv_alloc(r, n) == 0, elib.last_error()
-    rf_single_early = single_launch_rate(torch, elib, sh, w.ctx_lens, all_reqs, q, out)
+    rf_single_plain = single_launch_rate(torch, elib, sh, w.ctx_lens, all_reqs, q, out)
     elib.destroy()
     del elib
     clocks = sampler.stop()
@@ -1103,9 +1103,9 @@ def run_gpu(args):
             "single_launch_gbs": rf_single["gbs"], "single_launch_us": rf_single["us_per_launch"],
             "single_launch_frac": rf_single["gbs"] / hbm_peak,
             "single_launch_frac_of_read_peak": rf_single["gbs"] / read_peak,
-            "single_launch_early_setup_gbs": rf_single_early["gbs"],
-            "single_launch_early_setup_us": rf_single_early["us_per_launch"],
-            "single_launch_early_setup_frac": rf_single_early["gbs"] / hbm_peak,
+            "single_launch_plain_gbs": rf_single_plain["gbs"],
+            "single_launch_plain_us": rf_single_plain["us_per_launch"],
+            "single_launch_plain_frac": rf_single_plain["gbs"] / hbm_peak,
             "residents48_gbs": rf_res["gbs"], "residents48_us_per_launch": rf_res["us_per_layer"],
         }
         result["swap"] = {

@@ -79,13 +79,14 @@ enum ps_flags {
     /* Ablation (Section 5, block-management ablation "w/o async"): ps_step finishes the whole
        reload before the first attention launch instead of pipelining it layer by layer. */
     PS_FLAG_SYNC_RELOAD = 4,
-    /* ps_decode_attn (one layer per call) launches the tensor-core kernel programmatically dependent on the
-       kernel that precedes it on the compute stream: its CTAs are scheduled and set up under that kernel's
-       tail and wait for its completion before they read the queries, the KV pools or the batch metadata.
-       Results are unchanged after any predecessor; time is gained only after kernels that let dependents
-       start early (this library's attention kernel does; an engine's own kernels may, with
-       cudaTriggerProgrammaticLaunchCompletion). */
-    PS_FLAG_ATTN_EARLY_SETUP = 8
+    /* By default ps_decode_attn (one layer per call) launches the tensor-core kernel programmatically
+       dependent on the kernel that precedes it on the compute stream: its CTAs are scheduled and set up
+       under that kernel's tail and wait for its completion before they read the queries, the KV pools or the
+       batch metadata.  Results are the same after any predecessor; time is gained only after kernels that
+       let dependents start early (this library's attention kernel does; an engine's own kernels may, with
+       cudaTriggerProgrammaticLaunchCompletion).  This flag turns that off: an ordinary launch, for
+       comparison and diagnosis. */
+    PS_FLAG_ATTN_PLAIN_LAUNCH = 8
 };
 
 enum ps_attn_kernel {

@@ -22,7 +22,7 @@ LIB_PATH = os.environ.get("PS_KVSWAP_LIB") or os.path.join(_PKG, "lib", "libps_k
 PS_OK, PS_ERR_INVALID, PS_ERR_NOMEM, PS_ERR_HOST_NOMEM = 0, -1, -2, -3
 PS_ERR_STATE, PS_ERR_BUSY, PS_ERR_TIMEOUT, PS_ERR_CUDA, PS_ERR_BOUNDS = -4, -5, -6, -7, -8
 PS_REQ_NONE, PS_REQ_RESIDENT, PS_REQ_SWAPPING_OUT, PS_REQ_HOST, PS_REQ_SWAPPING_IN = 0, 1, 2, 3, 4
-PS_FLAG_BOOKKEEPING_ONLY, PS_FLAG_PROFILE, PS_FLAG_SYNC_RELOAD, PS_FLAG_ATTN_EARLY_SETUP = 1, 2, 4, 8
+PS_FLAG_BOOKKEEPING_ONLY, PS_FLAG_PROFILE, PS_FLAG_SYNC_RELOAD, PS_FLAG_ATTN_PLAIN_LAUNCH = 1, 2, 4, 8
 PS_ATTN_AUTO, PS_ATTN_SIMT, PS_ATTN_MMA, PS_ATTN_MMA_ROWS = 0, 1, 2, 3
 
 EXPORTS = [

@@ -327,7 +327,7 @@ int32_t launch_layer_attn(ps_ctx* ctx, int32_t layer, const void* q, void* out, 
         const bool overlap = follows_own && mma && !ctx->profile && m.dev.n_cta[0] == ctx->num_sms;
         // one layer per call: the caller's kernels sit between the launches, so only the set-up may run early
         const bool early_setup = !follows_own && mma && !ctx->profile && wait_event == nullptr &&
-                                 (ctx->cfg.flags & PS_FLAG_ATTN_EARLY_SETUP) != 0;
+                                 (ctx->cfg.flags & PS_FLAG_ATTN_PLAIN_LAUNCH) == 0;
         const int set = ctx->scratch_set;
         ctx->scratch_set ^= 1;
         const int64_t bytes = m.kv_bytes_per_layer * m.n_ungated_items / m.n_items;

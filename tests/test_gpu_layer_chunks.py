@@ -220,13 +220,14 @@ def test_attention_recovers_after_a_kernel_side_timeout_report():
     assert p.lib.sync() == B.PS_OK
 
 
-def test_attention_with_early_set_up_matches_after_any_predecessor():
-    """PS_FLAG_ATTN_EARLY_SETUP: one-layer-per-call launches are programmatically dependent on the kernel before
-    them and wait for it before reading any input.  Back to back (the predecessor is the same kernel, which lets
+@pytest.mark.parametrize("flags", [0, B.PS_FLAG_ATTN_PLAIN_LAUNCH])
+def test_attention_with_early_set_up_matches_after_any_predecessor(flags):
+    """One-layer-per-call launches are by default programmatically dependent on the kernel before them and wait
+    for it before reading any input (PS_FLAG_ATTN_PLAIN_LAUNCH: ordinary launches).  Back to back (the predecessor is the same kernel, which lets
     dependents start early), after another library's kernel that produces the queries, and after a table
     change (the predecessor is the metadata upload): results equal the checker's every time."""
     sh, rng, p = build_pair(4, 420, 59, Hkv=8, Hq=32, D=128, max_batch=8, max_blocks_per_req=64,
-                            attn_kernel=B.PS_ATTN_MMA, flags=B.PS_FLAG_ATTN_EARLY_SETUP)
+                            attn_kernel=B.PS_ATTN_MMA, flags=flags)
     tokens = [700, 33, 720, 512, 1, 705]
     reqs = list(range(len(tokens)))
     for r, n in enumerate(tokens):
