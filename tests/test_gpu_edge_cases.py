@@ -190,3 +190,44 @@ def test_two_contexts_of_different_shapes_interleaved():
     assert rc_b == B.PS_OK
     b.sync()
     check_attn(ob, want_b)
+
+
+@pytest.mark.parametrize("Hkv,Hq,D,S,kernel", [(8, 32, 128, 16, B.PS_ATTN_MMA), (8, 64, 128, 32, B.PS_ATTN_MMA_ROWS),
+                                               (4, 28, 128, 32, B.PS_ATTN_MMA), (1, 8, 128, 48, B.PS_ATTN_MMA),
+                                               (4, 8, 64, 16, B.PS_ATTN_SIMT), (8, 32, 128, 16, B.PS_ATTN_SIMT)])
+def test_non_finite_leftovers_past_a_context_end_do_not_reach_the_output(Hkv, Hq, D, S, kernel):
+    """Slots of a request's last block beyond its context, and every block it does not own, hold NaN and
+    infinity patterns in K and V: the output must be what the checker computes from the first ctx tokens."""
+    L, nb = 1, 96
+    sh, rng, p = make_pair(L, Hkv, Hq, D, S, nb, [15, Hkv, S], max_batch=8, attn_kernel=kernel, kv_split_tokens=3 * S)
+    ctxs = [1, S - 1, S + 1, 5 * S + 7, 9 * S - 1, 2 * S]
+    for r, c in enumerate(ctxs):
+        assert p.both("kv_alloc", r, c) == B.PS_OK
+    poison = np.array([0x7FC0, 0x7F80, 0xFF80, 0xFFC1], np.uint16)        # NaN, +inf, -inf, another NaN
+    owned = set()
+    for r, c in enumerate(ctxs):
+        table = p.orc.block_table(r)[0]
+        owned.update(table)
+        used = c - (len(table) - 1) * S                                     # tokens in the last block
+        if used < S:
+            fill = poison[rng.integers(0, 4, size=(S - used, Hkv, D))]
+            for pool_d, pool_o in ((p.Kd, p.orc.K), (p.Vd, p.orc.V)):
+                pool_o[0, table[-1], used:] = fill
+                pool_d[0, table[-1], used:] = bits_to_dev(fill)
+    foreign = [b for b in range(nb) if b not in owned]
+    fill = poison[rng.integers(0, 4, size=(len(foreign), S, Hkv, D))]
+    for pool_d, pool_o in ((p.Kd, p.orc.K), (p.Vd, p.orc.V)):
+        pool_o[0, foreign] = fill
+        pool_d[0, foreign] = bits_to_dev(fill)
+    reqs = list(range(len(ctxs)))
+    q = wl.randn_bf16_bits(rng, (L, len(reqs), Hq, D))
+    qd = bits_to_dev(q)
+    out = torch.zeros_like(qd)
+    lse = torch.zeros((len(reqs), Hq), dtype=torch.float32, device="cuda")
+    assert p.lib.decode_attn(0, qd[0], out[0], reqs, lse) == B.PS_OK, p.lib.last_error()
+    assert p.lib.sync() == B.PS_OK, p.lib.last_error()
+    want, wlse = p.orc.decode_attn(0, q[0], reqs)
+    assert np.isfinite(want).all()
+    assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
+    check_attn(out[0], want)
+    assert np.max(np.abs(lse.double().cpu().numpy() - wlse)) < 1e-3
