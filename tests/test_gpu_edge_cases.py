@@ -231,3 +231,46 @@ def test_non_finite_leftovers_past_a_context_end_do_not_reach_the_output(Hkv, Hq
     assert torch.isfinite(out.float()).all() and torch.isfinite(lse).all()
     check_attn(out[0], want)
     assert np.max(np.abs(lse.double().cpu().numpy() - wlse)) < 1e-3
+
+
+@pytest.mark.parametrize("Hkv,Hq,D,S,kernel,split", [(8, 32, 128, 16, B.PS_ATTN_MMA, 0), (8, 64, 128, 32, B.PS_ATTN_MMA_ROWS, 0),
+                                                     (2, 16, 128, 16, B.PS_ATTN_MMA, 0), (4, 8, 64, 16, B.PS_ATTN_SIMT, 48),
+                                                     (8, 32, 128, 16, B.PS_ATTN_SIMT, 64)])
+def test_peaked_and_flat_softmax_with_large_logits(Hkv, Hq, D, S, kernel, split):
+    """Logits of magnitude in the hundreds.  Request 0: q and K eight times the usual scale, so each head's
+    weights collapse onto a few tokens and the running maximum jumps by hundreds between tiles and between
+    the parts of a split row.  Request 1: every key equals -6 q of its head's first query, so that query's
+    logits are one large negative constant and its output is the plain mean of V."""
+    L, nb = 1, 128
+    sh, rng, p = make_pair(L, Hkv, Hq, D, S, nb, [16, Hkv, D], max_batch=4, attn_kernel=kernel, kv_split_tokens=split)
+    G = Hq // Hkv
+    n0, n1 = 37 * S + 5, 21 * S - 2
+    assert p.both("kv_alloc", 0, n0) == B.PS_OK
+    assert p.both("kv_alloc", 1, n1) == B.PS_OK
+    from oracle.ps_oracle import bf16_bits_to_f64
+    q = wl.randn_bf16_bits(rng, (L, 2, Hq, D))
+    q[0, 0] = wl.f32_to_bf16_bits((8.0 * bf16_bits_to_f64(q[0, 0])).astype(np.float32))
+    t0 = p.orc.block_table(0)[0]
+    big = wl.f32_to_bf16_bits((8.0 * rng.standard_normal((len(t0), S, Hkv, D))).astype(np.float32))
+    p.orc.K[0, t0] = big
+    p.Kd[0, t0] = bits_to_dev(big)
+    t1 = p.orc.block_table(1)[0]
+    qf = bf16_bits_to_f64(q[0, 1])
+    for h in range(Hkv):
+        kb = wl.f32_to_bf16_bits((-6.0 * qf[h * G]).astype(np.float32))
+        p.orc.K[0, t1, :, h] = kb
+        p.Kd[0, t1, :, h] = bits_to_dev(kb)
+    qd = bits_to_dev(q)
+    out = torch.zeros_like(qd)
+    lse = torch.zeros((2, Hq), dtype=torch.float32, device="cuda")
+    assert p.lib.decode_attn(0, qd[0], out[0], [0, 1], lse) == B.PS_OK, p.lib.last_error()
+    assert p.lib.sync() == B.PS_OK
+    want, wlse = p.orc.decode_attn(0, q[0], [0, 1])
+    check_attn(out[0], want, rel_l2=2e-2)
+    got_lse = lse.double().cpu().numpy()
+    assert np.max(np.abs(got_lse - wlse) / np.maximum(1.0, np.abs(wlse))) < 2e-3
+    assert np.abs(wlse[0]).max() > 100 and wlse[1].min() < -30          # the logits really are large
+    Vf = bf16_bits_to_f64(p.orc.V[0])
+    for h in range(Hkv):                                                 # flat rows: the mean of the value rows
+        rows = np.concatenate([Vf[b, :, h] for b in t1])[:n1]
+        assert np.max(np.abs(want[1, h * G] - rows.mean(0))) < 1e-9
