@@ -1041,6 +1041,9 @@ def run_gpu(args):
     rf_all = decode_roofline(torch, lib, sh, w.ctx_lens, all_reqs, q, out, steps=5)
     time_decode_steps(torch, lib, residents, q_res, out_res, 2)
     rf_res = decode_roofline(torch, lib, sh, w.ctx_lens, residents, q_res, out_res, steps=5)
+    # the same kernel over half a second of decode-only steps: the board reaches its power cap and the SM clock
+    # settles lower than in the burst above
+    rf_sust = decode_roofline(torch, lib, sh, w.ctx_lens, all_reqs, q, out, steps=150)
     rf_single = single_launch_rate(torch, lib, sh, w.ctx_lens, all_reqs, q, out)
     # the same with PS_FLAG_ATTN_PLAIN_LAUNCH: no set-up under the predecessor's tail (the default has it)
     elib = make_ctx(B, w, K, V, sh.num_gpu_blocks, max_batch=nreq, host_pool_bytes=64 << 20,
@@ -1107,6 +1110,8 @@ def run_gpu(args):
             "single_launch_plain_us": rf_single_plain["us_per_launch"],
             "single_launch_plain_frac": rf_single_plain["gbs"] / hbm_peak,
             "residents48_gbs": rf_res["gbs"], "residents48_us_per_launch": rf_res["us_per_layer"],
+            "sustained_150_steps_gbs": rf_sust["gbs"], "sustained_150_steps_us_per_launch": rf_sust["us_per_layer"],
+            "sustained_150_steps_frac": rf_sust["gbs"] / hbm_peak,
         }
         result["swap"] = {
             "swap_out_gbs": victim_bytes * args.steps / out_ms / 1e6, "swap_in_gbs": victim_bytes * args.steps / in_ms / 1e6,
