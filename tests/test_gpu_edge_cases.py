@@ -274,3 +274,58 @@ def test_peaked_and_flat_softmax_with_large_logits(Hkv, Hq, D, S, kernel, split)
     for h in range(Hkv):                                                 # flat rows: the mean of the value rows
         rows = np.concatenate([Vf[b, :, h] for b in t1])[:n1]
         assert np.max(np.abs(want[1, h * G] - rows.mean(0))) < 1e-9
+
+
+def test_destroy_with_an_offload_and_a_reload_in_flight():
+    """ps_destroy right behind ps_swap_out / a budgeted step, without a sync in between: it waits for the
+    transfers itself, the pools stay intact, and a new context over the same pools works at once."""
+    L, Hkv, Hq, D, S, nb = 8, 8, 32, 128, 16, 1200
+    sh = wl.KVShape(L, Hkv, Hq, D, S, nb)
+    g = torch.Generator(device="cuda"); g.manual_seed(17)
+    K = torch.empty((L, nb, S, Hkv, D), dtype=torch.bfloat16, device="cuda").normal_(generator=g)
+    V = torch.empty_like(K).normal_(generator=g)
+    K0, V0 = K.clone(), V.clone()
+
+    def ctx():
+        return B.KVSwap(num_layers=L, num_kv_heads=Hkv, num_q_heads=Hq, head_dim=D, block_size=S, num_gpu_blocks=nb,
+                        max_blocks_per_req=1024, max_batch=4, host_pool_bytes=(1024 + 64) * sh.block_bytes,
+                        k_pools=[K[l] for l in range(L)], v_pools=[V[l] for l in range(L)])
+
+    lib = ctx()
+    assert lib.kv_alloc(1, 1000 * S) == B.PS_OK            # 1000 blocks x 512 KiB = 500 MiB of KV
+    assert lib.kv_alloc(2, 100 * S) == B.PS_OK
+    assert lib.swap_out(1) == B.PS_OK
+    lib.destroy()                                           # offload in flight
+    lib = ctx()
+    assert lib.kv_alloc(1, 1000 * S) == B.PS_OK
+    old = torch.tensor(lib.block_table(1)[0], device="cuda", dtype=torch.long)
+    assert lib.swap_out(1) == B.PS_OK
+    assert lib.sync() == B.PS_OK
+    assert torch.equal(K, K0) and torch.equal(V, V0)        # offloading reads the pools only
+    assert lib.swap_in_begin(1) == B.PS_OK
+    new = torch.tensor(lib.block_table(1)[0], device="cuda", dtype=torch.long)
+    K[:, new] = 0                                           # the fresh blocks hold nothing yet
+    V[:, new] = 0
+    rc, _, st = lib.step(None, None, [], 600 * sh.block_bytes)
+    assert rc == B.PS_OK and st["blocks_copied"] == 600
+    lib.destroy()                                           # reload in flight: destroy waits for it
+    torch.cuda.synchronize()
+    assert torch.equal(K[:, new[:600]], K0[:, old[:600]]) and torch.equal(V[:, new[:600]], V0[:, old[:600]])
+    assert not K[:, new[600:]].any() and not V[:, new[600:]].any()       # nothing written beyond the budget
+    rest = torch.ones(nb, dtype=torch.bool, device="cuda")
+    rest[new] = False
+    assert torch.equal(K[:, rest], K0[:, rest]) and torch.equal(V[:, rest], V0[:, rest])
+    lib = ctx()
+    assert lib.kv_alloc(5, 300 * S + 3) == B.PS_OK
+    q = torch.randn((Hq, D), generator=g, device="cuda").to(torch.bfloat16).unsqueeze(0)
+    out = torch.zeros_like(q)
+    assert lib.decode_attn(0, q, out, [5]) == B.PS_OK
+    assert lib.sync() == B.PS_OK
+    ids = torch.tensor(lib.block_table(5)[0], device="cuda", dtype=torch.long)
+    kk = K[0][ids].reshape(-1, Hkv, D)[: 300 * S + 3].float()
+    vv = V[0][ids].reshape(-1, Hkv, D)[: 300 * S + 3].float()
+    G = Hq // Hkv
+    sc = torch.einsum("hd,thd->ht", q[0].float(), kk.repeat_interleave(G, dim=1)) / D ** 0.5
+    ref = torch.einsum("ht,thd->hd", torch.softmax(sc, dim=-1), vv.repeat_interleave(G, dim=1))
+    assert (out[0].float() - ref).abs().max() < 2e-2
+    lib.destroy()
