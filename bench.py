@@ -1115,6 +1115,7 @@ def run_gpu(args):
         }
         result["swap"] = {
             "swap_out_gbs": victim_bytes * args.steps / out_ms / 1e6, "swap_in_gbs": victim_bytes * args.steps / in_ms / 1e6,
+            "out_ms_per_step": [round(r["out_ms"], 2) for r in recs], "in_ms_per_step": [round(r["in_ms"], 2) for r in recs],
             "swap_out_frac_of_link": victim_bytes * args.steps / out_ms / 1e6 / link["d2h_gbs"],
             "swap_in_frac_of_link": victim_bytes * args.steps / in_ms / 1e6 / link["h2d_gbs"],
             "decode_steps_during_out": recs[-1]["steps_out"], "decode_steps_during_in": recs[-1]["steps_in"],
